@@ -1,0 +1,164 @@
+"""ctypes binding of ``libmoc.so``.  Same names as the C entry points (include/moc.h);
+argument marshalling only.  torch supplies device memory and the stream."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_DIR = os.path.dirname(os.path.abspath(__file__))
+FLAG_CAUSAL = 0x1
+FLAG_SCALAR_ATTEND = 0x2
+WHOLE_SHOT = -1
+
+
+class MocError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(what)
+        self.code = code
+
+
+class _Problem(C.Structure):
+    _fields_ = [("n_heads", C.c_int32), ("n_tokens", C.c_int32), ("head_dim", C.c_int32),
+                ("n_chunks", C.c_int32), ("top_k", C.c_int32), ("win_back", C.c_int32), ("win_fwd", C.c_int32),
+                ("flags", C.c_uint32), ("softmax_scale", C.c_float),
+                ("chunk_off", C.c_void_p), ("chunk_shot", C.c_void_p), ("chunk_mod", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return os.path.join(_DIR, "libmoc.so")
+
+
+def load_library():
+    """dlopen the CUDA library.  Raises if it has not been built: nothing else can run the path."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = lib_path()
+    if not os.path.exists(path):
+        raise MocError(-100, f"{path} is missing: build it with `python -m paper_2508_21058_b200.build` "
+                             "(there is no fallback implementation)")
+    lib = C.CDLL(path)
+    vp, i32, sz = C.c_void_p, C.c_int, C.c_size_t
+    lib.moc_plan_create.argtypes = [C.POINTER(_Problem), C.POINTER(vp)]
+    lib.moc_plan_destroy.argtypes = [vp]
+    lib.moc_workspace_bytes.argtypes = [vp, i32, C.POINTER(sz)]
+    lib.moc_chunk_pool.argtypes = [vp, vp, vp, vp, vp]
+    lib.moc_route.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.moc_attend.argtypes = [vp] * 9
+    lib.moc_attend_bwd.argtypes = [vp] * 13
+    lib.moc_selected_pairs.argtypes = [vp, vp, vp, C.POINTER(C.c_int64)]
+    lib.moc_get_status.argtypes = [vp, vp, vp, C.POINTER(i32), C.POINTER(i32)]
+    lib.moc_launch_count.restype = C.c_int64
+    lib.moc_strerror.restype = C.c_char_p
+    lib.moc_strerror.argtypes = [i32]
+    lib.moc_last_cuda_error.restype = C.c_char_p
+    _lib = lib
+    return lib
+
+
+def launch_count() -> int:
+    return int(load_library().moc_launch_count())
+
+
+def _check(code: int):
+    if code != 0:
+        lib = load_library()
+        msg = lib.moc_strerror(code).decode()
+        if code == -7:
+            msg += ": " + lib.moc_last_cuda_error().decode()
+        raise MocError(code, f"moc error {code}: {msg}")
+
+
+def _ptr(t):
+    return C.c_void_p(0) if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class MocPlan:
+    """Owns a ``moc_plan``.  Methods mirror the C entry points and take torch CUDA tensors."""
+
+    def __init__(self, n_heads, n_tokens, head_dim, chunk_off, chunk_shot, chunk_mod, top_k,
+                 win_back=0, win_fwd=0, causal=True, scalar_attend=False, softmax_scale=0.0):
+        self._lib = load_library()
+        self._h = C.c_void_p(0)
+        off = np.ascontiguousarray(chunk_off, np.int32)
+        shot = np.ascontiguousarray(chunk_shot, np.int32)
+        mod = np.ascontiguousarray(chunk_mod, np.uint8)
+        flags = (FLAG_CAUSAL if causal else 0) | (FLAG_SCALAR_ATTEND if scalar_attend else 0)
+        pr = _Problem(int(n_heads), int(n_tokens), int(head_dim), len(shot), int(top_k), int(win_back), int(win_fwd),
+                      flags, float(softmax_scale), off.ctypes.data, shot.ctypes.data, mod.ctypes.data)
+        if len(off) != len(shot) + 1 or len(mod) != len(shot):
+            raise MocError(-3, "moc error -3: chunk tables have inconsistent lengths")
+        _check(self._lib.moc_plan_create(C.byref(pr), C.byref(self._h)))
+        self.H, self.L, self.d, self.C, self.k = int(n_heads), int(n_tokens), int(head_dim), len(shot), int(top_k)
+
+    @classmethod
+    def from_workload(cls, wl, n_heads=None, **kw):
+        lay = wl.layout
+        return cls(wl.n_heads if n_heads is None else n_heads, lay.n_tokens, wl.head_dim, lay.chunk_off,
+                   lay.chunk_shot, lay.chunk_mod, wl.top_k, wl.win_back, wl.win_fwd, wl.causal, **kw)
+
+    def close(self):
+        if self._h:
+            self._lib.moc_plan_destroy(self._h)
+            self._h = C.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def workspace_bytes(self, with_bwd=False) -> int:
+        n = C.c_size_t(0)
+        _check(self._lib.moc_workspace_bytes(self._h, int(with_bwd), C.byref(n)))
+        return int(n.value)
+
+    def new_workspace(self, with_bwd=False, device="cuda") -> torch.Tensor:
+        return torch.empty(self.workspace_bytes(with_bwd), dtype=torch.uint8, device=device)
+
+    def moc_chunk_pool(self, K, desc, ws):
+        _check(self._lib.moc_chunk_pool(self._h, _ptr(K), _ptr(desc), _ptr(ws), _stream()))
+
+    def moc_route(self, Q, desc, sel_idx, ws):
+        _check(self._lib.moc_route(self._h, _ptr(Q), _ptr(desc), _ptr(sel_idx), _ptr(ws), _stream()))
+
+    def moc_attend(self, Q, K, V, sel_idx, O, lse, ws):
+        _check(self._lib.moc_attend(self._h, _ptr(Q), _ptr(K), _ptr(V), _ptr(sel_idx), _ptr(O), _ptr(lse), _ptr(ws),
+                                    _stream()))
+
+    def moc_attend_bwd(self, Q, K, V, O, lse, dO, sel_idx, dQ, dK, dV, ws):
+        _check(self._lib.moc_attend_bwd(self._h, _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(lse), _ptr(dO),
+                                        _ptr(sel_idx), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws), _stream()))
+
+    def moc_selected_pairs(self, ws) -> int:
+        n = C.c_int64(0)
+        _check(self._lib.moc_selected_pairs(self._h, _ptr(ws), _stream(), C.byref(n)))
+        return int(n.value)
+
+    def moc_get_status(self, ws):
+        st, det = C.c_int(0), C.c_int(0)
+        _check(self._lib.moc_get_status(self._h, _ptr(ws), _stream(), C.byref(st), C.byref(det)))
+        return int(st.value), int(det.value)
+
+    # convenience: allocate outputs and run the forward path
+    def forward(self, Q, K, V, ws=None):
+        dev = Q.device
+        ws = self.new_workspace(False, dev) if ws is None else ws
+        desc = torch.empty((self.H, self.C, self.d), dtype=torch.float32, device=dev)
+        sel = torch.empty((self.H, self.L, self.k), dtype=torch.int32, device=dev)
+        O = torch.empty_like(Q)
+        lse = torch.empty((self.H, self.L), dtype=torch.float32, device=dev)
+        self.moc_chunk_pool(K, desc, ws)
+        self.moc_route(Q, desc, sel, ws)
+        self.moc_attend(Q, K, V, sel, O, lse, ws)
+        return desc, sel, O, lse, ws

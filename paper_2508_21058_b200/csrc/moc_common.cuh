@@ -1,0 +1,111 @@
+// Shared declarations of the MoC library: plan object, workspace layout, launch helpers.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <atomic>
+#include <vector>
+
+#include "../../include/moc.h"
+
+namespace moc {
+
+constexpr int kQTileRows = 128;     // query rows per attention tile
+constexpr int kPoolSlice = 256;     // tokens per chunk-pool work unit
+constexpr int kStatusWords = 16;    // status area at the head of the workspace (int32 each)
+
+// One contiguous range of key tokens [t0, t1).
+struct KeyRange { int32_t t0, t1; };
+
+// A tile of <= kQTileRows consecutive query rows that all live in chunk c.
+struct QTile { int32_t chunk, row0, rows, pad; };
+
+struct WsLayout {
+    size_t status;      // int32[kStatusWords]: [0] device status, [1] detail, [2] routed-flag
+    size_t cnt;         // int32[H][C]     routed picks per (head, chunk)
+    size_t qoff;        // int32[H][C+1]   CSR offsets of the query lists
+    size_t cursor;      // int32[H][C]     scatter cursors
+    size_t tile_off;    // int32[H][C+1]   prefix of ceil(cnt/128) routed tiles per head
+    size_t qlist;       // int32[H][L*k]   entries i*k+s, grouped by chunk
+    size_t pool_part;   // float[H][n_pool_units][d] partial key sums
+    size_t pool_done;   // int32[H][C] arrival counters (self-resetting)
+    size_t part_o;      // bf16 [H][L][k][d] routed partial outputs (normalised)
+    size_t part_lse;    // float[H][L][k]    routed partial log-sum-exp (-inf = unused slot)
+    size_t fwd_end;
+    size_t delta;       // float[H][L]       rowsum(dO * O)
+    size_t dq_acc;      // float[H][L][d]    fp32 dQ accumulator
+    size_t bwd_end;
+};
+
+}  // namespace moc
+
+struct moc_plan {
+    int H, L, d, C, k, win_back, win_fwd;
+    unsigned flags;
+    float scale;
+    int device;
+    int n_sm;
+    std::vector<int32_t> off, shot;
+    std::vector<uint8_t> mod;
+    // host-side derived tables
+    std::vector<int32_t> anc_off;            // [C+1] into anc_rng
+    std::vector<moc::KeyRange> anc_rng;      // merged anchor token ranges per query chunk
+    std::vector<int64_t> anc_tokens;         // [C] anchor key tokens per query chunk
+    std::vector<int32_t> ranc_off, ranc;     // reverse anchors: key chunk -> query chunks
+    std::vector<moc::QTile> qtiles;
+    std::vector<int32_t> pool_unit_off;      // [C+1] prefix of pool units per chunk
+    int words;                               // uint32 words per anchor bitmap row
+    int n_pool_units;
+    // device tables (one allocation)
+    void *d_blob;
+    int32_t *d_off, *d_shot, *d_tok_chunk, *d_anc_off, *d_ranc_off, *d_ranc, *d_pool_unit_off, *d_pool_unit_chunk;
+    uint8_t *d_mod;
+    uint32_t *d_anc_bits;
+    moc::KeyRange *d_anc_rng;
+    moc::QTile *d_qtiles;
+    moc::WsLayout ws;
+};
+
+namespace moc {
+
+extern std::atomic<long long> g_launches;
+void set_cuda_error(cudaError_t e, const char *where);
+
+#define MOC_CUDA_TRY(expr)                                         \
+    do {                                                           \
+        cudaError_t e_ = (expr);                                   \
+        if (e_ != cudaSuccess) {                                   \
+            moc::set_cuda_error(e_, #expr);                        \
+            return MOC_ERR_CUDA;                                   \
+        }                                                          \
+    } while (0)
+
+#define MOC_LAUNCH_CHECK()                                         \
+    do {                                                           \
+        moc::g_launches.fetch_add(1);                              \
+        cudaError_t e_ = cudaGetLastError();                       \
+        if (e_ != cudaSuccess) {                                   \
+            moc::set_cuda_error(e_, "kernel launch");              \
+            return MOC_ERR_CUDA;                                   \
+        }                                                          \
+    } while (0)
+
+template <typename T>
+static inline T *ws_ptr(void *ws, size_t off) { return reinterpret_cast<T *>(static_cast<char *>(ws) + off); }
+template <typename T>
+static inline const T *ws_ptr(const void *ws, size_t off) { return reinterpret_cast<const T *>(static_cast<const char *>(ws) + off); }
+
+static inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// kernels' host launchers (each returns a moc_status)
+int launch_chunk_pool(const moc_plan *p, const __nv_bfloat16 *K, float *desc, void *ws, cudaStream_t s);
+int launch_route(const moc_plan *p, const __nv_bfloat16 *Q, const float *desc, int32_t *sel, void *ws, cudaStream_t s);
+int launch_attend_scalar(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
+                         const int32_t *sel, __nv_bfloat16 *O, float *lse, void *ws, cudaStream_t s);
+int launch_attend_bwd_scalar(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
+                             const __nv_bfloat16 *O, const float *lse, const __nv_bfloat16 *dO, const int32_t *sel,
+                             __nv_bfloat16 *dQ, __nv_bfloat16 *dK, __nv_bfloat16 *dV, void *ws, cudaStream_t s);
+int launch_attend_tc(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
+                     const int32_t *sel, __nv_bfloat16 *O, float *lse, void *ws, cudaStream_t s);
+
+}  // namespace moc

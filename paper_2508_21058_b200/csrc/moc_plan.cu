@@ -1,0 +1,288 @@
+// Plan object (validated problem + derived chunk tables on the device), workspace layout,
+// argument checking and the C entry points.
+#include <math.h>
+#include <string.h>
+#include <mutex>
+#include <new>
+#include <string>
+
+#include "moc_common.cuh"
+
+namespace moc {
+
+std::atomic<long long> g_launches{0};
+static std::mutex g_err_mu;
+static std::string g_err = "";
+
+void set_cuda_error(cudaError_t e, const char *where) {
+    std::lock_guard<std::mutex> g(g_err_mu);
+    g_err = std::string(cudaGetErrorName(e)) + ": " + cudaGetErrorString(e) + " (" + where + ")";
+    (void)cudaGetLastError();
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Sec. 3.2: text chunks are anchors of every query; so are the chunks of the query's shot
+// inside the window around its own chunk.
+static bool is_anchor(const moc_plan *p, int c, int j) {
+    if (p->mod[j] == 1) return true;
+    if (p->shot[j] != p->shot[c]) return false;
+    if (j < c && p->win_back != MOC_WHOLE_SHOT && c - j > p->win_back) return false;
+    if (j > c && p->win_fwd != MOC_WHOLE_SHOT && j - c > p->win_fwd) return false;
+    return true;
+}
+
+static void layout_workspace(moc_plan *p) {
+    WsLayout &w = p->ws;
+    const size_t H = p->H, L = p->L, d = p->d, C = p->C, k = p->k;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    w.status = take(sizeof(int32_t) * kStatusWords);
+    w.cnt = take(sizeof(int32_t) * H * C);
+    w.qoff = take(sizeof(int32_t) * H * (C + 1));
+    w.cursor = take(sizeof(int32_t) * H * C);
+    w.tile_off = take(sizeof(int32_t) * H * (C + 1));
+    w.qlist = take(sizeof(int32_t) * H * L * (k ? k : 1));
+    w.pool_part = take(sizeof(float) * H * (size_t)p->n_pool_units * d);
+    w.pool_done = take(sizeof(int32_t) * H * C);
+    w.part_o = take(sizeof(__nv_bfloat16) * H * L * k * d);
+    w.part_lse = take(sizeof(float) * H * L * (k ? k : 1));
+    w.fwd_end = o;
+    w.delta = take(sizeof(float) * H * L);
+    w.dq_acc = take(sizeof(float) * H * L * d);
+    w.bwd_end = o;
+}
+
+}  // namespace moc
+
+using namespace moc;
+
+extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
+    if (!pr || !out) return MOC_ERR_NULL;
+    *out = nullptr;
+    if (!pr->chunk_off || !pr->chunk_shot || !pr->chunk_mod) return MOC_ERR_NULL;
+    if (pr->n_heads < 1 || pr->n_tokens < 1 || pr->n_chunks < 1 || pr->n_chunks > pr->n_tokens) return MOC_ERR_SHAPE;
+    if (pr->head_dim != 64 && pr->head_dim != 128) return MOC_ERR_SHAPE;
+    if (pr->top_k < 0 || pr->top_k > 512) return MOC_ERR_SHAPE;
+    if (pr->win_back < MOC_WHOLE_SHOT || pr->win_fwd < MOC_WHOLE_SHOT) return MOC_ERR_SHAPE;
+    if ((double)pr->n_tokens * (pr->top_k ? pr->top_k : 1) >= 2147483647.0) return MOC_ERR_SHAPE;
+    if ((double)pr->n_heads * pr->n_chunks >= 1e8) return MOC_ERR_SHAPE;
+    if (pr->flags & ~(MOC_FLAG_CAUSAL | MOC_FLAG_SCALAR_ATTEND)) return MOC_ERR_SHAPE;
+    if (!(pr->softmax_scale >= 0.f) || isinf(pr->softmax_scale)) return MOC_ERR_SHAPE;
+    const int C = pr->n_chunks, L = pr->n_tokens;
+    if (pr->chunk_off[0] != 0 || pr->chunk_off[C] != L) return MOC_ERR_CHUNK_TABLE;
+    for (int c = 0; c < C; ++c) {
+        if (pr->chunk_off[c + 1] <= pr->chunk_off[c]) return MOC_ERR_CHUNK_TABLE;
+        if (pr->chunk_mod[c] > 1) return MOC_ERR_CHUNK_TABLE;
+        if (c > 0 && pr->chunk_shot[c] < pr->chunk_shot[c - 1]) return MOC_ERR_CHUNK_TABLE;
+    }
+    int dev = 0;
+    MOC_CUDA_TRY(cudaGetDevice(&dev));
+    cudaDeviceProp prop;
+    MOC_CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) return MOC_ERR_ARCH;
+
+    moc_plan *p = new (std::nothrow) moc_plan();
+    if (!p) return MOC_ERR_CUDA;
+    p->H = pr->n_heads; p->L = L; p->d = pr->head_dim; p->C = C; p->k = pr->top_k;
+    p->win_back = pr->win_back; p->win_fwd = pr->win_fwd; p->flags = pr->flags;
+    p->scale = pr->softmax_scale > 0.f ? pr->softmax_scale : 1.0f / sqrtf((float)pr->head_dim);
+    p->device = dev; p->n_sm = prop.multiProcessorCount;
+    p->off.assign(pr->chunk_off, pr->chunk_off + C + 1);
+    p->shot.assign(pr->chunk_shot, pr->chunk_shot + C);
+    p->mod.assign(pr->chunk_mod, pr->chunk_mod + C);
+
+    // anchor bitmaps, merged anchor key ranges, reverse anchors
+    p->words = (C + 31) / 32;
+    std::vector<uint32_t> bits((size_t)C * p->words, 0u);
+    std::vector<std::vector<int32_t>> rev(C);
+    p->anc_off.assign(C + 1, 0);
+    p->anc_tokens.assign(C, 0);
+    for (int c = 0; c < C; ++c) {
+        for (int j = 0; j < C; ++j) {
+            if (!is_anchor(p, c, j)) continue;
+            bits[(size_t)c * p->words + j / 32] |= 1u << (j % 32);
+            rev[j].push_back(c);
+            p->anc_tokens[c] += p->off[j + 1] - p->off[j];
+            if ((int)p->anc_rng.size() > p->anc_off[c] && p->anc_rng.back().t1 == p->off[j])
+                p->anc_rng.back().t1 = p->off[j + 1];
+            else
+                p->anc_rng.push_back(KeyRange{p->off[j], p->off[j + 1]});
+        }
+        p->anc_off[c + 1] = (int32_t)p->anc_rng.size();
+    }
+    p->ranc_off.assign(C + 1, 0);
+    for (int j = 0; j < C; ++j) {
+        p->ranc.insert(p->ranc.end(), rev[j].begin(), rev[j].end());
+        p->ranc_off[j + 1] = (int32_t)p->ranc.size();
+    }
+    // query tiles (never straddle a chunk) and pool work units
+    std::vector<int32_t> tok_chunk(L), unit_chunk;
+    p->pool_unit_off.assign(C + 1, 0);
+    for (int c = 0; c < C; ++c) {
+        for (int t = p->off[c]; t < p->off[c + 1]; ++t) tok_chunk[t] = c;
+        for (int r = p->off[c]; r < p->off[c + 1]; r += kQTileRows)
+            p->qtiles.push_back(QTile{c, r, std::min(kQTileRows, p->off[c + 1] - r), 0});
+        int units = (p->off[c + 1] - p->off[c] + kPoolSlice - 1) / kPoolSlice;
+        p->pool_unit_off[c + 1] = p->pool_unit_off[c] + units;
+        for (int u = 0; u < units; ++u) unit_chunk.push_back(c);
+    }
+    p->n_pool_units = p->pool_unit_off[C];
+    layout_workspace(p);
+
+    // one device blob
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    size_t o_off = take(4 * (C + 1)), o_shot = take(4 * C), o_mod = take(C), o_tok = take(4 * (size_t)L);
+    size_t o_bits = take(4 * bits.size()), o_aoff = take(4 * (C + 1)), o_arng = take(sizeof(KeyRange) * p->anc_rng.size());
+    size_t o_roff = take(4 * (C + 1)), o_ranc = take(4 * p->ranc.size()), o_qt = take(sizeof(QTile) * p->qtiles.size());
+    size_t o_puo = take(4 * (C + 1)), o_puc = take(4 * unit_chunk.size());
+    cudaError_t e = cudaMalloc(&p->d_blob, o);
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaMalloc(plan tables)"); delete p; return MOC_ERR_CUDA; }
+    char *b = static_cast<char *>(p->d_blob);
+    auto up = [&](size_t at, const void *src, size_t bytes) {
+        return bytes ? cudaMemcpy(b + at, src, bytes, cudaMemcpyHostToDevice) : cudaSuccess;
+    };
+    cudaError_t es[] = {up(o_off, p->off.data(), 4 * (C + 1)), up(o_shot, p->shot.data(), 4 * C), up(o_mod, p->mod.data(), C),
+                        up(o_tok, tok_chunk.data(), 4 * (size_t)L), up(o_bits, bits.data(), 4 * bits.size()),
+                        up(o_aoff, p->anc_off.data(), 4 * (C + 1)), up(o_arng, p->anc_rng.data(), sizeof(KeyRange) * p->anc_rng.size()),
+                        up(o_roff, p->ranc_off.data(), 4 * (C + 1)), up(o_ranc, p->ranc.data(), 4 * p->ranc.size()),
+                        up(o_qt, p->qtiles.data(), sizeof(QTile) * p->qtiles.size()),
+                        up(o_puo, p->pool_unit_off.data(), 4 * (C + 1)), up(o_puc, unit_chunk.data(), 4 * unit_chunk.size())};
+    for (cudaError_t x : es)
+        if (x != cudaSuccess) { set_cuda_error(x, "cudaMemcpy(plan tables)"); cudaFree(p->d_blob); delete p; return MOC_ERR_CUDA; }
+    p->d_off = (int32_t *)(b + o_off); p->d_shot = (int32_t *)(b + o_shot); p->d_mod = (uint8_t *)(b + o_mod);
+    p->d_tok_chunk = (int32_t *)(b + o_tok); p->d_anc_bits = (uint32_t *)(b + o_bits);
+    p->d_anc_off = (int32_t *)(b + o_aoff); p->d_anc_rng = (KeyRange *)(b + o_arng);
+    p->d_ranc_off = (int32_t *)(b + o_roff); p->d_ranc = (int32_t *)(b + o_ranc); p->d_qtiles = (QTile *)(b + o_qt);
+    p->d_pool_unit_off = (int32_t *)(b + o_puo); p->d_pool_unit_chunk = (int32_t *)(b + o_puc);
+    *out = p;
+    return MOC_OK;
+}
+
+extern "C" int moc_plan_destroy(moc_plan *p) {
+    if (!p) return MOC_ERR_NULL;
+    if (p->d_blob) cudaFree(p->d_blob);
+    delete p;
+    return MOC_OK;
+}
+
+extern "C" int moc_workspace_bytes(const moc_plan *p, int with_bwd, size_t *bytes) {
+    if (!p || !bytes) return MOC_ERR_NULL;
+    *bytes = with_bwd ? p->ws.bwd_end : p->ws.fwd_end;
+    return MOC_OK;
+}
+
+static int check_dev_ptrs(std::initializer_list<const void *> ptrs, size_t a) {
+    for (const void *q : ptrs) {
+        if (!q) return MOC_ERR_NULL;
+        if (!aligned(q, a)) return MOC_ERR_ALIGN;
+    }
+    return MOC_OK;
+}
+
+static int enter(const moc_plan *p) {
+    if (!p) return MOC_ERR_NULL;
+    int dev = -1;
+    MOC_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != p->device) return MOC_ERR_ARCH;
+    return MOC_OK;
+}
+
+extern "C" int moc_chunk_pool(const moc_plan *p, const void *K, float *desc, void *ws, void *stream) {
+    if (int r = enter(p)) return r;
+    if (int r = check_dev_ptrs({K, desc}, 16)) return r;
+    if (!ws) return MOC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return MOC_ERR_ALIGN;
+    return launch_chunk_pool(p, (const __nv_bfloat16 *)K, desc, ws, (cudaStream_t)stream);
+}
+
+extern "C" int moc_route(const moc_plan *p, const void *Q, const float *desc, int32_t *sel_idx, void *ws, void *stream) {
+    if (int r = enter(p)) return r;
+    if (int r = check_dev_ptrs({Q, desc}, 16)) return r;
+    if (p->k > 0) { if (int r = check_dev_ptrs({sel_idx}, 4)) return r; }
+    if (!ws) return MOC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return MOC_ERR_ALIGN;
+    return launch_route(p, (const __nv_bfloat16 *)Q, desc, sel_idx, ws, (cudaStream_t)stream);
+}
+
+extern "C" int moc_attend(const moc_plan *p, const void *Q, const void *K, const void *V, const int32_t *sel_idx,
+                          void *O, float *lse, void *ws, void *stream) {
+    if (int r = enter(p)) return r;
+    if (int r = check_dev_ptrs({Q, K, V, O}, 16)) return r;
+    if (int r = check_dev_ptrs({lse}, 4)) return r;
+    if (p->k > 0) { if (int r = check_dev_ptrs({sel_idx}, 4)) return r; }
+    if (!ws) return MOC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return MOC_ERR_ALIGN;
+    auto q = (const __nv_bfloat16 *)Q, k = (const __nv_bfloat16 *)K, v = (const __nv_bfloat16 *)V;
+    if (p->flags & MOC_FLAG_SCALAR_ATTEND)
+        return launch_attend_scalar(p, q, k, v, sel_idx, (__nv_bfloat16 *)O, lse, ws, (cudaStream_t)stream);
+    return launch_attend_tc(p, q, k, v, sel_idx, (__nv_bfloat16 *)O, lse, ws, (cudaStream_t)stream);
+}
+
+extern "C" int moc_attend_bwd(const moc_plan *p, const void *Q, const void *K, const void *V, const void *O,
+                              const float *lse, const void *dO, const int32_t *sel_idx, void *dQ, void *dK, void *dV,
+                              void *ws, void *stream) {
+    if (int r = enter(p)) return r;
+    if (int r = check_dev_ptrs({Q, K, V, O, dO, dQ, dK, dV}, 16)) return r;
+    if (int r = check_dev_ptrs({lse}, 4)) return r;
+    if (p->k > 0) { if (int r = check_dev_ptrs({sel_idx}, 4)) return r; }
+    if (!ws) return MOC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return MOC_ERR_ALIGN;
+    return launch_attend_bwd_scalar(p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V,
+                                    (const __nv_bfloat16 *)O, lse, (const __nv_bfloat16 *)dO, sel_idx,
+                                    (__nv_bfloat16 *)dQ, (__nv_bfloat16 *)dK, (__nv_bfloat16 *)dV, ws, (cudaStream_t)stream);
+}
+
+extern "C" int moc_selected_pairs(const moc_plan *p, const void *ws, void *stream, int64_t *pairs) {
+    if (int r = enter(p)) return r;
+    if (!pairs) return MOC_ERR_NULL;
+    if (!ws) return MOC_ERR_WORKSPACE;
+    std::vector<int32_t> cnt((size_t)p->H * p->C);
+    MOC_CUDA_TRY(cudaMemcpyAsync(cnt.data(), ws_ptr<int32_t>(ws, p->ws.cnt), cnt.size() * 4, cudaMemcpyDeviceToHost,
+                                 (cudaStream_t)stream));
+    MOC_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    int64_t per_head = 0;
+    for (int c = 0; c < p->C; ++c) per_head += p->anc_tokens[c] * (int64_t)(p->off[c + 1] - p->off[c]);
+    int64_t total = per_head * p->H;
+    for (int h = 0; h < p->H; ++h)
+        for (int c = 0; c < p->C; ++c) total += (int64_t)cnt[(size_t)h * p->C + c] * (p->off[c + 1] - p->off[c]);
+    *pairs = total;
+    return MOC_OK;
+}
+
+extern "C" int moc_get_status(const moc_plan *p, const void *ws, void *stream, int *device_status, int *detail) {
+    if (int r = enter(p)) return r;
+    if (!device_status) return MOC_ERR_NULL;
+    if (!ws) return MOC_ERR_WORKSPACE;
+    int32_t st[2] = {0, 0};
+    MOC_CUDA_TRY(cudaMemcpyAsync(st, ws_ptr<int32_t>(ws, p->ws.status), sizeof st, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    MOC_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    *device_status = st[0];
+    if (detail) *detail = st[1];
+    return MOC_OK;
+}
+
+extern "C" int64_t moc_launch_count(void) { return (int64_t)g_launches.load(); }
+
+extern "C" const char *moc_strerror(int s) {
+    switch (s) {
+        case MOC_OK: return "ok";
+        case MOC_ERR_NULL: return "a required pointer is NULL";
+        case MOC_ERR_SHAPE: return "unsupported shape or parameter";
+        case MOC_ERR_CHUNK_TABLE: return "invalid chunk table";
+        case MOC_ERR_ALIGN: return "misaligned device pointer";
+        case MOC_ERR_WORKSPACE: return "workspace missing or not routed";
+        case MOC_ERR_ARCH: return "device is not sm_100 or differs from the plan's device";
+        case MOC_ERR_CUDA: return "CUDA runtime error";
+        case MOC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        default: return "unknown status";
+    }
+}
+
+extern "C" const char *moc_last_cuda_error(void) {
+    static thread_local std::string copy;
+    std::lock_guard<std::mutex> g(g_err_mu);
+    copy = g_err;
+    return copy.c_str();
+}

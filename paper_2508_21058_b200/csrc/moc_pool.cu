@@ -1,0 +1,117 @@
+// Chunk descriptors: desc[h][c][:] = mean of K[h][t][:] over the chunk's tokens.
+//
+// HBM-bound stream of K.  A work unit is (head, chunk, slice of kPoolSlice tokens); a
+// block of 256 threads reads its slice with 128-bit loads (a token row of d bf16 is
+// d/8 lanes wide, so one pass covers 256*8/d rows and every warp reads whole 128-byte
+// lines), accumulates in fp32 registers, folds the row groups through shared memory
+// and writes one partial sum.  The last block to finish a chunk (arrival counter)
+// adds the partials in slice order and scales by 1/n, so the result does not depend
+// on block scheduling.
+#include "moc_common.cuh"
+
+namespace moc {
+
+template <int D>
+__global__ void __launch_bounds__(256) chunk_pool_kernel(const __nv_bfloat16 *__restrict__ K, float *__restrict__ desc,
+                                                          float *__restrict__ part, int *__restrict__ done,
+                                                          const int32_t *__restrict__ off,
+                                                          const int32_t *__restrict__ unit_off,
+                                                          const int32_t *__restrict__ unit_chunk, int L, int C,
+                                                          int n_units) {
+    constexpr int LANES = D / 8;          // 16-byte lanes per token row
+    constexpr int ROWS = 256 / LANES;     // rows per pass
+    __shared__ float red[ROWS][D + 4];
+    __shared__ int is_last;
+    const int h = blockIdx.y;
+    const int lane = threadIdx.x % LANES, rg = threadIdx.x / LANES;
+    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+        const int c = unit_chunk[unit];
+        const int slice = unit - unit_off[c];
+        const int t0 = off[c] + slice * kPoolSlice;
+        const int t1 = min(off[c + 1], t0 + kPoolSlice);
+        float acc[8];
+#pragma unroll
+        for (int x = 0; x < 8; ++x) acc[x] = 0.f;
+        const uint4 *base = reinterpret_cast<const uint4 *>(K + ((size_t)h * L) * D) + lane;
+        int t = t0 + rg;
+        // 4 independent 16-byte loads in flight per thread
+        for (; t + 3 * ROWS < t1; t += 4 * ROWS) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = __ldg(base + (size_t)(t + u * ROWS) * LANES);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&v[u]);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                    float2 f = __bfloat1622float2(b[x]);
+                    acc[2 * x] += f.x;
+                    acc[2 * x + 1] += f.y;
+                }
+            }
+        }
+        for (; t < t1; t += ROWS) {
+            uint4 v = __ldg(base + (size_t)t * LANES);
+            const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&v);
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                float2 f = __bfloat1622float2(b[x]);
+                acc[2 * x] += f.x;
+                acc[2 * x + 1] += f.y;
+            }
+        }
+#pragma unroll
+        for (int x = 0; x < 8; ++x) red[rg][lane * 8 + x] = acc[x];
+        __syncthreads();
+        float *mine = part + ((size_t)h * n_units + unit) * D;
+        if (threadIdx.x < D) {
+            float s = 0.f;
+#pragma unroll
+            for (int r = 0; r < ROWS; ++r) s += red[r][threadIdx.x];
+            mine[threadIdx.x] = s;
+            __threadfence();
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int n_slices = unit_off[c + 1] - unit_off[c];
+            int prev = atomicAdd(&done[h * C + c], 1);
+            is_last = (prev == n_slices - 1);
+        }
+        __syncthreads();
+        if (is_last) {
+            __threadfence();
+            if (threadIdx.x < D) {
+                const int u0 = unit_off[c], u1 = unit_off[c + 1];
+                float s = 0.f;
+                for (int u = u0; u < u1; ++u) s += __ldcg(part + ((size_t)h * n_units + u) * D + threadIdx.x);
+                desc[((size_t)h * C + c) * D + threadIdx.x] = s / (float)(off[c + 1] - off[c]);
+            }
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void zero_i32_kernel(int *p, size_t n) {
+    size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
+    if (i < n) p[i] = 0;
+}
+
+int launch_chunk_pool(const moc_plan *p, const __nv_bfloat16 *K, float *desc, void *ws, cudaStream_t s) {
+    float *part = ws_ptr<float>(ws, p->ws.pool_part);
+    int *done = ws_ptr<int>(ws, p->ws.pool_done);
+    // the arrival counters live in caller-owned scratch whose contents are unknown
+    size_t n = (size_t)p->H * p->C;
+    zero_i32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(done, n);
+    MOC_LAUNCH_CHECK();
+    dim3 grid((unsigned)std::min(p->n_pool_units, 65535), (unsigned)p->H);
+    if (p->d == 128)
+        chunk_pool_kernel<128><<<grid, 256, 0, s>>>(K, desc, part, done, p->d_off, p->d_pool_unit_off,
+                                                    p->d_pool_unit_chunk, p->L, p->C, p->n_pool_units);
+    else
+        chunk_pool_kernel<64><<<grid, 256, 0, s>>>(K, desc, part, done, p->d_off, p->d_pool_unit_off,
+                                                   p->d_pool_unit_chunk, p->L, p->C, p->n_pool_units);
+    MOC_LAUNCH_CHECK();
+    return MOC_OK;
+}
+
+}  // namespace moc
