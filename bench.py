@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the MoC hot path (pool -> route -> attend, + backward for the training
+workload) on seeded synthetic inputs.
+
+    python bench.py --gpus N --steps K --warmup W [--workload cfg1] [--impl reference]
+
+One step = one pass of the whole hot path over one batch.  The headline value is the
+selected-key attention throughput of the whole step: 4*d FLOPs per selected (query, key)
+pair (10*d more with the backward), divided by the device time of the step, summed over
+ranks.  Ranks are independent replicas (one process per GPU, no data-path collective;
+rank r draws its inputs with seed r): weak scaling.  Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "moc_sparse_attention_selected_key_tflops"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self._stop, self._t = index, [], threading.Event(), None
+
+    def _loop(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout.strip()
+                if out:
+                    self.rows.append([f.strip() for f in out.splitlines()[0].split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._t = threading.Thread(target=self._loop, daemon=True)
+        self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._t.join(timeout=10)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def step_flops(wl, pairs: int, with_bwd: bool) -> float:
+    return (4.0 + (10.0 if with_bwd else 0.0)) * wl.head_dim * pairs
+
+
+def route_bytes(wl) -> float:
+    H, L, d, C, k = wl.n_heads, wl.n_tokens, wl.head_dim, wl.n_chunks, wl.top_k
+    return 2.0 * (2 * L * d * H) + 4.0 * k * L * H + 2 * 4.0 * C * d * H   # K once + Q once + indices + desc write/read
+
+
+def run_reference(args, wl):
+    """The CPU oracle, as it stands, timed per step on a bounded sample of the workload:
+    one head's descriptors and routing in full, attention on a seeded sample of its rows."""
+    import numpy as np
+    import oracle
+    from oracle import Oracle
+    from paper_2508_21058_b200 import workloads as W
+    rows_per_step = args.ref_rows
+    heads = [s % wl.n_heads for s in range(args.warmup + args.steps)]
+    times, flops = [], []
+    for s, h in enumerate(heads):
+        x = {n: W.as_u16(t) for n, t in W.generate(wl, "cpu", ("q", "k", "v"), heads=[h]).items()}
+        orc = Oracle.from_workload(wl, n_heads=1)
+        rng = np.random.RandomState(100 + s)
+        rows = np.stack([np.zeros(rows_per_step, np.int32),
+                         np.sort(rng.randint(0, wl.n_tokens, rows_per_step)).astype(np.int32)], 1)
+        t0 = time.perf_counter()
+        desc = orc.chunk_pool(x["k"])
+        sel = orc.route(x["q"], desc)
+        orc.attend(x["q"], x["k"], x["v"], sel, rows)
+        dt = time.perf_counter() - t0
+        if s >= args.warmup:
+            times.append(dt)
+            flops.append(4.0 * wl.head_dim * orc.pair_count(sel, rows))
+    total_t, total_f = sum(times), sum(flops)
+    value = total_f / total_t / 1e12
+    sample = (f"per step: descriptors + routing of one head in full ({wl.n_tokens} rows), attention on "
+              f"{rows_per_step} seeded rows of that head")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / max(len(times), 1),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "layout": wl.note, "heads": wl.n_heads, "head_dim": wl.head_dim,
+                       "tokens": wl.n_tokens, "chunks": wl.n_chunks, "top_k": wl.top_k},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def cpu_baseline(wl, budget_s: float):
+    """Oracle attention on a bounded seeded row sample (sized from a short probe)."""
+    import numpy as np
+    import oracle
+    from oracle import Oracle
+    from paper_2508_21058_b200 import workloads as W
+    x = {n: W.as_u16(t) for n, t in W.generate(wl, "cpu", ("q", "k", "v"), heads=[0]).items()}
+    orc = Oracle.from_workload(wl, n_heads=1)
+    t0 = time.perf_counter()
+    sel = orc.route(x["q"], orc.chunk_pool(x["k"]))
+    t_route = time.perf_counter() - t0
+    rng = np.random.RandomState(42)
+
+    def sample(n):
+        return np.stack([np.zeros(n, np.int32), np.sort(rng.randint(0, wl.n_tokens, n)).astype(np.int32)], 1)
+
+    probe = sample(64)
+    t0 = time.perf_counter()
+    orc.attend(x["q"], x["k"], x["v"], sel, probe)
+    per_row = (time.perf_counter() - t0) / len(probe)
+    n = int(max(64, min(20000, budget_s / max(per_row, 1e-6))))
+    rows = sample(n)
+    t0 = time.perf_counter()
+    orc.attend(x["q"], x["k"], x["v"], sel, rows)
+    dt = time.perf_counter() - t0
+    fl = 4.0 * wl.head_dim * orc.pair_count(sel, rows)
+    return {"value": fl / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"attention of {n} seeded rows of head 0 ({dt:.1f} s); head-0 descriptors + routing took {t_route:.1f} s"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg1")
+    ap.add_argument("--scalar", action="store_true", help="use the CUDA-core attention kernels")
+    ap.add_argument("--bwd", action="store_true", help="include moc_attend_bwd in the step (implied by cfg4)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget-s", type=float, default=15.0)
+    ap.add_argument("--ref-rows", type=int, default=256)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2508_21058_b200 import workloads as W
+    wl = W.workload(args.workload, seed=rank)
+    with_bwd = args.bwd or args.workload == "cfg4"
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, wl)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2508_21058_b200 import MocPlan, launch_count
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    tensors = ("q", "k", "v", "do") if with_bwd else ("q", "k", "v")
+    x = W.generate(wl, "cuda", tensors)
+    plan = MocPlan.from_workload(wl, scalar_attend=args.scalar)
+    ws = plan.new_workspace(with_bwd)
+    H, L, d, C, k = wl.n_heads, wl.n_tokens, wl.head_dim, wl.n_chunks, wl.top_k
+    desc = torch.empty((H, C, d), dtype=torch.float32, device="cuda")
+    sel = torch.empty((H, L, k), dtype=torch.int32, device="cuda")
+    O = torch.empty_like(x["q"])
+    lse = torch.empty((H, L), dtype=torch.float32, device="cuda")
+    grads = [torch.empty_like(x["q"]) for _ in range(3)] if with_bwd else None
+
+    def step(q, kk, v, marks=None):
+        ev = (lambda: marks.append(_rec())) if marks is not None else (lambda: None)
+        ev()
+        plan.moc_chunk_pool(kk, desc, ws)
+        ev()
+        plan.moc_route(q, desc, sel, ws)
+        ev()
+        plan.moc_attend(q, kk, v, sel, O, lse, ws)
+        ev()
+        if with_bwd:
+            plan.moc_attend_bwd(q, kk, v, O, lse, x["do"], sel, *grads, ws)
+            ev()
+
+    def _rec():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
+        return e
+
+    for _ in range(max(args.warmup, 3)):
+        step(x["q"], x["k"], x["v"])
+    barrier()
+    st, det = plan.moc_get_status(ws)
+    if st != 0:
+        raise SystemExit(f"device status {st} detail {det}")
+    pairs = plan.moc_selected_pairs(ws)
+    flops = step_flops(wl, pairs, with_bwd)
+
+    # ---- timed region: inputs resident in HBM, device time by CUDA events on the launching stream
+    marks_all = []
+    n0 = launch_count()
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        for _ in range(args.steps):
+            m = []
+            step(x["q"], x["k"], x["v"], m)
+            marks_all.append(m)
+        barrier()
+    launches = launch_count() - n0
+    total_ms = marks_all[0][0].elapsed_time(marks_all[-1][-1])
+    seg = [sum(m[i].elapsed_time(m[i + 1]) for m in marks_all) / args.steps for i in range(len(marks_all[0]) - 1)]
+    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_per_step = float(t.item()) / args.steps
+    value = world * flops / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end: host buffers in, host results out, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        hq, hk, hv = (x[n].cpu().pin_memory() for n in ("q", "k", "v"))
+        dq, dk, dv = (torch.empty_like(x[n]) for n in ("q", "k", "v"))
+        hO = torch.empty(O.shape, dtype=O.dtype).pin_memory()
+        hl = torch.empty(lse.shape, dtype=lse.dtype).pin_memory()
+        hg = [torch.empty(O.shape, dtype=O.dtype).pin_memory() for _ in range(3)] if with_bwd else []
+
+        def e2e_step():
+            dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
+            step(dq, dk, dv)
+            hO.copy_(O, non_blocking=True); hl.copy_(lse, non_blocking=True)
+            for a, b in zip(hg, grads or []):
+                a.copy_(b, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+
+        n_e2e = max(2, min(args.steps, 5))
+        e2e_step()
+        barrier()
+        e0, e1 = _rec(), None
+        for _ in range(n_e2e):
+            e2e_step()
+        e1 = _rec()
+        barrier()
+        te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        h2d = 3 * hq.numel() * 2
+        d2h = hO.numel() * 2 + hl.numel() * 4 + sum(g.numel() * 2 for g in hg)
+        e2e = {"value": world * flops / (float(te.item()) / n_e2e * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = load_peaks()
+    t_pool, t_route, t_att = seg[0], seg[1], seg[2]
+    att_flops = step_flops(wl, pairs, False)
+    traffic = None
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            traffic = json.load(f).get(f"attend:{wl.name}")
+    except Exception:
+        pass
+    roofline = {"kernel": "moc_attend (tensor-core flash kernel over selected key chunks)" if not args.scalar
+                else "moc_attend (CUDA-core kernels)",
+                "bound": "tensor", "achieved": att_flops / (t_att * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s", "frac": att_flops / (t_att * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                "frac_of_sustained": att_flops / (t_att * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+                "traffic": traffic, "peak_source": f"{peak_kind} (burst bf16 matmul)", "ms": t_att}
+    rb = route_bytes(wl)
+    routing = {"kernel": "moc_chunk_pool + moc_route", "bound": "hbm", "achieved": rb / ((t_pool + t_route) * 1e-3) / 1e9,
+               "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rb / ((t_pool + t_route) * 1e-3) / 1e9 / peaks["hbm_gbs"],
+               "pool_ms": t_pool, "route_ms": t_route, "pool_gbs": (2.0 * L * d * H) / (t_pool * 1e-3) / 1e9,
+               "peak_source": peak_kind}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "layout": wl.note, "heads": H, "head_dim": d, "tokens": L, "chunks": C,
+                       "top_k": k, "window": [wl.win_back, wl.win_fwd], "backward": with_bwd,
+                       "selected_pairs": pairs, "sparsity_vs_dense": 1.0 - pairs / (float(H) * L * L),
+                       "l2": "inputs larger than L2 (Q, K, V %.0f MB each); no flush" % (H * L * d * 2 / 1e6),
+                       "parallelism": f"replicas x{world}"},
+            "segments_ms": {"pool": t_pool, "route": t_route, "attend": t_att, **({"attend_bwd": seg[3]} if with_bwd else {})},
+            "roofline": roofline, "roofline_routing": routing, "clocks": clocks.summary(), "gpu_launches": int(launches)}
+    if e2e:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl, args.cpu_budget_s)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
