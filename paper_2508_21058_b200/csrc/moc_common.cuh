@@ -25,7 +25,8 @@ struct WsLayout {
     size_t cnt;         // int32[H][C]     routed picks per (head, chunk)
     size_t qoff;        // int32[H][C+1]   CSR offsets of the query lists
     size_t cursor;      // int32[H][C]     scatter cursors
-    size_t tile_off;    // int32[H][C+1]   prefix of ceil(cnt/128) routed tiles per head
+    size_t gcnt;        // int32[H*C+1]    running pick count over (head, chunk) pairs
+    size_t tile_off;    // int32[H*C+1]    running count of 128-row routed tiles over (head, chunk) pairs
     size_t qlist;       // int32[H][L*k]   entries i*k+s, grouped by chunk
     size_t pool_part;   // float[H][n_pool_units][d] partial key sums
     size_t pool_done;   // int32[H][C] arrival counters (self-resetting)

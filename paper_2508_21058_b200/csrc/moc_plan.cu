@@ -41,7 +41,8 @@ static void layout_workspace(moc_plan *p) {
     w.cnt = take(sizeof(int32_t) * H * C);
     w.qoff = take(sizeof(int32_t) * H * (C + 1));
     w.cursor = take(sizeof(int32_t) * H * C);
-    w.tile_off = take(sizeof(int32_t) * H * (C + 1));
+    w.gcnt = take(sizeof(int32_t) * (H * C + 1));
+    w.tile_off = take(sizeof(int32_t) * (H * C + 1));
     w.qlist = take(sizeof(int32_t) * H * L * (k ? k : 1));
     w.pool_part = take(sizeof(float) * H * (size_t)p->n_pool_units * d);
     w.pool_done = take(sizeof(int32_t) * H * C);

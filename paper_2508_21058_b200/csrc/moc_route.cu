@@ -48,7 +48,8 @@ struct TopK {
 template <int D, int KMAX>
 __global__ void __launch_bounds__(kRouteRows) route_kernel(const __nv_bfloat16 *__restrict__ Q,
                                                             const float *__restrict__ desc, int32_t *__restrict__ sel,
-                                                            int *__restrict__ cnt, const int32_t *__restrict__ tok_chunk,
+                                                            int *__restrict__ cnt, float *__restrict__ part_lse,
+                                                            const int32_t *__restrict__ tok_chunk,
                                                             const uint32_t *__restrict__ anc_bits, int words, int L,
                                                             int C, int k, int causal) {
     constexpr int QS = D + 8;   // padded row stride (bf16 elements): conflict-free 16-byte row reads
@@ -121,12 +122,14 @@ __global__ void __launch_bounds__(kRouteRows) route_kernel(const __nv_bfloat16 *
     __syncthreads();
     if (live) {
         int32_t *out = sel + ((size_t)h * L + i) * k;
+        float *pl = part_lse + ((size_t)h * L + i) * k;   // empty slots never get a routed partial
         if (KMAX <= 8) {
 #pragma unroll
             for (int x = 0; x < (KMAX <= 8 ? KMAX : 1); ++x) {
                 if (x < k) {
                     out[x] = top.j[x];
                     if (top.j[x] >= 0) atomicAdd(&hist[top.j[x]], 1);
+                    else pl[x] = -INFINITY;
                 }
             }
         } else {
@@ -134,6 +137,7 @@ __global__ void __launch_bounds__(kRouteRows) route_kernel(const __nv_bfloat16 *
                 const int j = top.j[x];
                 out[x] = j;
                 if (j >= 0) atomicAdd(&hist[j], 1);
+                else pl[x] = -INFINITY;
             }
         }
     }
@@ -142,23 +146,37 @@ __global__ void __launch_bounds__(kRouteRows) route_kernel(const __nv_bfloat16 *
         if (hist[x]) atomicAdd(&cnt[h * C + x], hist[x]);
 }
 
-// per head: CSR offsets of the query lists and of their 128-row tiles; flags the workspace as routed
-__global__ void route_scan_kernel(const int *__restrict__ cnt, int *__restrict__ qoff, int *__restrict__ tile_off,
-                                  int *__restrict__ cursor, int *__restrict__ status, int C) {
-    const int h = blockIdx.x;
-    if (threadIdx.x == 0) {
-        int a = 0, t = 0;
-        for (int c = 0; c < C; ++c) {
-            qoff[h * (C + 1) + c] = a;
-            tile_off[h * (C + 1) + c] = t;
-            cursor[h * C + c] = 0;
-            const int n = cnt[h * C + c];
-            a += n;
-            t += (n + kQTileRows - 1) / kQTileRows;
-        }
-        qoff[h * (C + 1) + C] = a;
-        tile_off[h * (C + 1) + C] = t;
-        if (h == 0) status[2] = 1;
+// Running totals over the H*C (head, chunk) pairs in one block: gcnt[i] = picks before pair i,
+// gtile[i] = 128-row tiles before pair i (both with a final total entry), cursors zeroed;
+// then qoff[h][c] = picks of head h before chunk c.  Flags the workspace as routed.
+__global__ void __launch_bounds__(1024) route_scan_kernel(const int *__restrict__ cnt, int *__restrict__ gcnt,
+                                                          int *__restrict__ gtile, int *__restrict__ qoff,
+                                                          int *__restrict__ cursor, int *__restrict__ status, int H, int C) {
+    __shared__ int sc[1024], st[1024];
+    const int HC = H * C, t = threadIdx.x;
+    const int per = (HC + 1023) / 1024;
+    const int i0 = min(t * per, HC), i1 = min(i0 + per, HC);
+    int a = 0, b = 0;
+    for (int i = i0; i < i1; ++i) { a += cnt[i]; b += (cnt[i] + kQTileRows - 1) / kQTileRows; }
+    sc[t] = a; st[t] = b;
+    __syncthreads();
+    for (int o = 1; o < 1024; o <<= 1) {   // inclusive scan
+        int xa = 0, xb = 0;
+        if (t >= o) { xa = sc[t - o]; xb = st[t - o]; }
+        __syncthreads();
+        sc[t] += xa; st[t] += xb;
+        __syncthreads();
+    }
+    int ea = sc[t] - a, eb = st[t] - b;    // exclusive
+    for (int i = i0; i < i1; ++i) {
+        gcnt[i] = ea; gtile[i] = eb; cursor[i] = 0;
+        ea += cnt[i]; eb += (cnt[i] + kQTileRows - 1) / kQTileRows;
+    }
+    if (t == 1023) { gcnt[HC] = sc[1023]; gtile[HC] = st[1023]; status[2] = 1; }
+    __syncthreads();
+    for (int idx = t; idx < H * (C + 1); idx += 1024) {
+        const int h = idx / (C + 1), c = idx % (C + 1);
+        qoff[idx] = gcnt[h * C + c] - gcnt[h * C];
     }
 }
 
@@ -199,7 +217,7 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
 #define MOC_ROUTE_CASE(KM)                                                                                          \
     do {                                                                                                            \
         MOC_CUDA_TRY(cudaFuncSetAttribute(route_kernel<D, KM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        route_kernel<D, KM><<<grid, kRouteRows, smem, s>>>(Q, desc, sel, cnt, p->d_tok_chunk, p->d_anc_bits, p->words, \
+        route_kernel<D, KM><<<grid, kRouteRows, smem, s>>>(Q, desc, sel, cnt, ws_ptr<float>(ws, p->ws.part_lse), p->d_tok_chunk, p->d_anc_bits, p->words, \
                                                            p->L, p->C, p->k, causal);                               \
     } while (0)
         if (p->k <= 8) MOC_ROUTE_CASE(8);
@@ -208,8 +226,8 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
 #undef MOC_ROUTE_CASE
         MOC_LAUNCH_CHECK();
     }
-    route_scan_kernel<<<p->H, 32, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.qoff), ws_ptr<int>(ws, p->ws.tile_off),
-                                          ws_ptr<int>(ws, p->ws.cursor), status, p->C);
+    route_scan_kernel<<<1, 1024, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.gcnt), ws_ptr<int>(ws, p->ws.tile_off),
+                                         ws_ptr<int>(ws, p->ws.qoff), ws_ptr<int>(ws, p->ws.cursor), status, p->H, p->C);
     MOC_LAUNCH_CHECK();
     if (p->k > 0) {
         dim3 grid((unsigned)((p->L + 255) / 256), (unsigned)p->H);
