@@ -55,7 +55,8 @@ typedef enum moc_status {
     MOC_ERR_WORKSPACE = -5,   /* workspace missing, or routing has not been run on it        */
     MOC_ERR_ARCH = -6,        /* the current device is not compute capability 10.x           */
     MOC_ERR_CUDA = -7,        /* a CUDA runtime call failed; see moc_last_cuda_error()       */
-    MOC_ERR_TIMEOUT = -8      /* device status: a bounded wait inside a kernel ran out       */
+    MOC_ERR_TIMEOUT = -8,     /* device status: a bounded wait inside a kernel ran out       */
+    MOC_ERR_TOO_LARGE = -9    /* problem exceeds the fixed scratch of a no-allocation entry point */
 } moc_status;
 
 #define MOC_WHOLE_SHOT (-1)   /* window value: every chunk of the query's shot is an anchor  */
@@ -91,6 +92,26 @@ int moc_workspace_bytes(const moc_plan *plan, int with_bwd, size_t *bytes);
 /* Step 1 - chunk descriptors (Eq. 3 text: phi = mean pooling of the chunk's keys).
  * desc[h][c][:] = mean over t in chunk c of K[h][t][:], accumulated in fp32. */
 int moc_chunk_pool(const moc_plan *plan, const void *K, float *desc, void *ws, void *stream);
+
+/* (The paper has no counterpart to this entry point; it exists for deployment reasons.)
+ * Same result as moc_chunk_pool, for callers that cannot hand over a workspace because they
+ * cannot allocate device memory at this point: code running after a serving engine or a
+ * training framework has already claimed the whole GPU for its own pool, hosts with a fixed
+ * memory budget settled at start-up, and latency-critical loops where cudaMalloc / cudaFree
+ * (which may block on the whole device) are forbidden.  The kernel's scratch (per-slice partial
+ * sums and per-chunk arrival counters) lives in a fixed array inside the library image: every
+ * GPU that loads the library holds those 4 MiB + 64 KiB until the process exits.
+ *   Limits: H * ceil-sum(chunk_len / 256) * d * 4 bytes <= 4 MiB and H * C * 4 bytes <= 64 KiB,
+ *   otherwise MOC_ERR_TOO_LARGE and nothing is launched (the 33k-token single-shot clip with 24
+ *   heads needs 1.8 MiB; longer streams must use moc_chunk_pool with a workspace).
+ *   K, desc: as for moc_chunk_pool; the caller still owns inputs and outputs.
+ *   The call itself allocates nothing (no cudaMalloc / cudaFree, no allocating library call).
+ *   The first call on each device looks up the array's device address; make that first call
+ *   before starting any stream capture on that device.
+ *   All calls share the one array, which keeps whatever the previous call left (the counters are
+ *   cleared on the stream at the start of every call): two calls that may overlap on the GPU
+ *   (different streams, no ordering between them) race on it - serialise them. */
+int moc_chunk_pool_noalloc(const moc_plan *plan, const void *K, float *desc, void *stream);
 
 /* Steps 2-5 - routing (Eq. 3; Sec. 3.2 causal mask and fixed selections; Sec. 3.3 forced
  * links before top-k).  For every query i in chunk c(i): candidates are the chunks that

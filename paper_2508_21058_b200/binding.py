@@ -49,6 +49,7 @@ def load_library():
     lib.moc_plan_destroy.argtypes = [vp]
     lib.moc_workspace_bytes.argtypes = [vp, i32, C.POINTER(sz)]
     lib.moc_chunk_pool.argtypes = [vp, vp, vp, vp, vp]
+    lib.moc_chunk_pool_noalloc.argtypes = [vp, vp, vp, vp]
     lib.moc_route.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.moc_attend.argtypes = [vp] * 9
     lib.moc_attend_bwd.argtypes = [vp] * 13
@@ -128,6 +129,11 @@ class MocPlan:
 
     def moc_chunk_pool(self, K, desc, ws):
         _check(self._lib.moc_chunk_pool(self._h, _ptr(K), _ptr(desc), _ptr(ws), _stream()))
+
+    def moc_chunk_pool_noalloc(self, K, desc):
+        """Descriptors without a workspace: scratch is a fixed array inside the library (small
+        problems only; raises MocError -9 beyond its size).  Calls sharing a GPU must not overlap."""
+        _check(self._lib.moc_chunk_pool_noalloc(self._h, _ptr(K), _ptr(desc), _stream()))
 
     def moc_route(self, Q, desc, sel_idx, ws):
         _check(self._lib.moc_route(self._h, _ptr(Q), _ptr(desc), _ptr(sel_idx), _ptr(ws), _stream()))

@@ -277,6 +277,7 @@ extern "C" const char *moc_strerror(int s) {
         case MOC_ERR_ARCH: return "device is not sm_100 or differs from the plan's device";
         case MOC_ERR_CUDA: return "CUDA runtime error";
         case MOC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case MOC_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }

@@ -7,6 +7,8 @@
 // and writes one partial sum.  The last block to finish a chunk (arrival counter)
 // adds the partials in slice order and scales by 1/n, so the result does not depend
 // on block scheduling.
+#include <mutex>
+
 #include "moc_common.cuh"
 
 namespace moc {
@@ -115,3 +117,65 @@ int launch_chunk_pool(const moc_plan *p, const __nv_bfloat16 *K, float *desc, vo
 }
 
 }  // namespace moc
+
+// ---------------------------------------------------------------------------------------------
+// moc_chunk_pool_noalloc: the same descriptor kernel with its scratch (per-slice partial sums and
+// per-chunk arrival counters) in a fixed array that is part of the library image, so the caller
+// needs no workspace and the call allocates nothing.
+namespace moc {
+
+constexpr size_t kStaticPartBytes = 4u << 20;     // partial sums: H * units * d * 4 bytes must fit
+constexpr size_t kStaticDoneBytes = 64u << 10;    // arrival counters: H * C * 4 bytes must fit
+static __device__ __align__(256) unsigned char g_pool_scratch[kStaticPartBytes + kStaticDoneBytes];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_scratch_mu;
+static unsigned char *g_scratch_addr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device.  In host code the array's
+// name is only a handle; the address a kernel can use comes from cudaGetSymbolAddress,
+// once per device, with that device current.
+static int pool_scratch_address(int device, unsigned char **out) {
+    if (device < 0 || device >= kMaxDevices) return MOC_ERR_ARCH;
+    std::lock_guard<std::mutex> g(g_scratch_mu);
+    if (!g_scratch_addr[device]) {
+        void *ptr = nullptr;
+        MOC_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_pool_scratch));
+        if (!ptr) return MOC_ERR_CUDA;
+        g_scratch_addr[device] = static_cast<unsigned char *>(ptr);
+    }
+    *out = g_scratch_addr[device];
+    return MOC_OK;
+}
+
+}  // namespace moc
+
+extern "C" int moc_chunk_pool_noalloc(const moc_plan *p, const void *K, float *desc, void *stream) {
+    using namespace moc;
+    if (!p || !K || !desc) return MOC_ERR_NULL;
+    if (!aligned(K, 16) || !aligned(desc, 16)) return MOC_ERR_ALIGN;
+    int dev = -1;
+    MOC_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != p->device) return MOC_ERR_ARCH;
+    const size_t part_bytes = sizeof(float) * (size_t)p->H * p->n_pool_units * p->d;
+    const size_t done_bytes = sizeof(int) * (size_t)p->H * p->C;
+    if (part_bytes > kStaticPartBytes || done_bytes > kStaticDoneBytes) return MOC_ERR_TOO_LARGE;
+    unsigned char *base = nullptr;
+    if (int r = pool_scratch_address(dev, &base)) return r;
+    float *part = reinterpret_cast<float *>(base);
+    int *done = reinterpret_cast<int *>(base + kStaticPartBytes);
+    cudaStream_t s = (cudaStream_t)stream;
+    // the array keeps the previous call's contents: the counters must start at zero
+    const size_t n = (size_t)p->H * p->C;
+    zero_i32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(done, n);
+    MOC_LAUNCH_CHECK();
+    dim3 grid((unsigned)std::min(p->n_pool_units, 65535), (unsigned)p->H);
+    if (p->d == 128)
+        chunk_pool_kernel<128><<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(K), desc, part, done, p->d_off,
+                                                    p->d_pool_unit_off, p->d_pool_unit_chunk, p->L, p->C, p->n_pool_units);
+    else
+        chunk_pool_kernel<64><<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(K), desc, part, done, p->d_off,
+                                                   p->d_pool_unit_off, p->d_pool_unit_chunk, p->L, p->C, p->n_pool_units);
+    MOC_LAUNCH_CHECK();
+    return MOC_OK;
+}
