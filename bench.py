@@ -175,6 +175,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     ap.add_argument("--ref-rows", type=int, default=256)
+    ap.add_argument("--heads", type=int, default=0, help="override the head count (profiling a smaller case)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -184,6 +185,9 @@ def main():
 
     from paper_2508_21058_b200 import workloads as W
     wl = W.workload(args.workload, seed=rank)
+    if args.heads > 0:
+        wl.n_heads = args.heads
+        wl.name = f"{wl.name}-h{args.heads}"
     with_bwd = args.bwd or args.workload == "cfg4"
 
     if args.impl == "reference":

@@ -1,21 +1,25 @@
 // Tensor-core sparse attention forward (tcgen05 MMA, TMEM accumulators, TMA-fed K/V).
 //
 // Two passes share one kernel:
-//   routed pass (key-chunk stationary): work item = (head, chunk c, 128 entries of the list
-//     of (query, slot) pairs that picked c).  The Q rows are gathered into shared memory,
-//     the keys are exactly the tokens of chunk c, and each (query, slot) gets a partial
-//     result (normalised output + log-sum-exp) in the workspace.
-//   anchor pass (query-tile stationary): work item = (head, 128 consecutive rows of one
-//     chunk); keys are the chunk's mandatory anchors (merged token ranges).  Its epilogue
-//     merges the row's <= k routed partials by log-sum-exp and writes O and LSE.
+//   routed pass (key-chunk stationary): work item = (head, chunk c, up to 256 entries of the
+//     list of (query, slot) pairs that picked c).  The Q rows are gathered into shared
+//     memory, the keys are exactly the tokens of chunk c, and each (query, slot) gets a
+//     partial result (normalised output + log-sum-exp) in the workspace.
+//   anchor pass (query-tile stationary): work item = (head, up to 256 consecutive rows of
+//     one chunk); keys are the chunk's mandatory anchors (merged token ranges).  Its
+//     epilogue merges the row's <= k routed partials by log-sum-exp and writes O and LSE.
 //
-// One CTA = 6 warps, two CTAs per SM so that one CTA's softmax overlaps the other's MMAs:
-//   warps 0-3  one query row per thread (TMEM lane = row): load/gather Q into the
-//              swizzled shared tile, online softmax straight from TMEM, P written back to
-//              TMEM as packed bf16 (aliasing S), lazy rescale of O, epilogue;
-//   warp 4     TMA producer: K and V tiles (128 keys) with 128-byte swizzle;
-//   warp 5     one thread issues S = Q K^T (operands in shared memory) and O += P V
-//              (P from TMEM, V as an MN-major shared-memory operand), accumulators in TMEM.
+// One CTA per SM, 10 warps, two 128-row query tiles that share every K/V tile:
+//   warps 0-3 / 4-7  softmax group of query tile 0 / 1, one row per thread (TMEM lane = row):
+//              load or gather Q into the swizzled shared tile, read S from TMEM, online
+//              softmax, write P back to TMEM as packed bf16 (aliasing S), lazily rescale O,
+//              epilogue;
+//   warp 8     TMA producer: K and V tiles of 128 keys, two stages each, 128-byte swizzle;
+//   warp 9     one thread issues the MMAs in the order  PV0(j), S0(j+1), PV1(j), S1(j+1), so
+//              one group's softmax overlaps the other group's MMAs.  S = Q K^T takes both
+//              operands from shared memory, O += P V takes P from TMEM and V as an MN-major
+//              shared-memory operand; all accumulators live in TMEM (S0, S1, O0, O1 = 512
+//              columns).
 // Every mbarrier wait is bounded; a wait that runs out flags the workspace status word
 // and the CTA drains and leaves.
 #include "moc_common.cuh"
@@ -44,12 +48,12 @@ struct AttendParams {
 };
 
 constexpr int kBN = 128;               // keys per tile
-constexpr int kThreads = 192;
-constexpr int kTmemCols = 256;         // S/P: columns [0,128), O: [128, 128 + D)
+constexpr int kThreads = 320;
+constexpr int kTmemCols = 512;         // S0/P0 [0,128) S1/P1 [128,256) O0 [256,384) O1 [384,512)
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: O is rescaled only when the row max grows by more
 
-enum WaitCode { W_QFULL = 1, W_KFULL, W_VFULL, W_SFULL, W_PFULL, W_PVDONE, W_KEMPTY, W_VEMPTY, W_EPILOGUE };
+enum WaitCode { W_QFULL = 1, W_KFULL, W_VFULL, W_SFULL, W_PFULL, W_OFULL, W_KEMPTY, W_VEMPTY };
 
 struct TileIter {
     const KeyRange *rng;
@@ -66,15 +70,35 @@ struct TileIter {
     }
 };
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// (x0, x1) * (c, c) + (m, m) in one packed instruction
+__device__ __forceinline__ void fma2(float &r0, float &r1, float x0, float x1, float c, float m) {
+    asm("{ .reg .b64 p, q, r, d; mov.b64 p, {%2, %3}; mov.b64 q, {%4, %4}; mov.b64 r, {%5, %5}; "
+        "fma.rn.f32x2 d, p, q, r; mov.b64 {%0, %1}, d; }"
+        : "=f"(r0), "=f"(r1) : "f"(x0), "f"(x1), "f"(c), "f"(m));
+}
+__device__ __forceinline__ void add2(float &a0, float &a1, float b0, float b1) {
+    asm("{ .reg .b64 p, q, d; mov.b64 p, {%0, %1}; mov.b64 q, {%2, %3}; add.rn.f32x2 d, p, q; mov.b64 {%0, %1}, d; }"
+        : "+f"(a0), "+f"(a1) : "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void mul2(float &a0, float &a1, float s) {
+    asm("{ .reg .b64 p, q, d; mov.b64 p, {%0, %1}; mov.b64 q, {%2, %2}; mul.rn.f32x2 d, p, q; mov.b64 {%0, %1}, d; }"
+        : "+f"(a0), "+f"(a1) : "f"(s));
+}
+
 template <int D, bool ROUTED>
-__global__ void __launch_bounds__(kThreads, 2) attend_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+__global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                 const __grid_constant__ CUtensorMap tmV,
                                                                 const AttendParams p) {
     constexpr int TILE_BYTES = 128 * D * 2;
     constexpr int SUB = D / 64;            // 64-column (128-byte) sub-tiles per row
     constexpr int SUB_BYTES = 128 * 128;   // one sub-tile: 128 rows of 128 bytes
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[6];
+    __shared__ __align__(8) uint64_t bars[16];
     __shared__ uint32_t tmem_slot;
     __shared__ int s_abort;
     __shared__ int w_valid, w_h, w_rows, w_first, w_nrng, w_ntiles;
@@ -84,9 +108,11 @@ __global__ void __launch_bounds__(kThreads, 2) attend_tc_kernel(const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gbase = smem_raw + (sbase - smem_u32(smem_raw));
-    const uint32_t sQ = sbase, sK = sbase + TILE_BYTES, sV = sbase + 2 * TILE_BYTES;
-    const uint32_t q_full = smem_u32(&bars[0]), k_full = smem_u32(&bars[1]), v_full = smem_u32(&bars[2]),
-                   s_full = smem_u32(&bars[3]), p_full = smem_u32(&bars[4]), pv_done = smem_u32(&bars[5]);
+    // shared tiles: Q0 Q1 | K stage 0,1 | V stage 0,1
+    const uint32_t sQ = sbase, sK = sbase + 2 * TILE_BYTES, sV = sbase + 4 * TILE_BYTES;
+    auto bar = [&](int i) { return smem_u32(&bars[i]); };
+    // barrier indices
+    constexpr int Q_FULL = 0, K_FULL = 2, K_EMPTY = 4, V_FULL = 6, V_EMPTY = 8, S_FULL = 10, P_FULL = 12, O_FULL = 14;
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -124,17 +150,21 @@ __global__ void __launch_bounds__(kThreads, 2) attend_tc_kernel(const __grid_con
             w_ntiles = nt;
         }
         w_valid = valid;
-        mbar_init(q_full, 128);
-        mbar_init(k_full, 1);
-        mbar_init(v_full, 1);
-        mbar_init(s_full, 1);
-        mbar_init(p_full, 128);
-        mbar_init(pv_done, 1);
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(bar(Q_FULL + t), 128);
+            mbar_init(bar(K_FULL + t), 1);
+            mbar_init(bar(K_EMPTY + t), 1);
+            mbar_init(bar(V_FULL + t), 1);
+            mbar_init(bar(V_EMPTY + t), 1);
+            mbar_init(bar(S_FULL + t), 1);
+            mbar_init(bar(P_FULL + t), 128);
+            mbar_init(bar(O_FULL + t), 1);
+        }
         fence_barrier_init();
     }
     __syncthreads();
     if (!w_valid) return;
-    if (warp == 4) {
+    if (warp == 8) {
         tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
         tmem_relinquish();
     }
@@ -143,174 +173,181 @@ __global__ void __launch_bounds__(kThreads, 2) attend_tc_kernel(const __grid_con
     tc_fence_after();
 
     const uint32_t tmem = tmem_slot;
-    const uint32_t tS = tmem, tP = tmem, tO = tmem + 128;
     const int h = w_h, rows = w_rows, first = w_first, n_tiles = w_ntiles;
+    const bool two = rows > 128;            // is query tile 1 populated?
     volatile int *abort_flag = &s_abort;
 
-    if (warp < 4) {
-        // ------------------------------------------------------------ softmax / epilogue threads
-        const int r = threadIdx.x;
-        const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
-        int qi = -1, slot = 0;
-        if (r < rows) {
-            if (ROUTED) {
-                const int e = p.qlist[(size_t)h * p.L * p.k + first + r];
-                qi = e / p.k;
-                slot = e - qi * p.k;
-            } else {
-                qi = first + r;
-            }
-        }
-        {
-            const uint4 *src = reinterpret_cast<const uint4 *>(p.Q + ((size_t)h * p.L + (qi >= 0 ? qi : 0)) * D);
-#pragma unroll
-            for (int c16 = 0; c16 < D / 8; ++c16) {
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (qi >= 0) v = __ldg(src + c16);
-                *reinterpret_cast<uint4 *>(gbase + (c16 >> 3) * SUB_BYTES + sw128_offset(r, c16 & 7)) = v;
-            }
-        }
-        fence_proxy_async_smem();
-        mbar_arrive(q_full);
-
-        float m_run = -INFINITY, l_run = 0.f;
-        const float c = p.scale_log2;
-        TileIter it(w_rng, w_nrng);
-        int t0, valid, jt = 0;
-        bool ok = true;
-        while (it.next(t0, valid)) {
-            const uint32_t par = jt & 1;
-            ok = mbar_wait(s_full, par, abort_flag, p.status, W_SFULL);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            uint32_t v[32];
-            // pass 1: row maximum over the valid columns
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int ch = 0; ch * 32 < valid; ++ch) {
-                tmem_ld32(tS + lane_off + ch * 32, v);
-                tmem_wait_ld();
-#pragma unroll
-                for (int x = 0; x < 32; ++x) {
-                    const float s = __uint_as_float(v[x]);
-                    mx = fmaxf(mx, (ch * 32 + x < valid) ? s : -INFINITY);
+    if (warp < 8) {
+        // ------------------------------------------------------------ softmax / epilogue groups
+        const int g = warp >> 2;                       // query tile of this group
+        const int r = threadIdx.x & 127;               // row within the tile = TMEM lane
+        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + g * 128 + lane_off, tP = tS, tO = tmem + 256 + g * 128 + lane_off;
+        if (g == 0 || two) {
+            const int rt = g * 128 + r;                // row within the work item
+            int qi = -1, slot = 0;
+            if (rt < rows) {
+                if (ROUTED) {
+                    const int e = p.qlist[(size_t)h * p.L * p.k + first + rt];
+                    qi = e / p.k;
+                    slot = e - qi * p.k;
+                } else {
+                    qi = first + rt;
                 }
             }
-            const float m_new = fmaxf(m_run, mx * c);
-            float alpha = 1.f;
-            if (jt == 0) {
-                m_run = m_new;
-            } else if (m_new - m_run > kRescaleThreshold) {
-                alpha = exp2f(m_run - m_new);
-                m_run = m_new;
+            {
+                const uint4 *src = reinterpret_cast<const uint4 *>(p.Q + ((size_t)h * p.L + (qi >= 0 ? qi : 0)) * D);
+                uint8_t *dstq = gbase + g * TILE_BYTES;
+#pragma unroll
+                for (int c16 = 0; c16 < D / 8; ++c16) {
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (qi >= 0) v = __ldg(src + c16);
+                    *reinterpret_cast<uint4 *>(dstq + (c16 >> 3) * SUB_BYTES + sw128_offset(r, c16 & 7)) = v;
+                }
             }
-            if (__any_sync(0xffffffffu, alpha != 1.f)) {
-                // PV of the previous tile has completed (its commit precedes this tile's S)
+            fence_proxy_async_smem();
+            mbar_arrive(bar(Q_FULL + g));
+
+            float m_run = -INFINITY, l_run = 0.f;
+            const float c = p.scale_log2;
+            TileIter it(w_rng, w_nrng);
+            int t0, valid, jt = 0;
+            bool ok = true;
+            while (it.next(t0, valid)) {
+                ok = mbar_wait(bar(S_FULL + g), jt & 1, abort_flag, p.status, W_SFULL);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t v[4][32];
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) tmem_ld32(tS + ch * 32, v[ch]);
+                tmem_wait_ld();
+                if (valid < kBN) {
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch)
+#pragma unroll
+                        for (int x = 0; x < 32; ++x)
+                            if (ch * 32 + x >= valid) v[ch][x] = 0xff800000u;   // -inf
+                }
+                float mx = -INFINITY;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch)
+#pragma unroll
+                    for (int x = 0; x < 32; x += 2) mx = max3(mx, __uint_as_float(v[ch][x]), __uint_as_float(v[ch][x + 1]));
+                const float m_new = fmaxf(m_run, mx * c);
+                float alpha = 1.f;
+                if (jt == 0) {
+                    m_run = m_new;
+                } else if (m_new - m_run > kRescaleThreshold) {
+                    alpha = exp2f(m_run - m_new);
+                    m_run = m_new;
+                }
+                // P = exp2(s * c - m), packed bf16 into the P columns (aliasing S)
+                const float neg_m = -m_run;
+                float ls0 = 0.f, ls1 = 0.f;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t u[16];
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) {
+                        float a0, a1;
+                        fma2(a0, a1, __uint_as_float(v[ch][2 * x]), __uint_as_float(v[ch][2 * x + 1]), c, neg_m);
+                        a0 = exp2f(a0);
+                        a1 = exp2f(a1);
+                        add2(ls0, ls1, a0, a1);
+                        __nv_bfloat162 b = __floats2bfloat162_rn(a0, a1);
+                        u[x] = *reinterpret_cast<uint32_t *>(&b);
+                    }
+                    tmem_st16(tP + ch * 16, u);
+                }
+                if (__any_sync(0xffffffffu, alpha != 1.f)) {
+                    // this group's PV of the previous tile has completed (its commit precedes this tile's S)
+#pragma unroll 1
+                    for (int ch = 0; ch < D / 32; ++ch) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + ch * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * alpha);
+                        tmem_st32(tO + ch * 32, o);
+                    }
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(P_FULL + g));
+                l_run = l_run * alpha + (ls0 + ls1);
+                ++jt;
+            }
+            // ---- epilogue
+            if (ok) {
+                ok = mbar_wait(bar(O_FULL + g), 0, abort_flag, p.status, W_OFULL);
+                ok = __all_sync(0xffffffffu, ok);
+            }
+            if (ok) {
+                tc_fence_after();
+                const float inv_l = 1.f / l_run;
+                const float lse_own = (m_run + log2f(l_run)) * kLn2;
+                float w_own = inv_l, big = lse_own, wsum = 1.f;
+                const float *pl = nullptr;
+                const __nv_bfloat16 *po = nullptr;
+                if (!ROUTED && qi >= 0 && p.k > 0) {
+                    pl = p.part_lse + ((size_t)h * p.L + qi) * p.k;
+                    po = p.part_o + ((size_t)h * p.L + qi) * p.k * D;
+                    for (int s = 0; s < p.k; ++s) big = fmaxf(big, pl[s]);
+                    wsum = __expf(lse_own - big);
+                    for (int s = 0; s < p.k; ++s) wsum += __expf(pl[s] - big);
+                    w_own = __expf(lse_own - big) / wsum * inv_l;
+                }
 #pragma unroll 1
                 for (int ch = 0; ch < D / 32; ++ch) {
-                    tmem_ld32(tO + lane_off + ch * 32, v);
+                    uint32_t v[32];
+                    __syncwarp();
+                    tmem_ld32(tO + ch * 32, v);
                     tmem_wait_ld();
+                    float acc[32];
 #pragma unroll
-                    for (int x = 0; x < 32; ++x) v[x] = __float_as_uint(__uint_as_float(v[x]) * alpha);
-                    tmem_st32(tO + lane_off + ch * 32, v);
-                }
-            }
-            l_run *= alpha;
-            // pass 2: P = exp2(s * c - m), packed bf16 into the P columns (aliasing S)
-            const float neg_m = -m_run;
-            float lsum = 0.f;
-#pragma unroll 1
-            for (int ch = 0; ch * 32 < valid; ++ch) {
-                tmem_ld32(tS + lane_off + ch * 32, v);
-                tmem_wait_ld();
-                uint32_t u[16];
+                    for (int x = 0; x < 32; ++x) acc[x] = __uint_as_float(v[x]) * w_own;
+                    if (pl) {
+                        for (int s = 0; s < p.k; ++s) {
+                            const float ls = pl[s];
+                            if (ls == -INFINITY) continue;
+                            const float w = __expf(ls - big) / wsum;
+                            const uint4 *src = reinterpret_cast<const uint4 *>(po + (size_t)s * D + ch * 32);
 #pragma unroll
-                for (int x = 0; x < 16; ++x) {
-                    const int col = ch * 32 + 2 * x;
-                    const float p0 = (col < valid) ? exp2f(fmaf(__uint_as_float(v[2 * x]), c, neg_m)) : 0.f;
-                    const float p1 = (col + 1 < valid) ? exp2f(fmaf(__uint_as_float(v[2 * x + 1]), c, neg_m)) : 0.f;
-                    lsum += p0 + p1;
-                    __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
-                    u[x] = *reinterpret_cast<uint32_t *>(&b);
-                }
-                tmem_st16(tP + lane_off + ch * 16, u);
-            }
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(p_full);
-            l_run += lsum;
-            ++jt;
-        }
-        // ---- epilogue
-        if (ok) {
-            ok = mbar_wait(pv_done, (uint32_t)((n_tiles - 1) & 1), abort_flag, p.status, W_EPILOGUE);
-            ok = __all_sync(0xffffffffu, ok);
-        }
-        if (ok) {
-            tc_fence_after();
-            const float inv_l = 1.f / l_run;
-            const float lse_own = (m_run + log2f(l_run)) * kLn2;
-            float w_own = inv_l, big = lse_own, wsum = 1.f;
-            const float *pl = nullptr;
-            const __nv_bfloat16 *po = nullptr;
-            if (!ROUTED && qi >= 0 && p.k > 0) {
-                pl = p.part_lse + ((size_t)h * p.L + qi) * p.k;
-                po = p.part_o + ((size_t)h * p.L + qi) * p.k * D;
-                for (int s = 0; s < p.k; ++s) big = fmaxf(big, pl[s]);
-                wsum = __expf(lse_own - big);
-                for (int s = 0; s < p.k; ++s) wsum += __expf(pl[s] - big);
-                w_own = __expf(lse_own - big) / wsum * inv_l;
-            }
-            uint32_t v[32];
-#pragma unroll 1
-            for (int ch = 0; ch < D / 32; ++ch) {
-                __syncwarp();
-                tmem_ld32(tO + lane_off + ch * 32, v);
-                tmem_wait_ld();
-                float acc[32];
+                            for (int q4 = 0; q4 < 4; ++q4) {
+                                const uint4 raw = __ldcg(src + q4);
+                                const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&raw);
 #pragma unroll
-                for (int x = 0; x < 32; ++x) acc[x] = __uint_as_float(v[x]) * w_own;
-                if (pl) {
-                    for (int s = 0; s < p.k; ++s) {
-                        const float ls = pl[s];
-                        if (ls == -INFINITY) continue;
-                        const float w = __expf(ls - big) / wsum;
-                        const uint4 *src = reinterpret_cast<const uint4 *>(po + (size_t)s * D + ch * 32);
-#pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4) {
-                            const uint4 raw = __ldcg(src + q4);
-                            const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&raw);
-#pragma unroll
-                            for (int y = 0; y < 4; ++y) {
-                                const float2 f = __bfloat1622float2(b[y]);
-                                acc[q4 * 8 + 2 * y] = fmaf(w, f.x, acc[q4 * 8 + 2 * y]);
-                                acc[q4 * 8 + 2 * y + 1] = fmaf(w, f.y, acc[q4 * 8 + 2 * y + 1]);
+                                for (int y = 0; y < 4; ++y) {
+                                    const float2 f = __bfloat1622float2(b[y]);
+                                    acc[q4 * 8 + 2 * y] = fmaf(w, f.x, acc[q4 * 8 + 2 * y]);
+                                    acc[q4 * 8 + 2 * y + 1] = fmaf(w, f.y, acc[q4 * 8 + 2 * y + 1]);
+                                }
                             }
                         }
                     }
-                }
-                if (qi < 0) continue;
-                __nv_bfloat16 *dst = ROUTED ? p.part_o + (((size_t)h * p.L + qi) * p.k + slot) * D + ch * 32
-                                            : p.O + ((size_t)h * p.L + qi) * D + ch * 32;
+                    if (qi < 0) continue;
+                    __nv_bfloat16 *dst = ROUTED ? p.part_o + (((size_t)h * p.L + qi) * p.k + slot) * D + ch * 32
+                                                : p.O + ((size_t)h * p.L + qi) * D + ch * 32;
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    uint4 out;
-                    uint32_t *o32 = reinterpret_cast<uint32_t *>(&out);
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint4 out;
+                        uint32_t *o32 = reinterpret_cast<uint32_t *>(&out);
 #pragma unroll
-                    for (int y = 0; y < 4; ++y) {
-                        __nv_bfloat162 b = __floats2bfloat162_rn(acc[q4 * 8 + 2 * y], acc[q4 * 8 + 2 * y + 1]);
-                        o32[y] = *reinterpret_cast<uint32_t *>(&b);
+                        for (int y = 0; y < 4; ++y) {
+                            __nv_bfloat162 b = __floats2bfloat162_rn(acc[q4 * 8 + 2 * y], acc[q4 * 8 + 2 * y + 1]);
+                            o32[y] = *reinterpret_cast<uint32_t *>(&b);
+                        }
+                        reinterpret_cast<uint4 *>(dst)[q4] = out;
                     }
-                    reinterpret_cast<uint4 *>(dst)[q4] = out;
                 }
-            }
-            if (qi >= 0) {
-                if (ROUTED) p.part_lse[((size_t)h * p.L + qi) * p.k + slot] = lse_own;
-                else p.lse[(size_t)h * p.L + qi] = (pl ? big + __logf(wsum) : lse_own);
+                if (qi >= 0) {
+                    if (ROUTED) p.part_lse[((size_t)h * p.L + qi) * p.k + slot] = lse_own;
+                    else p.lse[(size_t)h * p.L + qi] = (pl ? big + __logf(wsum) : lse_own);
+                }
             }
         }
-    } else if (warp == 4) {
+    } else if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             prefetch_tensormap(&tmK);
@@ -319,60 +356,113 @@ __global__ void __launch_bounds__(kThreads, 2) attend_tc_kernel(const __grid_con
             int t0, valid, jt = 0;
             int k_last = -1, v_last = -1;   // last tile whose K / V copy was issued
             while (it.next(t0, valid)) {
-                if (jt > 0 && !mbar_wait(s_full, (jt - 1) & 1, abort_flag, p.status, W_KEMPTY)) break;
-                mbar_expect_tx(k_full, TILE_BYTES);
+                const int st = jt & 1;
+                const uint32_t ph = (jt >> 1) & 1;
+                if (!mbar_wait(bar(K_EMPTY + st), ph ^ 1, abort_flag, p.status, W_KEMPTY)) break;
+                mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
 #pragma unroll
-                for (int sub = 0; sub < SUB; ++sub) tma_load_2d(sK + sub * SUB_BYTES, &tmK, sub * 64, h * p.L + t0, k_full);
+                for (int sub = 0; sub < SUB; ++sub)
+                    tma_load_2d(sK + st * TILE_BYTES + sub * SUB_BYTES, &tmK, sub * 64, h * p.L + t0, bar(K_FULL + st));
                 k_last = jt;
-                if (jt > 0 && !mbar_wait(pv_done, (jt - 1) & 1, abort_flag, p.status, W_VEMPTY)) break;
-                mbar_expect_tx(v_full, TILE_BYTES);
+                if (!mbar_wait(bar(V_EMPTY + st), ph ^ 1, abort_flag, p.status, W_VEMPTY)) break;
+                mbar_expect_tx(bar(V_FULL + st), TILE_BYTES);
 #pragma unroll
-                for (int sub = 0; sub < SUB; ++sub) tma_load_2d(sV + sub * SUB_BYTES, &tmV, sub * 64, h * p.L + t0, v_full);
+                for (int sub = 0; sub < SUB; ++sub)
+                    tma_load_2d(sV + st * TILE_BYTES + sub * SUB_BYTES, &tmV, sub * 64, h * p.L + t0, bar(V_FULL + st));
                 v_last = jt;
                 ++jt;
             }
             if (*abort_flag) {
                 // drain: copies already issued must land before the CTA's shared memory is released
                 int dummy_flag = 0;
-                if (k_last >= 0) mbar_wait(k_full, (uint32_t)(k_last & 1), &dummy_flag, p.status, W_KFULL);
-                if (v_last >= 0) mbar_wait(v_full, (uint32_t)(v_last & 1), &dummy_flag, p.status, W_VFULL);
+                for (int b = 0; b < 2; ++b) {
+                    const int kj = k_last - b, vj = v_last - b;
+                    if (kj >= 0) mbar_wait(bar(K_FULL + (kj & 1)), (kj >> 1) & 1, &dummy_flag, p.status, W_KFULL);
+                    if (vj >= 0) mbar_wait(bar(V_FULL + (vj & 1)), (vj >> 1) & 1, &dummy_flag, p.status, W_VFULL);
+                }
             }
         }
     } else {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t IDESC_PV = idesc_bf16_f32(128, D, 0, 1);
-            bool ok = mbar_wait(q_full, 0, abort_flag, p.status, W_QFULL);
-            TileIter it(w_rng, w_nrng);
-            int t0, valid, jt = 0;
-            while (ok && it.next(t0, valid)) {
-                const uint32_t par = jt & 1;
-                if (!mbar_wait(k_full, par, abort_flag, p.status, W_KFULL)) break;
-                // S and P share columns: the previous tile's PV must have consumed P
-                if (jt > 0 && !mbar_wait(pv_done, par ^ 1, abort_flag, p.status, W_PVDONE)) break;
-                tc_fence_after();
+            auto issue_qk = [&](int g, int st, int valid) {
                 const int n_qk = max(16, (valid + 15) & ~15);
                 const uint32_t idesc_qk = idesc_bf16_f32(128, n_qk, 0, 0);
+                const uint32_t q0 = sQ + g * TILE_BYTES, k0 = sK + st * TILE_BYTES;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t o = (ks >> 2) * SUB_BYTES + (ks & 3) * 32;
-                    mma_ss(tS, smem_desc_sw128(sQ + o, 16, 1024), smem_desc_sw128(sK + o, 16, 1024), idesc_qk, ks > 0);
+                    mma_ss(tmem + g * 128, smem_desc_sw128(q0 + o, 16, 1024), smem_desc_sw128(k0 + o, 16, 1024), idesc_qk, ks > 0);
                 }
-                tc_commit(s_full);
-                if (!mbar_wait(p_full, par, abort_flag, p.status, W_PFULL)) break;
-                if (!mbar_wait(v_full, par, abort_flag, p.status, W_VFULL)) break;
-                tc_fence_after();
+            };
+            auto issue_pv = [&](int g, int st, int valid, bool accumulate) {
                 const int steps = (valid + 15) >> 4;
+                const uint32_t v0 = sV + st * TILE_BYTES;
                 for (int ks = 0; ks < steps; ++ks)
-                    mma_ts(tO, tP + ks * 8, smem_desc_sw128(sV + ks * 2048, SUB_BYTES, 1024), IDESC_PV, (jt > 0 || ks > 0));
-                tc_commit(pv_done);
-                ++jt;
+                    mma_ts(tmem + 256 + g * 128, tmem + g * 128 + ks * 8, smem_desc_sw128(v0 + ks * 2048, SUB_BYTES, 1024),
+                           IDESC_PV, accumulate || ks > 0);
+            };
+            TileIter it(w_rng, w_nrng);
+            int t0, valid, valid_next = 0;
+            bool ok = it.next(t0, valid);
+            // prologue: S0(0), S1(0)
+            ok = ok && mbar_wait(bar(Q_FULL + 0), 0, abort_flag, p.status, W_QFULL);
+            ok = ok && mbar_wait(bar(K_FULL + 0), 0, abort_flag, p.status, W_KFULL);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(0, 0, valid);
+                tc_commit(bar(S_FULL + 0));
+                if (two) {
+                    ok = mbar_wait(bar(Q_FULL + 1), 0, abort_flag, p.status, W_QFULL);
+                    if (ok) {
+                        tc_fence_after();
+                        issue_qk(1, 0, valid);
+                        tc_commit(bar(S_FULL + 1));
+                    }
+                }
+                tc_commit(bar(K_EMPTY + 0));
+            }
+            for (int jt = 0; ok && jt < n_tiles; ++jt) {
+                const int st = jt & 1, sn = (jt + 1) & 1;
+                const uint32_t ph = (jt >> 1) & 1, phn = ((jt + 1) >> 1) & 1;
+                const bool more = it.next(t0, valid_next);
+                if (!mbar_wait(bar(V_FULL + st), ph, abort_flag, p.status, W_VFULL)) break;
+                // group 0: O0 += P0 V(jt), then S0(jt + 1)
+                if (!mbar_wait(bar(P_FULL + 0), jt & 1, abort_flag, p.status, W_PFULL)) break;
+                tc_fence_after();
+                issue_pv(0, st, valid, jt > 0);
+                if (more) {
+                    if (!mbar_wait(bar(K_FULL + sn), phn, abort_flag, p.status, W_KFULL)) break;
+                    tc_fence_after();
+                    issue_qk(0, sn, valid_next);
+                    tc_commit(bar(S_FULL + 0));
+                } else {
+                    tc_commit(bar(O_FULL + 0));
+                }
+                // group 1
+                if (two) {
+                    if (!mbar_wait(bar(P_FULL + 1), jt & 1, abort_flag, p.status, W_PFULL)) break;
+                    tc_fence_after();
+                    issue_pv(1, st, valid, jt > 0);
+                }
+                tc_commit(bar(V_EMPTY + st));
+                if (more) {
+                    if (two) {
+                        issue_qk(1, sn, valid_next);
+                        tc_commit(bar(S_FULL + 1));
+                    }
+                    tc_commit(bar(K_EMPTY + sn));
+                } else if (two) {
+                    tc_commit(bar(O_FULL + 1));
+                }
+                valid = valid_next;
             }
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 8) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ---- host side
@@ -417,7 +507,9 @@ static int attend_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfl
     a.status = ws_ptr<int>(ws, p->ws.status);
     a.H = p->H; a.L = p->L; a.C = p->C; a.k = p->k;
     a.scale_log2 = p->scale * 1.4426950408889634f;
-    const size_t smem = 3 * (size_t)128 * D * 2 + 1024;
+    // always the d = 128 footprint: more than half an SM's shared memory, so CTAs (which each
+    // take all 512 TMEM columns) never share an SM
+    const size_t smem = 6 * (size_t)128 * 128 * 2 + 1024;
     static bool attr_done[2] = {false, false};
     if (!attr_done[D == 128]) {
         MOC_CUDA_TRY(cudaFuncSetAttribute(attend_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

@@ -10,7 +10,7 @@
 
 namespace moc {
 
-constexpr int kQTileRows = 128;     // query rows per attention tile
+constexpr int kQTileRows = 256;     // query rows per attention work item (two 128-row MMA tiles)
 constexpr int kPoolSlice = 256;     // tokens per chunk-pool work unit
 constexpr int kStatusWords = 16;    // status area at the head of the workspace (int32 each)
 
