@@ -152,7 +152,7 @@ def cpu_baseline(wl, budget_s: float):
     t0 = time.perf_counter()
     orc.attend(x["q"], x["k"], x["v"], sel, probe)
     per_row = (time.perf_counter() - t0) / len(probe)
-    n = int(max(64, min(20000, budget_s / max(per_row, 1e-6))))
+    n = int(max(64, min(2000000, budget_s / max(per_row, 1e-6))))
     rows = sample(n)
     t0 = time.perf_counter()
     orc.attend(x["q"], x["k"], x["v"], sel, rows)

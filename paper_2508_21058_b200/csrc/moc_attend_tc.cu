@@ -9,17 +9,19 @@
 //     one chunk); keys are the chunk's mandatory anchors (merged token ranges).  Its
 //     epilogue merges the row's <= k routed partials by log-sum-exp and writes O and LSE.
 //
-// One CTA per SM, 10 warps, two 128-row query tiles that share every K/V tile:
+// One CTA per SM, 11 warps, two 128-row query tiles that share every K/V tile:
 //   warps 0-3 / 4-7  softmax group of query tile 0 / 1, one row per thread (TMEM lane = row):
 //              load or gather Q into the swizzled shared tile, read S from TMEM, online
 //              softmax, write P back to TMEM as packed bf16 (aliasing S), lazily rescale O,
 //              epilogue;
 //   warp 8     TMA producer: K and V tiles of 128 keys, two stages each, 128-byte swizzle;
-//   warp 9     one thread issues the MMAs in the order  PV0(j), S0(j+1), PV1(j), S1(j+1), so
-//              one group's softmax overlaps the other group's MMAs.  S = Q K^T takes both
-//              operands from shared memory, O += P V takes P from TMEM and V as an MN-major
-//              shared-memory operand; all accumulators live in TMEM (S0, S1, O0, O1 = 512
-//              columns).
+//   warps 9, 10  one MMA-issuing thread per query tile g:  S_g(0), then  O_g += P_g V(j),
+//              S_g(j + 1)  per key tile.  The tensor pipe takes the next MMA only as the
+//              previous one retires, so an issuer that waits on a barrier idles the pipe; with
+//              one issuer per tile the other tile's MMAs fill that time, and one tile's softmax
+//              overlaps the other tile's MMAs.  S = Q K^T takes both operands from shared
+//              memory, O += P V takes P from TMEM and V as an MN-major shared-memory operand;
+//              all accumulators live in TMEM (S0, S1, O0, O1 = 512 columns).
 // Every mbarrier wait is bounded; a wait that runs out flags the workspace status word
 // and the CTA drains and leaves.
 #include "moc_common.cuh"
@@ -48,12 +50,12 @@ struct AttendParams {
 };
 
 constexpr int kBN = 128;               // keys per tile
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;
 constexpr int kTmemCols = 512;         // S0/P0 [0,128) S1/P1 [128,256) O0 [256,384) O1 [384,512)
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: O is rescaled only when the row max grows by more
 
-enum WaitCode { W_QFULL = 1, W_KFULL, W_VFULL, W_SFULL, W_PFULL, W_OFULL, W_KEMPTY, W_VEMPTY };
+enum WaitCode { W_QFULL = 1, W_KFULL, W_VFULL, W_SFULL, W_PFULL, W_OFULL, W_KEMPTY, W_VEMPTY, W_TURN };
 
 struct TileIter {
     const KeyRange *rng;
@@ -98,7 +100,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     constexpr int SUB = D / 64;            // 64-column (128-byte) sub-tiles per row
     constexpr int SUB_BYTES = 128 * 128;   // one sub-tile: 128 rows of 128 bytes
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[16];
+    __shared__ __align__(8) uint64_t bars[18];
     __shared__ uint32_t tmem_slot;
     __shared__ int s_abort;
     __shared__ int w_valid, w_h, w_rows, w_first, w_nrng, w_ntiles;
@@ -112,7 +114,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     const uint32_t sQ = sbase, sK = sbase + 2 * TILE_BYTES, sV = sbase + 4 * TILE_BYTES;
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     // barrier indices
-    constexpr int Q_FULL = 0, K_FULL = 2, K_EMPTY = 4, V_FULL = 6, V_EMPTY = 8, S_FULL = 10, P_FULL = 12, O_FULL = 14;
+    constexpr int Q_FULL = 0, K_FULL = 2, K_EMPTY = 4, V_FULL = 6, V_EMPTY = 8, S_FULL = 10, P_FULL = 12, O_FULL = 14, TURN = 16;
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -153,12 +155,13 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar(Q_FULL + t), 128);
             mbar_init(bar(K_FULL + t), 1);
-            mbar_init(bar(K_EMPTY + t), 1);
+            mbar_init(bar(K_EMPTY + t), valid && w_rows > 128 ? 2 : 1);   // one commit per MMA issuer
             mbar_init(bar(V_FULL + t), 1);
-            mbar_init(bar(V_EMPTY + t), 1);
+            mbar_init(bar(V_EMPTY + t), valid && w_rows > 128 ? 2 : 1);
             mbar_init(bar(S_FULL + t), 1);
             mbar_init(bar(P_FULL + t), 128);
             mbar_init(bar(O_FULL + t), 1);
+            mbar_init(bar(TURN + t), 128);
         }
         fence_barrier_init();
     }
@@ -242,6 +245,15 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                     alpha = exp2f(m_run - m_new);
                     m_run = m_new;
                 }
+                // The exponentials of the two query tiles take turns (tile 0 of key tile j, tile 1
+                // of j, tile 0 of j + 1, ...): each then has the special-function unit to itself
+                // while the other tile's MMAs run, instead of both drifting into lock step.
+                // TURN + g is arrived on by group g when its exponentials of a key tile are done.
+                if (two && (g == 1 || jt > 0)) {
+                    ok = mbar_wait(bar(TURN + (g ^ 1)), (g == 1 ? jt : jt - 1) & 1, abort_flag, p.status, W_TURN);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                }
                 // P = exp2(s * c - m), packed bf16 into the P columns (aliasing S)
                 const float neg_m = -m_run;
                 float ls0 = 0.f, ls1 = 0.f;
@@ -260,6 +272,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                     }
                     tmem_st16(tP + ch * 16, u);
                 }
+                if (two) mbar_arrive(bar(TURN + g));
                 if (__any_sync(0xffffffffu, alpha != 1.f)) {
                     // this group's PV of the previous tile has completed (its commit precedes this tile's S)
 #pragma unroll 1
@@ -383,44 +396,50 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             }
         }
     } else {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issuers (one per query tile)
+        const int g = warp - 9;
+        if (lane == 0 && (g == 0 || two)) {
             constexpr uint32_t IDESC_PV = idesc_bf16_f32(128, D, 0, 1);
+            // Descriptors are built once; inside the issue loops only the 14-bit start-address field
+            // (low word, 16-byte units) moves, so one tcgen05.mma costs the issuing thread a few
+            // integer instructions.
+            const uint64_t q_desc0 = smem_desc_sw128(sQ, 16, 1024), k_desc0 = smem_desc_sw128(sK, 16, 1024);
+            const uint64_t v_desc0 = smem_desc_sw128(sV, SUB_BYTES, 1024);
+            constexpr uint64_t STAGE = TILE_BYTES >> 4;   // next tile / next stage, in address-field units
             auto issue_qk = [&](int g, int st, int valid) {
                 const int n_qk = max(16, (valid + 15) & ~15);
                 const uint32_t idesc_qk = idesc_bf16_f32(128, n_qk, 0, 0);
-                const uint32_t q0 = sQ + g * TILE_BYTES, k0 = sK + st * TILE_BYTES;
+                const uint64_t qd = q_desc0 + (g ? STAGE : 0), kd = k_desc0 + (st ? STAGE : 0);
+                const uint32_t d_s = tmem + g * 128;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t o = (ks >> 2) * SUB_BYTES + (ks & 3) * 32;
-                    mma_ss(tmem + g * 128, smem_desc_sw128(q0 + o, 16, 1024), smem_desc_sw128(k0 + o, 16, 1024), idesc_qk, ks > 0);
+                    const uint32_t o = ((ks >> 2) * SUB_BYTES + (ks & 3) * 32) >> 4;
+                    mma_ss(d_s, qd + o, kd + o, idesc_qk, ks > 0);
                 }
             };
             auto issue_pv = [&](int g, int st, int valid, bool accumulate) {
-                const int steps = (valid + 15) >> 4;
-                const uint32_t v0 = sV + st * TILE_BYTES;
-                for (int ks = 0; ks < steps; ++ks)
-                    mma_ts(tmem + 256 + g * 128, tmem + g * 128 + ks * 8, smem_desc_sw128(v0 + ks * 2048, SUB_BYTES, 1024),
-                           IDESC_PV, accumulate || ks > 0);
+                const uint64_t vd = v_desc0 + (st ? STAGE : 0);
+                const uint32_t d_o = tmem + 256 + g * 128, a_p = tmem + g * 128;
+                if (valid == kBN) {
+                    mma_ts(d_o, a_p, vd, IDESC_PV, accumulate);
+#pragma unroll
+                    for (int ks = 1; ks < kBN / 16; ++ks) mma_ts(d_o, a_p + ks * 8, vd + ks * (2048 >> 4), IDESC_PV, 1);
+                } else {
+                    const int steps = (valid + 15) >> 4;
+                    for (int ks = 0; ks < steps; ++ks)
+                        mma_ts(d_o, a_p + ks * 8, vd + ks * (2048 >> 4), IDESC_PV, accumulate || ks > 0);
+                }
             };
+            // this issuer serves query tile g: S_g(0), then per key tile  O_g += P_g V(j),  S_g(j + 1)
             TileIter it(w_rng, w_nrng);
             int t0, valid, valid_next = 0;
             bool ok = it.next(t0, valid);
-            // prologue: S0(0), S1(0)
-            ok = ok && mbar_wait(bar(Q_FULL + 0), 0, abort_flag, p.status, W_QFULL);
+            ok = ok && mbar_wait(bar(Q_FULL + g), 0, abort_flag, p.status, W_QFULL);
             ok = ok && mbar_wait(bar(K_FULL + 0), 0, abort_flag, p.status, W_KFULL);
             if (ok) {
                 tc_fence_after();
-                issue_qk(0, 0, valid);
-                tc_commit(bar(S_FULL + 0));
-                if (two) {
-                    ok = mbar_wait(bar(Q_FULL + 1), 0, abort_flag, p.status, W_QFULL);
-                    if (ok) {
-                        tc_fence_after();
-                        issue_qk(1, 0, valid);
-                        tc_commit(bar(S_FULL + 1));
-                    }
-                }
+                issue_qk(g, 0, valid);
+                tc_commit(bar(S_FULL + g));
                 tc_commit(bar(K_EMPTY + 0));
             }
             for (int jt = 0; ok && jt < n_tiles; ++jt) {
@@ -428,33 +447,17 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 const uint32_t ph = (jt >> 1) & 1, phn = ((jt + 1) >> 1) & 1;
                 const bool more = it.next(t0, valid_next);
                 if (!mbar_wait(bar(V_FULL + st), ph, abort_flag, p.status, W_VFULL)) break;
-                // group 0: O0 += P0 V(jt), then S0(jt + 1)
-                if (!mbar_wait(bar(P_FULL + 0), jt & 1, abort_flag, p.status, W_PFULL)) break;
+                if (more && !mbar_wait(bar(K_FULL + sn), phn, abort_flag, p.status, W_KFULL)) break;
+                if (!mbar_wait(bar(P_FULL + g), jt & 1, abort_flag, p.status, W_PFULL)) break;
                 tc_fence_after();
-                issue_pv(0, st, valid, jt > 0);
-                if (more) {
-                    if (!mbar_wait(bar(K_FULL + sn), phn, abort_flag, p.status, W_KFULL)) break;
-                    tc_fence_after();
-                    issue_qk(0, sn, valid_next);
-                    tc_commit(bar(S_FULL + 0));
-                } else {
-                    tc_commit(bar(O_FULL + 0));
-                }
-                // group 1
-                if (two) {
-                    if (!mbar_wait(bar(P_FULL + 1), jt & 1, abort_flag, p.status, W_PFULL)) break;
-                    tc_fence_after();
-                    issue_pv(1, st, valid, jt > 0);
-                }
+                issue_pv(g, st, valid, jt > 0);
                 tc_commit(bar(V_EMPTY + st));
                 if (more) {
-                    if (two) {
-                        issue_qk(1, sn, valid_next);
-                        tc_commit(bar(S_FULL + 1));
-                    }
+                    issue_qk(g, sn, valid_next);
+                    tc_commit(bar(S_FULL + g));
                     tc_commit(bar(K_EMPTY + sn));
-                } else if (two) {
-                    tc_commit(bar(O_FULL + 1));
+                } else {
+                    tc_commit(bar(O_FULL + g));
                 }
                 valid = valid_next;
             }
