@@ -9,11 +9,13 @@
 //     one chunk); keys are the chunk's mandatory anchors (merged token ranges).  Its
 //     epilogue merges the row's <= k routed partials by log-sum-exp and writes O and LSE.
 //
-// One CTA per SM, 11 warps, two 128-row query tiles that share every K/V tile:
+// One CTA per SM, 12 warps in three warpgroups (the third gives most of its registers to the
+// other two), two 128-row query tiles that share every K/V tile:
 //   warps 0-3 / 4-7  softmax group of query tile 0 / 1, one row per thread (TMEM lane = row):
 //              load or gather Q into the swizzled shared tile, read S from TMEM, online
-//              softmax, write P back to TMEM as packed bf16 (aliasing S), lazily rescale O,
-//              epilogue;
+//              softmax, write P back to TMEM as packed bf16 (aliasing S; the first 64 keys are
+//              released to the issuer before the exponentials of the other 64), lazily rescale
+//              O, epilogue.  The exponentials of the two tiles take turns;
 //   warp 8     TMA producer: K and V tiles of 128 keys, two stages each, 128-byte swizzle;
 //   warps 9, 10  one MMA-issuing thread per query tile g:  S_g(0), then  O_g += P_g V(j),
 //              S_g(j + 1)  per key tile.  The tensor pipe takes the next MMA only as the
@@ -21,7 +23,8 @@
 //              one issuer per tile the other tile's MMAs fill that time, and one tile's softmax
 //              overlaps the other tile's MMAs.  S = Q K^T takes both operands from shared
 //              memory, O += P V takes P from TMEM and V as an MN-major shared-memory operand;
-//              all accumulators live in TMEM (S0, S1, O0, O1 = 512 columns).
+//              all accumulators live in TMEM (S0, S1, O0, O1 = 512 columns);
+//   warp 11    idle (fills the third warpgroup).
 // Every mbarrier wait is bounded; a wait that runs out flags the workspace status word
 // and the CTA drains and leaves.
 #include "moc_common.cuh"
@@ -30,6 +33,20 @@
 namespace moc {
 
 using namespace tc;
+
+// Optional cycle-stamp tracing of one CTA per pass (build with -DMOC_TRACE): each hook stores
+// clock64() into a slot of g_trace, read back with moc_trace_read().  Compiled out otherwise.
+#ifdef MOC_TRACE
+__device__ long long g_trace[8192];
+#define TRACE_CTA (blockIdx.x == (ROUTED ? 5000 : 1000) && (ROUTED || blockIdx.y == 3))
+#define TRACE(slot) do { if (TRACE_CTA) g_trace[(slot)] = clock64(); } while (0)
+#else
+#define TRACE(slot) ((void)0)
+#endif
+// slot map: 0 start, 1 TMEM ready, 10+g Q staged, 12+g epilogue begins, 14+g epilogue done;
+// softmax of tile g, key tile j: 100 + 1000 g + 8 j + {0 S ready, 1 S loaded, 2 max known,
+// 3 first half of P stored, 4 exponentials done, 5 P stored};  MMA issuer g: 2100 + 1000 g + 8 j +
+// {0 loop top, 1 K/V ready, 2 first half of P seen, 3 all of P seen, 4 P V issued, 5 next S issued}
 
 struct AttendParams {
     const __nv_bfloat16 *Q;
@@ -50,12 +67,13 @@ struct AttendParams {
 };
 
 constexpr int kBN = 128;               // keys per tile
-constexpr int kThreads = 352;
+constexpr int kThreads = 384;          // three warpgroups: softmax 0, softmax 1, {producer, two MMA issuers, one idle warp}
 constexpr int kTmemCols = 512;         // S0/P0 [0,128) S1/P1 [128,256) O0 [256,384) O1 [384,512)
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr float kRescaleThreshold = 8.0f;   // log2 units: O is rescaled only when the row max grows by more
+constexpr float kRescaleThreshold = 8.0f;
+   // log2 units: O is rescaled only when the row max grows by more
 
-enum WaitCode { W_QFULL = 1, W_KFULL, W_VFULL, W_SFULL, W_PFULL, W_OFULL, W_KEMPTY, W_VEMPTY, W_TURN };
+enum WaitCode { W_QFULL = 1, W_KFULL, W_VFULL, W_SFULL, W_PFULL, W_OFULL, W_KEMPTY, W_VEMPTY, W_TURN, W_PHALF };
 
 struct TileIter {
     const KeyRange *rng;
@@ -77,21 +95,36 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
-// (x0, x1) * (c, c) + (m, m) in one packed instruction
-__device__ __forceinline__ void fma2(float &r0, float &r1, float x0, float x1, float c, float m) {
-    asm("{ .reg .b64 p, q, r, d; mov.b64 p, {%2, %3}; mov.b64 q, {%4, %4}; mov.b64 r, {%5, %5}; "
-        "fma.rn.f32x2 d, p, q, r; mov.b64 {%0, %1}, d; }"
-        : "=f"(r0), "=f"(r1) : "f"(x0), "f"(x1), "f"(c), "f"(m));
+// two fp32 values in one 64-bit register pair, for the packed fp32 instructions
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
 }
-__device__ __forceinline__ void add2(float &a0, float &a1, float b0, float b1) {
-    asm("{ .reg .b64 p, q, d; mov.b64 p, {%0, %1}; mov.b64 q, {%2, %3}; add.rn.f32x2 d, p, q; mov.b64 {%0, %1}, d; }"
-        : "+f"(a0), "+f"(a1) : "f"(b0), "f"(b1));
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }
-__device__ __forceinline__ void mul2(float &a0, float &a1, float s) {
-    asm("{ .reg .b64 p, q, d; mov.b64 p, {%0, %1}; mov.b64 q, {%2, %2}; mul.rn.f32x2 d, p, q; mov.b64 {%0, %1}, d; }"
-        : "+f"(a0), "+f"(a1) : "f"(s));
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
 }
-
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// (lo, hi) -> packed bf16x2, round to nearest even
+__device__ __forceinline__ uint32_t bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
 template <int D, bool ROUTED>
 __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                 const __grid_constant__ CUtensorMap tmV,
@@ -100,7 +133,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     constexpr int SUB = D / 64;            // 64-column (128-byte) sub-tiles per row
     constexpr int SUB_BYTES = 128 * 128;   // one sub-tile: 128 rows of 128 bytes
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[18];
+    __shared__ __align__(8) uint64_t bars[20];
     __shared__ uint32_t tmem_slot;
     __shared__ int s_abort;
     __shared__ int w_valid, w_h, w_rows, w_first, w_nrng, w_ntiles;
@@ -114,8 +147,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     const uint32_t sQ = sbase, sK = sbase + 2 * TILE_BYTES, sV = sbase + 4 * TILE_BYTES;
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     // barrier indices
-    constexpr int Q_FULL = 0, K_FULL = 2, K_EMPTY = 4, V_FULL = 6, V_EMPTY = 8, S_FULL = 10, P_FULL = 12, O_FULL = 14, TURN = 16;
+    constexpr int Q_FULL = 0, K_FULL = 2, K_EMPTY = 4, V_FULL = 6, V_EMPTY = 8, S_FULL = 10, P_FULL = 12, O_FULL = 14, TURN = 16, P_HALF = 18;
 
+    if (threadIdx.x == 0) TRACE(0);
     if (threadIdx.x == 0) {
         s_abort = 0;
         int valid = (*(volatile int *)p.status == 0);
@@ -162,6 +196,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             mbar_init(bar(P_FULL + t), 128);
             mbar_init(bar(O_FULL + t), 1);
             mbar_init(bar(TURN + t), 128);
+            mbar_init(bar(P_HALF + t), 128);
         }
         fence_barrier_init();
     }
@@ -175,6 +210,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     __syncthreads();
     tc_fence_after();
 
+    if (threadIdx.x == 0) TRACE(1);
     const uint32_t tmem = tmem_slot;
     const int h = w_h, rows = w_rows, first = w_first, n_tiles = w_ntiles;
     const bool two = rows > 128;            // is query tile 1 populated?
@@ -182,6 +218,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
 
     if (warp < 8) {
         // ------------------------------------------------------------ softmax / epilogue groups
+        // the row-per-thread softmax holds a whole 128-key row of S in registers: take the
+        // registers the third warpgroup gives up
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         const int g = warp >> 2;                       // query tile of this group
         const int r = threadIdx.x & 127;               // row within the tile = TMEM lane
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
@@ -210,6 +249,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             }
             fence_proxy_async_smem();
             mbar_arrive(bar(Q_FULL + g));
+            if (r == 0) TRACE(10 + g);
 
             float m_run = -INFINITY, l_run = 0.f;
             const float c = p.scale_log2;
@@ -220,11 +260,13 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 ok = mbar_wait(bar(S_FULL + g), jt & 1, abort_flag, p.status, W_SFULL);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+                if (r == 0) TRACE(100 + g * 1000 + jt * 8 + 0);
                 tc_fence_after();
                 uint32_t v[4][32];
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) tmem_ld32(tS + ch * 32, v[ch]);
                 tmem_wait_ld();
+                if (r == 0) TRACE(100 + g * 1000 + jt * 8 + 1);
                 if (valid < kBN) {
 #pragma unroll
                     for (int ch = 0; ch < 4; ++ch)
@@ -232,12 +274,15 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                         for (int x = 0; x < 32; ++x)
                             if (ch * 32 + x >= valid) v[ch][x] = 0xff800000u;   // -inf
                 }
-                float mx = -INFINITY;
+                float m4[4];
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch)
+                for (int ch = 0; ch < 4; ++ch) {
+                    m4[ch] = -INFINITY;
 #pragma unroll
-                    for (int x = 0; x < 32; x += 2) mx = max3(mx, __uint_as_float(v[ch][x]), __uint_as_float(v[ch][x + 1]));
-                const float m_new = fmaxf(m_run, mx * c);
+                    for (int x = 0; x < 32; x += 2) m4[ch] = max3(m4[ch], __uint_as_float(v[ch][x]), __uint_as_float(v[ch][x + 1]));
+                }
+                const float m_new = fmaxf(m_run, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * c);
+                if (r == 0) TRACE(100 + g * 1000 + jt * 8 + 2);
                 float alpha = 1.f;
                 if (jt == 0) {
                     m_run = m_new;
@@ -246,33 +291,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                     m_run = m_new;
                 }
                 // The exponentials of the two query tiles take turns (tile 0 of key tile j, tile 1
-                // of j, tile 0 of j + 1, ...): each then has the special-function unit to itself
-                // while the other tile's MMAs run, instead of both drifting into lock step.
+                // of j, tile 0 of j + 1, ...): each then has the arithmetic pipes to itself while
+                // the other tile's MMAs run, instead of both drifting into lock step.
                 // TURN + g is arrived on by group g when its exponentials of a key tile are done.
                 if (two && (g == 1 || jt > 0)) {
                     ok = mbar_wait(bar(TURN + (g ^ 1)), (g == 1 ? jt : jt - 1) & 1, abort_flag, p.status, W_TURN);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                 }
-                // P = exp2(s * c - m), packed bf16 into the P columns (aliasing S)
-                const float neg_m = -m_run;
-                float ls0 = 0.f, ls1 = 0.f;
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t u[16];
-#pragma unroll
-                    for (int x = 0; x < 16; ++x) {
-                        float a0, a1;
-                        fma2(a0, a1, __uint_as_float(v[ch][2 * x]), __uint_as_float(v[ch][2 * x + 1]), c, neg_m);
-                        a0 = exp2f(a0);
-                        a1 = exp2f(a1);
-                        add2(ls0, ls1, a0, a1);
-                        __nv_bfloat162 b = __floats2bfloat162_rn(a0, a1);
-                        u[x] = *reinterpret_cast<uint32_t *>(&b);
-                    }
-                    tmem_st16(tP + ch * 16, u);
-                }
-                if (two) mbar_arrive(bar(TURN + g));
                 if (__any_sync(0xffffffffu, alpha != 1.f)) {
                     // this group's PV of the previous tile has completed (its commit precedes this tile's S)
 #pragma unroll 1
@@ -285,13 +311,45 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                         tmem_st32(tO + ch * 32, o);
                     }
                 }
+                // P = exp2(s * c - m), packed bf16 into the P columns (aliasing S).  The first 64 keys
+                // are handed to the MMA issuer as soon as they are stored: their P V product overlaps
+                // the exponentials of the other 64.
+                const uint64_t c2 = pack2(c, c), nm2 = pack2(-m_run, -m_run);
+                uint64_t sum_a = 0ull, sum_b = 0ull;   // two packed partial row sums
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t u[16];
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) {
+                        float a0, a1;
+                        unpack2(fma2(pack2(__uint_as_float(v[ch][2 * x]), __uint_as_float(v[ch][2 * x + 1])), c2, nm2), a0, a1);
+                        a0 = ex2(a0);
+                        a1 = ex2(a1);
+                        if (x & 1) sum_b = add2(sum_b, pack2(a0, a1));
+                        else sum_a = add2(sum_a, pack2(a0, a1));
+                        u[x] = bf16x2(a0, a1);
+                    }
+                    tmem_st16(tP + ch * 16, u);
+                    if (ch == 1) {
+                        tmem_wait_st();
+                        tc_fence_before();
+                        mbar_arrive(bar(P_HALF + g));
+                        if (r == 0) TRACE(100 + g * 1000 + jt * 8 + 3);
+                    }
+                }
+                if (r == 0) TRACE(100 + g * 1000 + jt * 8 + 4);
+                if (two) mbar_arrive(bar(TURN + g));
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(P_FULL + g));
-                l_run = l_run * alpha + (ls0 + ls1);
+                if (r == 0) TRACE(100 + g * 1000 + jt * 8 + 5);
+                float s0, s1;
+                unpack2(add2(sum_a, sum_b), s0, s1);
+                l_run = l_run * alpha + (s0 + s1);
                 ++jt;
             }
             // ---- epilogue
+            if (r == 0) TRACE(12 + g);
             if (ok) {
                 ok = mbar_wait(bar(O_FULL + g), 0, abort_flag, p.status, W_OFULL);
                 ok = __all_sync(0xffffffffu, ok);
@@ -361,6 +419,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             }
         }
     } else if (warp == 8) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             prefetch_tensormap(&tmK);
@@ -396,9 +455,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             }
         }
     } else {
-        // ------------------------------------------------------------ MMA issuers (one per query tile)
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        // ------------------------------------------------------------ MMA issuers (one per query tile); warp 11 idles
         const int g = warp - 9;
-        if (lane == 0 && (g == 0 || two)) {
+        if (lane == 0 && g < 2 && (g == 0 || two)) {
             constexpr uint32_t IDESC_PV = idesc_bf16_f32(128, D, 0, 1);
             // Descriptors are built once; inside the issue loops only the 14-bit start-address field
             // (low word, 16-byte units) moves, so one tcgen05.mma costs the issuing thread a few
@@ -417,17 +477,16 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                     mma_ss(d_s, qd + o, kd + o, idesc_qk, ks > 0);
                 }
             };
-            auto issue_pv = [&](int g, int st, int valid, bool accumulate) {
+            // k-steps [ks0, ks1) of  O_g += P_g V(stage st)  (16 keys each)
+            auto issue_pv = [&](int g, int st, int ks0, int ks1, bool accumulate) {
                 const uint64_t vd = v_desc0 + (st ? STAGE : 0);
                 const uint32_t d_o = tmem + 256 + g * 128, a_p = tmem + g * 128;
-                if (valid == kBN) {
-                    mma_ts(d_o, a_p, vd, IDESC_PV, accumulate);
+                if (ks1 - ks0 == 4) {
 #pragma unroll
-                    for (int ks = 1; ks < kBN / 16; ++ks) mma_ts(d_o, a_p + ks * 8, vd + ks * (2048 >> 4), IDESC_PV, 1);
+                    for (int ks = 0; ks < 4; ++ks)
+                        mma_ts(d_o, a_p + (ks0 + ks) * 8, vd + (ks0 + ks) * (2048 >> 4), IDESC_PV, accumulate || ks > 0);
                 } else {
-                    const int steps = (valid + 15) >> 4;
-                    for (int ks = 0; ks < steps; ++ks)
-                        mma_ts(d_o, a_p + ks * 8, vd + ks * (2048 >> 4), IDESC_PV, accumulate || ks > 0);
+                    for (int ks = ks0; ks < ks1; ++ks) mma_ts(d_o, a_p + ks * 8, vd + ks * (2048 >> 4), IDESC_PV, accumulate || ks > ks0);
                 }
             };
             // this issuer serves query tile g: S_g(0), then per key tile  O_g += P_g V(j),  S_g(j + 1)
@@ -446,11 +505,20 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 const int st = jt & 1, sn = (jt + 1) & 1;
                 const uint32_t ph = (jt >> 1) & 1, phn = ((jt + 1) >> 1) & 1;
                 const bool more = it.next(t0, valid_next);
+                TRACE(2100 + g * 1000 + jt * 8 + 0);
                 if (!mbar_wait(bar(V_FULL + st), ph, abort_flag, p.status, W_VFULL)) break;
                 if (more && !mbar_wait(bar(K_FULL + sn), phn, abort_flag, p.status, W_KFULL)) break;
-                if (!mbar_wait(bar(P_FULL + g), jt & 1, abort_flag, p.status, W_PFULL)) break;
+                TRACE(2100 + g * 1000 + jt * 8 + 1);
+                const int steps = (valid + 15) >> 4, half = min(steps, 4);
+                if (!mbar_wait(bar(P_HALF + g), jt & 1, abort_flag, p.status, W_PHALF)) break;
+                TRACE(2100 + g * 1000 + jt * 8 + 2);
                 tc_fence_after();
-                issue_pv(g, st, valid, jt > 0);
+                issue_pv(g, st, 0, half, jt > 0);
+                if (!mbar_wait(bar(P_FULL + g), jt & 1, abort_flag, p.status, W_PFULL)) break;
+                TRACE(2100 + g * 1000 + jt * 8 + 3);
+                tc_fence_after();
+                if (steps > half) issue_pv(g, st, half, steps, true);
+                TRACE(2100 + g * 1000 + jt * 8 + 4);
                 tc_commit(bar(V_EMPTY + st));
                 if (more) {
                     issue_qk(g, sn, valid_next);
@@ -459,10 +527,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 } else {
                     tc_commit(bar(O_FULL + g));
                 }
+                TRACE(2100 + g * 1000 + jt * 8 + 5);
                 valid = valid_next;
             }
         }
     }
+    if (warp < 8 && (threadIdx.x & 127) == 0) TRACE(14 + (warp >> 2));
     tc_fence_before();
     __syncthreads();
     if (warp == 8) tmem_dealloc(tmem, kTmemCols);
@@ -529,6 +599,12 @@ static int attend_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfl
     MOC_LAUNCH_CHECK();
     return MOC_OK;
 }
+
+#ifdef MOC_TRACE
+extern "C" int moc_trace_read(long long *host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * (size_t)n);
+}
+#endif
 
 int launch_attend_tc(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
                      const int32_t *, __nv_bfloat16 *O, float *lse, void *ws, cudaStream_t s) {
