@@ -207,7 +207,8 @@ __global__ void __launch_bounds__(128) dkv_scalar_kernel(const __nv_bfloat16 *__
                                                           __nv_bfloat16 *__restrict__ dK, __nv_bfloat16 *__restrict__ dV,
                                                           const int32_t *__restrict__ off, const int32_t *__restrict__ tok_chunk,
                                                           const int32_t *__restrict__ ranc_off, const int32_t *__restrict__ ranc,
-                                                          const int *__restrict__ qoff, const int32_t *__restrict__ qlist,
+                                                          const int *__restrict__ cnt, const int32_t *__restrict__ cap_off,
+                                                          const int32_t *__restrict__ qlist, size_t cap_total,
                                                           int H, int L, int C, int k, float scale) {
     constexpr int E = D / 32;
     __shared__ float ks[4][D], vs[4][D];
@@ -227,8 +228,8 @@ __global__ void __launch_bounds__(128) dkv_scalar_kernel(const __nv_bfloat16 *__
 #pragma unroll
     for (int e = 0; e < E; ++e) { ak[e] = 0.f; av[e] = 0.f; }
     const int n_ra = ranc_off[j + 1] - ranc_off[j];
-    const int q0 = qoff[h * (C + 1) + j], q1 = qoff[h * (C + 1) + j + 1];
-    const int32_t *list = qlist + (size_t)h * L * (k ? k : 1);
+    const int q0 = cap_off[j], q1 = q0 + cnt[h * C + j];
+    const int32_t *list = qlist + (size_t)h * cap_total;
     // segments: n_ra query-chunk ranges, then the routed list
     for (int seg = 0; seg <= n_ra; ++seg) {
         int b0, b1;
@@ -289,7 +290,8 @@ static int attend_bwd_scalar_d(const moc_plan *p, const __nv_bfloat16 *Q, const 
                                              p->d_anc_rng, p->H, p->L, p->k, p->scale);
     MOC_LAUNCH_CHECK();
     dkv_scalar_kernel<D><<<grid, 128, 0, s>>>(Q, K, V, dO, lse, delta, dK, dV, p->d_off, p->d_tok_chunk, p->d_ranc_off,
-                                              p->d_ranc, ws_ptr<int>(ws, p->ws.qoff), ws_ptr<int32_t>(ws, p->ws.qlist),
+                                              p->d_ranc, ws_ptr<int>(ws, p->ws.cnt), p->d_cap_off, ws_ptr<int32_t>(ws, p->ws.qlist),
+                                              (size_t)p->cap_off[p->C],
                                               p->H, p->L, p->C, p->k, p->scale);
     MOC_LAUNCH_CHECK();
     return MOC_OK;

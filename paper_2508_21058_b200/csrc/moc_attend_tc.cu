@@ -59,8 +59,10 @@ struct AttendParams {
     const KeyRange *anc_rng;
     const QTile *qtiles;
     const int *gtile_off;   // [H*C + 1] running count of routed tiles over (head, chunk)
-    const int *qoff;        // [H][C + 1]
-    const int32_t *qlist;   // [H][L * k]
+    const int *cnt;         // [H][C] picks per (head, chunk)
+    const int32_t *cap_off; // [C + 1] start of chunk c's list inside a head's list area
+    const int32_t *qlist;   // [H][cap_total]
+    size_t cap_total;
     int *status;
     int H, L, C, k;
     float scale_log2;       // softmax scale * log2(e)
@@ -165,10 +167,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 }
                 const int h = lo / p.C, c = lo % p.C;
                 const int nth = tile - p.gtile_off[lo];
-                const int e0 = p.qoff[h * (p.C + 1) + c] + nth * kQTileRows;
                 w_h = h;
-                w_first = e0;
-                w_rows = min(kQTileRows, p.qoff[h * (p.C + 1) + c + 1] - e0);
+                w_first = p.cap_off[c] + nth * kQTileRows;
+                w_rows = min(kQTileRows, p.cnt[lo] - nth * kQTileRows);
                 w_rng0 = KeyRange{p.off[c], p.off[c + 1]};
                 w_rng = &w_rng0;
                 w_nrng = 1;
@@ -230,7 +231,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             int qi = -1, slot = 0;
             if (rt < rows) {
                 if (ROUTED) {
-                    const int e = p.qlist[(size_t)h * p.L * p.k + first + rt];
+                    const int e = p.qlist[(size_t)h * p.cap_total + first + rt];
                     qi = e / p.k;
                     slot = e - qi * p.k;
                 } else {
@@ -575,8 +576,10 @@ static int attend_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfl
     a.part_lse = ws_ptr<float>(ws, p->ws.part_lse);
     a.off = p->d_off; a.anc_off = p->d_anc_off; a.anc_rng = p->d_anc_rng; a.qtiles = p->d_qtiles;
     a.gtile_off = ws_ptr<int>(ws, p->ws.tile_off);
-    a.qoff = ws_ptr<int>(ws, p->ws.qoff);
+    a.cnt = ws_ptr<int>(ws, p->ws.cnt);
+    a.cap_off = p->d_cap_off;
     a.qlist = ws_ptr<int32_t>(ws, p->ws.qlist);
+    a.cap_total = (size_t)p->cap_off[p->C];
     a.status = ws_ptr<int>(ws, p->ws.status);
     a.H = p->H; a.L = p->L; a.C = p->C; a.k = p->k;
     a.scale_log2 = p->scale * 1.4426950408889634f;

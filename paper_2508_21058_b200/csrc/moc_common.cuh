@@ -22,12 +22,10 @@ struct QTile { int32_t chunk, row0, rows, pad; };
 
 struct WsLayout {
     size_t status;      // int32[kStatusWords]: [0] device status, [1] detail, [2] routed-flag
-    size_t cnt;         // int32[H][C]     routed picks per (head, chunk)
-    size_t qoff;        // int32[H][C+1]   CSR offsets of the query lists
-    size_t cursor;      // int32[H][C]     scatter cursors
-    size_t gcnt;        // int32[H*C+1]    running pick count over (head, chunk) pairs
-    size_t tile_off;    // int32[H*C+1]    running count of 128-row routed tiles over (head, chunk) pairs
-    size_t qlist;       // int32[H][L*k]   entries i*k+s, grouped by chunk
+    size_t cnt;         // int32[H][C]     routed picks per (head, chunk); doubles as the list cursor while routing
+    size_t tile_off;    // int32[H*C+1]    running count of routed attention tiles over (head, chunk) pairs
+    size_t qlist;       // int32[H][cap_total]  per (head, chunk) list at cap_off[c]: entries i*k+s of the picks of c
+    size_t desc3;       // bf16 [H][3][Cpad][d]  descriptors split into three bf16 terms (hi + mid + lo)
     size_t pool_part;   // float[H][n_pool_units][d] partial key sums
     size_t pool_done;   // int32[H][C] arrival counters (self-resetting)
     size_t part_o;      // bf16 [H][L][k][d] routed partial outputs (normalised)
@@ -56,10 +54,12 @@ struct moc_plan {
     std::vector<moc::QTile> qtiles;
     std::vector<int32_t> pool_unit_off;      // [C+1] prefix of pool units per chunk
     int words;                               // uint32 words per anchor bitmap row
+    std::vector<int32_t> cap_off;            // [C+1] start of chunk c's query list inside a head's list area
+    int c_pad;                               // C rounded up to a multiple of 16 (MMA N granularity)
     int n_pool_units;
     // device tables (one allocation)
     void *d_blob;
-    int32_t *d_off, *d_shot, *d_tok_chunk, *d_anc_off, *d_ranc_off, *d_ranc, *d_pool_unit_off, *d_pool_unit_chunk;
+    int32_t *d_off, *d_shot, *d_tok_chunk, *d_anc_off, *d_ranc_off, *d_ranc, *d_pool_unit_off, *d_pool_unit_chunk, *d_cap_off;
     uint8_t *d_mod;
     uint32_t *d_anc_bits;
     moc::KeyRange *d_anc_rng;

@@ -1,6 +1,7 @@
 // Plan object (validated problem + derived chunk tables on the device), workspace layout,
 // argument checking and the C entry points.
 #include <math.h>
+#include <algorithm>
 #include <string.h>
 #include <mutex>
 #include <new>
@@ -39,11 +40,9 @@ static void layout_workspace(moc_plan *p) {
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
     w.status = take(sizeof(int32_t) * kStatusWords);
     w.cnt = take(sizeof(int32_t) * H * C);
-    w.qoff = take(sizeof(int32_t) * H * (C + 1));
-    w.cursor = take(sizeof(int32_t) * H * C);
-    w.gcnt = take(sizeof(int32_t) * (H * C + 1));
     w.tile_off = take(sizeof(int32_t) * (H * C + 1));
-    w.qlist = take(sizeof(int32_t) * H * L * (k ? k : 1));
+    w.qlist = take(sizeof(int32_t) * H * (size_t)std::max(p->cap_off[C], 1));
+    w.desc3 = take(sizeof(__nv_bfloat16) * H * 3 * (size_t)p->c_pad * d);
     w.pool_part = take(sizeof(float) * H * (size_t)p->n_pool_units * d);
     w.pool_done = take(sizeof(int32_t) * H * C);
     w.part_o = take(sizeof(__nv_bfloat16) * H * L * k * d);
@@ -129,6 +128,17 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
         for (int u = 0; u < units; ++u) unit_chunk.push_back(c);
     }
     p->n_pool_units = p->pool_unit_off[C];
+    // Query-list capacities: chunk c can be picked by at most the rows after it (causal) or by
+    // every row (non-causal); the lists sit back to back at these fixed offsets, so routing can
+    // append to them without a counting pass.
+    p->cap_off.assign(C + 1, 0);
+    for (int c = 0; c < C; ++c) {
+        const int64_t cap = p->k == 0 ? 0 : ((p->flags & MOC_FLAG_CAUSAL) ? L - p->off[c + 1] : L);
+        const int64_t next = (int64_t)p->cap_off[c] + cap;
+        if (next >= 2147483647LL) { delete p; return MOC_ERR_SHAPE; }
+        p->cap_off[c + 1] = (int32_t)next;
+    }
+    p->c_pad = (C + 15) / 16 * 16;
     layout_workspace(p);
 
     // one device blob
@@ -137,7 +147,7 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
     size_t o_off = take(4 * (C + 1)), o_shot = take(4 * C), o_mod = take(C), o_tok = take(4 * (size_t)L);
     size_t o_bits = take(4 * bits.size()), o_aoff = take(4 * (C + 1)), o_arng = take(sizeof(KeyRange) * p->anc_rng.size());
     size_t o_roff = take(4 * (C + 1)), o_ranc = take(4 * p->ranc.size()), o_qt = take(sizeof(QTile) * p->qtiles.size());
-    size_t o_puo = take(4 * (C + 1)), o_puc = take(4 * unit_chunk.size());
+    size_t o_puo = take(4 * (C + 1)), o_puc = take(4 * unit_chunk.size()), o_cap = take(4 * (C + 1));
     cudaError_t e = cudaMalloc(&p->d_blob, o);
     if (e != cudaSuccess) { set_cuda_error(e, "cudaMalloc(plan tables)"); delete p; return MOC_ERR_CUDA; }
     char *b = static_cast<char *>(p->d_blob);
@@ -149,7 +159,8 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
                         up(o_aoff, p->anc_off.data(), 4 * (C + 1)), up(o_arng, p->anc_rng.data(), sizeof(KeyRange) * p->anc_rng.size()),
                         up(o_roff, p->ranc_off.data(), 4 * (C + 1)), up(o_ranc, p->ranc.data(), 4 * p->ranc.size()),
                         up(o_qt, p->qtiles.data(), sizeof(QTile) * p->qtiles.size()),
-                        up(o_puo, p->pool_unit_off.data(), 4 * (C + 1)), up(o_puc, unit_chunk.data(), 4 * unit_chunk.size())};
+                        up(o_puo, p->pool_unit_off.data(), 4 * (C + 1)), up(o_puc, unit_chunk.data(), 4 * unit_chunk.size()),
+                        up(o_cap, p->cap_off.data(), 4 * (C + 1))};
     for (cudaError_t x : es)
         if (x != cudaSuccess) { set_cuda_error(x, "cudaMemcpy(plan tables)"); cudaFree(p->d_blob); delete p; return MOC_ERR_CUDA; }
     p->d_off = (int32_t *)(b + o_off); p->d_shot = (int32_t *)(b + o_shot); p->d_mod = (uint8_t *)(b + o_mod);
@@ -157,6 +168,7 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
     p->d_anc_off = (int32_t *)(b + o_aoff); p->d_anc_rng = (KeyRange *)(b + o_arng);
     p->d_ranc_off = (int32_t *)(b + o_roff); p->d_ranc = (int32_t *)(b + o_ranc); p->d_qtiles = (QTile *)(b + o_qt);
     p->d_pool_unit_off = (int32_t *)(b + o_puo); p->d_pool_unit_chunk = (int32_t *)(b + o_puc);
+    p->d_cap_off = (int32_t *)(b + o_cap);
     *out = p;
     return MOC_OK;
 }

@@ -3,18 +3,41 @@
 // and the inverse index (per head and chunk, the list of (query, slot) pairs that
 // picked it) which the key-stationary attention pass consumes.
 //
-// route_kernel: one query per thread, 128 queries per block.  The Q tile is staged in
-// shared memory with coalesced 128-bit loads; descriptors are visited in blocks of 32
-// chunks held in shared memory as fp32 and read as warp-wide broadcasts; each thread
-// keeps 32 fp32 accumulators and folds them into its running sorted top-k list.
+// The scores are a dense [L, d] x [d, C] contraction per head, so they run on the tensor
+// cores.  Q is bf16 already; each fp32 descriptor is split once into three bf16 terms
+// (hi + mid + lo carries its 24-bit mantissa), and S = Q hi^T + Q mid^T + Q lo^T is
+// accumulated in fp32 in TMEM: every product is exact, only the fp32 accumulation rounds.
+//
+// route_prep_kernel   splits the descriptors, clears the pick counters and the status words.
+// route_tc_kernel     persistent, one CTA per SM, each owning a contiguous range of
+//                     (head, 128-query tile) units:
+//     warp 0      TMA producer: Q tiles (ring of stages) and the head's descriptor block;
+//     warp 1      MMA issuer: 3 x d/16 MMAs per 128 chunks into one of two TMEM accumulators;
+//     warps 2-5 / 6-9   two selection groups (even / odd units), one query per thread (TMEM
+//                 lane = query): read the scores 32 chunks at a time, drop non-candidates,
+//                 keep a sorted top-k in registers, then write sel_idx and append the picks
+//                 to the per-(head, chunk) query lists (tile-local ranks from a shared-memory
+//                 histogram, one global atomic per (tile, chunk) to reserve the range).
+//   The descriptor block of a head stays in shared memory while the CTA's units stay in that
+//   head (C <= 192); with more chunks it is streamed in blocks of 128.
+// route_tiles_kernel  running count of attention tiles over (head, chunk) from the pick counts.
+// Every mbarrier wait is bounded; a wait that runs out flags the workspace status word.
 #include <float.h>
+#include <algorithm>
 
 #include "moc_common.cuh"
+#include "moc_tc.cuh"
 
 namespace moc {
 
-constexpr int kRouteRows = 128;
-constexpr int kRouteCB = 32;   // chunks per descriptor block (= bits of one anchor word)
+using namespace tc;
+
+constexpr int kRtRows = 128;          // queries per tile
+constexpr int kRtThreads = 320;
+constexpr int kRtResident = 192;      // up to this many (padded) chunks the whole block stays resident
+constexpr int kRtBlock = 128;         // otherwise chunks are streamed in blocks of this many
+
+enum RouteWait { RW_QFULL = 32, RW_QEMPTY, RW_DFULL, RW_DEMPTY, RW_ACCFULL, RW_ACCEMPTY, RW_GROUP };
 
 template <int KMAX>
 struct TopK {
@@ -45,159 +68,332 @@ struct TopK {
     }
 };
 
-template <int D, int KMAX>
-__global__ void __launch_bounds__(kRouteRows) route_kernel(const __nv_bfloat16 *__restrict__ Q,
-                                                            const float *__restrict__ desc, int32_t *__restrict__ sel,
-                                                            int *__restrict__ cnt, float *__restrict__ part_lse,
-                                                            const int32_t *__restrict__ tok_chunk,
-                                                            const uint32_t *__restrict__ anc_bits, int words, int L,
-                                                            int C, int k, int causal) {
-    constexpr int QS = D + 8;   // padded row stride (bf16 elements): conflict-free 16-byte row reads
-    extern __shared__ __align__(16) unsigned char smem[];
-    __nv_bfloat16 *qs = reinterpret_cast<__nv_bfloat16 *>(smem);
-    float *ds = reinterpret_cast<float *>(smem + sizeof(__nv_bfloat16) * kRouteRows * QS);
-    int *hist = reinterpret_cast<int *>(ds + kRouteCB * D);
-    const int h = blockIdx.y, r0 = blockIdx.x * kRouteRows;
-    const int rows = min(kRouteRows, L - r0);
-    const int tid = threadIdx.x;
-    // stage the Q tile
-    {
-        constexpr int LANES = D / 8;
-        const uint4 *src = reinterpret_cast<const uint4 *>(Q + ((size_t)h * L + r0) * D);
-        for (int e = tid; e < rows * LANES; e += kRouteRows) {
-            int r = e / LANES, l = e % LANES;
-            *reinterpret_cast<uint4 *>(qs + r * QS + l * 8) = __ldg(src + e);
-        }
-    }
-    for (int x = tid; x < C; x += kRouteRows) hist[x] = 0;
-    const int i = r0 + tid;
-    const bool live = tid < rows;
-    const int ci = live ? tok_chunk[i] : 0;
-    const int c_hi = causal ? tok_chunk[r0 + rows - 1] : C;   // exclusive bound on useful chunks for this tile
-    TopK<KMAX> top;
-    top.init();
-    for (int jb = 0; jb < c_hi; jb += kRouteCB) {
-        __syncthreads();
-        const int nb = min(kRouteCB, C - jb);
-        {
-            const float4 *src = reinterpret_cast<const float4 *>(desc + ((size_t)h * C + jb) * D);
-            for (int e = tid; e < nb * D / 4; e += kRouteRows) reinterpret_cast<float4 *>(ds)[e] = __ldg(src + e);
-        }
-        __syncthreads();
-        float acc[kRouteCB];
-#pragma unroll
-        for (int c = 0; c < kRouteCB; ++c) acc[c] = 0.f;
-#pragma unroll 1
-        for (int x0 = 0; x0 < D; x0 += 8) {
-            float q[8];
-            {
-                uint4 v = *reinterpret_cast<const uint4 *>(qs + tid * QS + x0);
-                const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&v);
-#pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                    float2 f = __bfloat1622float2(b[x]);
-                    q[2 * x] = f.x; q[2 * x + 1] = f.y;
-                }
-            }
-#pragma unroll
-            for (int c = 0; c < kRouteCB; ++c) {
-                float4 a = *reinterpret_cast<const float4 *>(ds + c * D + x0);
-                float4 b = *reinterpret_cast<const float4 *>(ds + c * D + x0 + 4);
-                acc[c] = fmaf(q[0], a.x, acc[c]); acc[c] = fmaf(q[1], a.y, acc[c]);
-                acc[c] = fmaf(q[2], a.z, acc[c]); acc[c] = fmaf(q[3], a.w, acc[c]);
-                acc[c] = fmaf(q[4], b.x, acc[c]); acc[c] = fmaf(q[5], b.y, acc[c]);
-                acc[c] = fmaf(q[6], b.z, acc[c]); acc[c] = fmaf(q[7], b.w, acc[c]);
-            }
-        }
-        if (live) {
-            const uint32_t aw = anc_bits[(size_t)ci * words + jb / 32];
-#pragma unroll
-            for (int c = 0; c < kRouteCB; ++c) {
-                const int j = jb + c;
-                const bool cand = (c < nb) && !((aw >> c) & 1u) && (!causal || j < ci);
-                if (cand) top.push(acc[c], j, k);
-            }
-        }
-    }
-    __syncthreads();
-    if (live) {
-        int32_t *out = sel + ((size_t)h * L + i) * k;
-        float *pl = part_lse + ((size_t)h * L + i) * k;   // empty slots never get a routed partial
-        if (KMAX <= 8) {
-#pragma unroll
-            for (int x = 0; x < (KMAX <= 8 ? KMAX : 1); ++x) {
-                if (x < k) {
-                    out[x] = top.j[x];
-                    if (top.j[x] >= 0) atomicAdd(&hist[top.j[x]], 1);
-                    else pl[x] = -INFINITY;
-                }
-            }
-        } else {
-            for (int x = 0; x < k; ++x) {
-                const int j = top.j[x];
-                out[x] = j;
-                if (j >= 0) atomicAdd(&hist[j], 1);
-                else pl[x] = -INFINITY;
-            }
-        }
-    }
-    __syncthreads();
-    for (int x = tid; x < C; x += kRouteRows)
-        if (hist[x]) atomicAdd(&cnt[h * C + x], hist[x]);
+// desc3[h][t][c][:] for t = 0, 1, 2: bf16 terms of desc[h][c][:] (rows c >= C are zero);
+// also clears the pick counters and the status words.
+__global__ void route_prep_kernel(const float *__restrict__ desc, __nv_bfloat16 *__restrict__ desc3, int *__restrict__ cnt,
+                                  int *__restrict__ status, int H, int C, int c_pad, int d) {
+    const size_t n = (size_t)H * c_pad * d;
+    const size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
+    if (i < (size_t)H * C) cnt[i] = 0;
+    if (i < kStatusWords) status[i] = 0;
+    if (i >= n) return;
+    const int x = (int)(i % d);
+    const int c = (int)((i / d) % c_pad);
+    const int h = (int)(i / ((size_t)d * c_pad));
+    float v = c < C ? desc[((size_t)h * C + c) * d + x] : 0.f;
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    v -= __bfloat162float(hi);
+    const __nv_bfloat16 mid = __float2bfloat16_rn(v);
+    v -= __bfloat162float(mid);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(v);
+    const size_t plane = (size_t)c_pad * d, base = (size_t)h * 3 * plane + (size_t)c * d + x;
+    desc3[base] = hi;
+    desc3[base + plane] = mid;
+    desc3[base + 2 * plane] = lo;
 }
 
-// Running totals over the H*C (head, chunk) pairs in one block: gcnt[i] = picks before pair i,
-// gtile[i] = 128-row tiles before pair i (both with a final total entry), cursors zeroed;
-// then qoff[h][c] = picks of head h before chunk c.  Flags the workspace as routed.
-__global__ void __launch_bounds__(1024) route_scan_kernel(const int *__restrict__ cnt, int *__restrict__ gcnt,
-                                                          int *__restrict__ gtile, int *__restrict__ qoff,
-                                                          int *__restrict__ cursor, int *__restrict__ status, int H, int C) {
-    __shared__ int sc[1024], st[1024];
-    const int HC = H * C, t = threadIdx.x;
+struct RouteParams {
+    int32_t *sel;
+    float *part_lse;
+    int *cnt;
+    int32_t *qlist;
+    const int32_t *tok_chunk;
+    const uint32_t *anc_bits;
+    const int32_t *cap_off;
+    int *status;
+    int H, L, C, c_pad, k, words, causal;
+    int tiles_per_head;     // ceil(L / 128)
+    int sb_rows;            // chunks per descriptor block held in shared memory
+    int q_stages;
+    size_t cap_total;
+};
+
+// number of descriptor blocks a tile needs: those that hold a chunk some row of the tile may pick
+__device__ __forceinline__ int blocks_needed(const RouteParams &p, int t) {
+    int c_hi = p.C;
+    if (p.causal) c_hi = p.tok_chunk[min(p.L, (t + 1) * kRtRows) - 1];   // picks are strictly earlier chunks
+    return max(1, (c_hi + p.sb_rows - 1) / p.sb_rows);
+}
+
+template <int D, int KMAX>
+__global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
+                                                                 const __grid_constant__ CUtensorMap tmD,
+                                                                 const RouteParams p) {
+    constexpr int SUB = D / 64;
+    constexpr int Q_SUB_BYTES = kRtRows * 128, Q_TILE_BYTES = SUB * Q_SUB_BYTES;
+    constexpr int kMaxStages = 4;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bars[2 * kMaxStages + 8];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int s_abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gbase = smem_raw + (sbase - smem_u32(smem_raw));
+    // shared memory: descriptor block (3 terms x SUB sub-tiles of sb_rows x 128 bytes) | Q stages | two histograms
+    const int d_sub_bytes = p.sb_rows * 128;
+    const uint32_t sD = sbase;
+    const uint32_t sQ = sD + ((3 * SUB * d_sub_bytes + 1023) & ~1023);
+    int *hist_base = reinterpret_cast<int *>(gbase + (sQ - sbase) + p.q_stages * Q_TILE_BYTES);
+    auto bar = [&](int i) { return smem_u32(&bars[i]); };
+    constexpr int Q_FULL = 0, Q_EMPTY = kMaxStages, D_FULL = 2 * kMaxStages, D_EMPTY = D_FULL + 1, ACC_FULL = D_FULL + 2,
+                  ACC_EMPTY = D_FULL + 4, GROUP = D_FULL + 6;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int t = 0; t < kMaxStages; ++t) { mbar_init(bar(Q_FULL + t), 1); mbar_init(bar(Q_EMPTY + t), 1); }
+        mbar_init(bar(D_FULL), 1);
+        mbar_init(bar(D_EMPTY), 1);
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(bar(ACC_FULL + t), 1);
+            mbar_init(bar(ACC_EMPTY + t), 128);
+            mbar_init(bar(GROUP + t), 128);
+        }
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+    volatile int *abort_flag = &s_abort;
+
+    // this CTA's units: a contiguous range of (head, tile), so the descriptor block changes rarely
+    const long long U = (long long)p.H * p.tiles_per_head;
+    const int u0 = (int)(U * blockIdx.x / gridDim.x), u1 = (int)(U * (blockIdx.x + 1) / gridDim.x);
+    constexpr int ACC_COLS = 256;   // TMEM columns per accumulator (sb_rows <= 192)
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            prefetch_tensormap(&tmQ);
+            prefetch_tensormap(&tmD);
+            int res_h = -1, res_sb = -1, qn = 0, dn = 0;
+            bool ok = true;
+            for (int u = u0; ok && u < u1; ++u) {
+                const int h = u / p.tiles_per_head, t = u % p.tiles_per_head;
+                const int n_sb = blocks_needed(p, t);
+                for (int sb = 0; ok && sb < n_sb; ++sb) {
+                    if (sb == 0) {
+                        const int st = qn % p.q_stages;
+                        ok = mbar_wait(bar(Q_EMPTY + st), ((qn / p.q_stages) & 1) ^ 1, abort_flag, p.status, RW_QEMPTY);
+                        if (!ok) break;
+                        mbar_expect_tx(bar(Q_FULL + st), Q_TILE_BYTES);
+#pragma unroll
+                        for (int sub = 0; sub < SUB; ++sub)
+                            tma_load_2d(sQ + st * Q_TILE_BYTES + sub * Q_SUB_BYTES, &tmQ, sub * 64, h * p.L + t * kRtRows, bar(Q_FULL + st));
+                        ++qn;
+                    }
+                    if (h != res_h || sb != res_sb) {
+                        ok = mbar_wait(bar(D_EMPTY), (dn & 1) ^ 1, abort_flag, p.status, RW_DEMPTY);
+                        if (!ok) break;
+                        mbar_expect_tx(bar(D_FULL), 3 * SUB * d_sub_bytes);
+                        for (int term = 0; term < 3; ++term)
+#pragma unroll
+                            for (int sub = 0; sub < SUB; ++sub)
+                                tma_load_2d(sD + (term * SUB + sub) * d_sub_bytes, &tmD, sub * 64,
+                                            (h * 3 + term) * p.c_pad + sb * p.sb_rows, bar(D_FULL));
+                        ++dn;
+                        res_h = h; res_sb = sb;
+                    }
+                }
+            }
+            if (*abort_flag) {
+                // drain: copies already issued must land before the CTA's shared memory is released
+                int dummy_flag = 0;
+                for (int b = 1; b <= p.q_stages; ++b) {
+                    const int qj = qn - b;
+                    if (qj >= 0) mbar_wait(bar(Q_FULL + qj % p.q_stages), (qj / p.q_stages) & 1, &dummy_flag, p.status, RW_QFULL);
+                }
+                if (dn > 0) mbar_wait(bar(D_FULL), (dn - 1) & 1, &dummy_flag, p.status, RW_DFULL);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint64_t q_desc0 = smem_desc_sw128(sQ, 16, 1024), d_desc0 = smem_desc_sw128(sD, 16, 1024);
+            int res_h = -1, res_sb = -1, qn = 0, dn = 0, nacc0 = 0, nacc1 = 0;
+            bool ok = true;
+            for (int u = u0; ok && u < u1; ++u) {
+                const int h = u / p.tiles_per_head, t = u % p.tiles_per_head;
+                const int n_sb = blocks_needed(p, t);
+                const int buf = (u - u0) & 1;
+                const int st = qn % p.q_stages;
+                for (int sb = 0; ok && sb < n_sb; ++sb) {
+                    if (sb == 0) {
+                        ok = mbar_wait(bar(Q_FULL + st), (qn / p.q_stages) & 1, abort_flag, p.status, RW_QFULL);
+                        if (!ok) break;
+                    }
+                    if (h != res_h || sb != res_sb) {
+                        ok = mbar_wait(bar(D_FULL), dn & 1, abort_flag, p.status, RW_DFULL);
+                        if (!ok) break;
+                        ++dn;
+                        res_h = h; res_sb = sb;
+                    }
+                    const int uses = buf ? nacc1 : nacc0;
+                    ok = mbar_wait(bar(ACC_EMPTY + buf), (uses & 1) ^ 1, abort_flag, p.status, RW_ACCEMPTY);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const int rows_sb = min(p.sb_rows, p.c_pad - sb * p.sb_rows);
+                    const uint64_t qd = q_desc0 + (uint64_t)(st * (Q_TILE_BYTES >> 4));
+                    for (int n0 = 0; n0 < rows_sb; n0 += 128) {
+                        const int n = min(128, rows_sb - n0);
+                        const uint32_t idesc = idesc_bf16_f32(128, n, 0, 0);
+                        const uint32_t acc = tmem + buf * ACC_COLS + n0;
+                        for (int term = 0; term < 3; ++term) {
+#pragma unroll
+                            for (int ks = 0; ks < D / 16; ++ks) {
+                                const uint32_t qo = ((ks >> 2) * Q_SUB_BYTES + (ks & 3) * 32) >> 4;
+                                const uint32_t dofs = ((term * SUB + (ks >> 2)) * d_sub_bytes + n0 * 128 + (ks & 3) * 32) >> 4;
+                                mma_ss(acc, qd + qo, d_desc0 + dofs, idesc, (term | ks) != 0);
+                            }
+                        }
+                    }
+                    tc_commit(bar(ACC_FULL + buf));
+                    if (buf) ++nacc1; else ++nacc0;
+                    // the next step, if it needs another block, may overwrite this one once these MMAs are done
+                    int nh = h, nsb = sb + 1;
+                    bool more = true;
+                    if (nsb >= n_sb) { nsb = 0; more = u + 1 < u1; nh = more ? (u + 1) / p.tiles_per_head : h; }
+                    if (more && (nh != h || nsb != sb)) tc_commit(bar(D_EMPTY));
+                }
+                if (ok) { tc_commit(bar(Q_EMPTY + st)); ++qn; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ selection groups
+        const int sg = (warp - 2) >> 2;                        // group; its units are those with (u - u0) & 1 == sg
+        const int gt = threadIdx.x - 64 - sg * 128;            // thread within the group
+        const int r = (warp & 3) * 32 + lane;                  // TMEM lane = query row of the tile
+        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t acc = tmem + sg * ACC_COLS + lane_off;
+        int *hist = hist_base + sg * p.C;
+        int nacc = 0, ngs = 0;
+        bool ok = true;
+        auto group_sync = [&]() {     // all 128 threads of the group, bounded
+            mbar_arrive(bar(GROUP + sg));
+            bool o = mbar_wait(bar(GROUP + sg), ngs & 1, abort_flag, p.status, RW_GROUP);
+            ++ngs;
+            return o;
+        };
+        for (int u = u0 + sg; ok && u < u1; u += 2) {
+            const int h = u / p.tiles_per_head, t = u % p.tiles_per_head;
+            const int n_sb = blocks_needed(p, t);
+            const int i = t * kRtRows + r;
+            const bool live = i < p.L;
+            const int ci = live ? p.tok_chunk[i] : 0;
+            TopK<KMAX> top;
+            top.init();
+            for (int x = gt; x < p.C; x += 128) hist[x] = 0;
+            for (int sb = 0; ok && sb < n_sb; ++sb) {
+                ok = mbar_wait(bar(ACC_FULL + sg), nacc & 1, abort_flag, p.status, RW_ACCFULL);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                ++nacc;
+                tc_fence_after();
+                const int rows_sb = min(p.sb_rows, p.c_pad - sb * p.sb_rows);
+                for (int cc = 0; cc < rows_sb; cc += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(acc + cc, v);
+                    tmem_wait_ld();
+                    const int j0 = sb * p.sb_rows + cc;
+                    if (live) {
+                        const uint32_t aw = p.anc_bits[(size_t)ci * p.words + (j0 >> 5)];
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            const int j = j0 + c;
+                            const bool cand = j < p.C && !((aw >> c) & 1u) && (!p.causal || j < ci);
+                            if (cand) top.push(__uint_as_float(v[c]), j, p.k);
+                        }
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(bar(ACC_EMPTY + sg));
+            }
+            if (!ok) break;
+            // sel_idx and the empty slots' partial log-sum-exp; tile-local rank of every pick
+            ok = group_sync();                      // histogram cleared
+            if (!ok) break;
+            int rank[KMAX <= 8 ? KMAX : 1];
+            int32_t *out = p.sel + ((size_t)h * p.L + i) * p.k;
+            float *pl = p.part_lse + ((size_t)h * p.L + i) * p.k;
+            if (live) {
+                if (KMAX <= 8) {
+#pragma unroll
+                    for (int x = 0; x < (KMAX <= 8 ? KMAX : 1); ++x) {
+                        if (x < p.k) {
+                            out[x] = top.j[x];
+                            if (top.j[x] >= 0) rank[x] = atomicAdd(&hist[top.j[x]], 1);
+                            else pl[x] = -INFINITY;
+                        }
+                    }
+                } else {
+                    for (int x = 0; x < p.k; ++x) {
+                        const int j = top.j[x];
+                        out[x] = j;
+                        if (j >= 0) top.s[x] = __int_as_float(atomicAdd(&hist[j], 1));   // the score is no longer needed
+                        else pl[x] = -INFINITY;
+                    }
+                }
+            }
+            ok = group_sync();                      // ranks taken
+            if (!ok) break;
+            for (int x = gt; x < p.C; x += 128) {   // reserve this tile's range in each picked chunk's list
+                const int n = hist[x];
+                if (n) hist[x] = atomicAdd(&p.cnt[h * p.C + x], n);
+            }
+            ok = group_sync();                      // bases known
+            if (!ok) break;
+            if (live) {
+                int32_t *list = p.qlist + (size_t)h * p.cap_total;
+                if (KMAX <= 8) {
+#pragma unroll
+                    for (int x = 0; x < (KMAX <= 8 ? KMAX : 1); ++x)
+                        if (x < p.k && top.j[x] >= 0) list[p.cap_off[top.j[x]] + hist[top.j[x]] + rank[x]] = i * p.k + x;
+                } else {
+                    for (int x = 0; x < p.k; ++x) {
+                        const int j = top.j[x];
+                        if (j >= 0) list[p.cap_off[j] + hist[j] + __float_as_int(top.s[x])] = i * p.k + x;
+                    }
+                }
+            }
+            ok = group_sync();                      // lists written before the histogram is cleared again
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+// gtile[i] = attention tiles (of kQTileRows picks) before (head, chunk) pair i, with a final total;
+// flags the workspace as routed.
+__global__ void __launch_bounds__(1024) route_tiles_kernel(const int *__restrict__ cnt, int *__restrict__ gtile,
+                                                           int *__restrict__ status, int HC) {
+    __shared__ int st[1024];
+    const int t = threadIdx.x;
     const int per = (HC + 1023) / 1024;
     const int i0 = min(t * per, HC), i1 = min(i0 + per, HC);
-    int a = 0, b = 0;
-    for (int i = i0; i < i1; ++i) { a += cnt[i]; b += (cnt[i] + kQTileRows - 1) / kQTileRows; }
-    sc[t] = a; st[t] = b;
+    int b = 0;
+    for (int i = i0; i < i1; ++i) b += (cnt[i] + kQTileRows - 1) / kQTileRows;
+    st[t] = b;
     __syncthreads();
     for (int o = 1; o < 1024; o <<= 1) {   // inclusive scan
-        int xa = 0, xb = 0;
-        if (t >= o) { xa = sc[t - o]; xb = st[t - o]; }
+        int xb = 0;
+        if (t >= o) xb = st[t - o];
         __syncthreads();
-        sc[t] += xa; st[t] += xb;
+        st[t] += xb;
         __syncthreads();
     }
-    int ea = sc[t] - a, eb = st[t] - b;    // exclusive
+    int eb = st[t] - b;    // exclusive
     for (int i = i0; i < i1; ++i) {
-        gcnt[i] = ea; gtile[i] = eb; cursor[i] = 0;
-        ea += cnt[i]; eb += (cnt[i] + kQTileRows - 1) / kQTileRows;
+        gtile[i] = eb;
+        eb += (cnt[i] + kQTileRows - 1) / kQTileRows;
     }
-    if (t == 1023) { gcnt[HC] = sc[1023]; gtile[HC] = st[1023]; status[2] = 1; }
-    __syncthreads();
-    for (int idx = t; idx < H * (C + 1); idx += 1024) {
-        const int h = idx / (C + 1), c = idx % (C + 1);
-        qoff[idx] = gcnt[h * C + c] - gcnt[h * C];
-    }
-}
-
-__global__ void route_scatter_kernel(const int32_t *__restrict__ sel, const int *__restrict__ qoff,
-                                     int *__restrict__ cursor, int32_t *__restrict__ qlist, int L, int C, int k) {
-    const int h = blockIdx.y;
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= L) return;
-    const int32_t *row = sel + ((size_t)h * L + i) * k;
-    int32_t *list = qlist + (size_t)h * L * k;
-    for (int s = 0; s < k; ++s) {
-        const int j = row[s];
-        if (j < 0) continue;
-        const int pos = atomicAdd(&cursor[h * C + j], 1);
-        list[qoff[h * (C + 1) + j] + pos] = i * k + s;
-    }
-}
-
-__global__ void zero_i32_kernel2(int *p, size_t n) {
-    size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
-    if (i < n) p[i] = 0;
+    if (t == 1023) { gtile[HC] = st[1023]; status[2] = 1; }
 }
 
 template <int D>
@@ -205,20 +401,36 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
                           cudaStream_t s) {
     int *cnt = ws_ptr<int>(ws, p->ws.cnt);
     int *status = ws_ptr<int>(ws, p->ws.status);
-    const size_t n = (size_t)p->H * p->C;
-    zero_i32_kernel2<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(cnt, n);
-    MOC_LAUNCH_CHECK();
-    zero_i32_kernel2<<<1, kStatusWords, 0, s>>>(status, kStatusWords);
-    MOC_LAUNCH_CHECK();
+    __nv_bfloat16 *desc3 = ws_ptr<__nv_bfloat16>(ws, p->ws.desc3);
+    {
+        const size_t n = std::max((size_t)p->H * p->c_pad * D, (size_t)kStatusWords);   // covers H * C too
+        route_prep_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(desc, desc3, cnt, status, p->H, p->C, p->c_pad, D);
+        MOC_LAUNCH_CHECK();
+    }
     if (p->k > 0) {
-        const size_t smem = sizeof(__nv_bfloat16) * kRouteRows * (D + 8) + sizeof(float) * kRouteCB * D + sizeof(int) * p->C;
-        dim3 grid((unsigned)((p->L + kRouteRows - 1) / kRouteRows), (unsigned)p->H);
-        const int causal = (p->flags & MOC_FLAG_CAUSAL) ? 1 : 0;
-#define MOC_ROUTE_CASE(KM)                                                                                          \
-    do {                                                                                                            \
-        MOC_CUDA_TRY(cudaFuncSetAttribute(route_kernel<D, KM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        route_kernel<D, KM><<<grid, kRouteRows, smem, s>>>(Q, desc, sel, cnt, ws_ptr<float>(ws, p->ws.part_lse), p->d_tok_chunk, p->d_anc_bits, p->words, \
-                                                           p->L, p->C, p->k, causal);                               \
+        RouteParams a;
+        a.sel = sel; a.part_lse = ws_ptr<float>(ws, p->ws.part_lse); a.cnt = cnt;
+        a.qlist = ws_ptr<int32_t>(ws, p->ws.qlist);
+        a.tok_chunk = p->d_tok_chunk; a.anc_bits = p->d_anc_bits; a.cap_off = p->d_cap_off; a.status = status;
+        a.H = p->H; a.L = p->L; a.C = p->C; a.c_pad = p->c_pad; a.k = p->k; a.words = p->words;
+        a.causal = (p->flags & MOC_FLAG_CAUSAL) ? 1 : 0;
+        a.tiles_per_head = (p->L + kRtRows - 1) / kRtRows;
+        a.sb_rows = p->c_pad <= kRtResident ? p->c_pad : kRtBlock;
+        a.cap_total = (size_t)p->cap_off[p->C];
+        const size_t q_tile = (size_t)kRtRows * D * 2, d_block = ((size_t)3 * a.sb_rows * D * 2 + 1023) & ~(size_t)1023;
+        const size_t hist = 2 * sizeof(int) * (size_t)p->C, budget = 227 * 1024 - 1024;
+        if (d_block + q_tile + hist > budget) return MOC_ERR_SHAPE;
+        a.q_stages = (int)std::min<size_t>(4, (budget - d_block - hist) / q_tile);
+        const size_t smem = 1024 + d_block + a.q_stages * q_tile + hist;
+        CUtensorMap tmQ, tmD;
+        if (int r = make_tmap_2d_bf16(&tmQ, Q, (uint64_t)p->H * p->L, D, kRtRows)) return r;
+        if (int r = make_tmap_2d_bf16(&tmD, desc3, (uint64_t)p->H * 3 * p->c_pad, D, (uint32_t)a.sb_rows)) return r;
+        const long long units = (long long)p->H * a.tiles_per_head;
+        const unsigned grid = (unsigned)std::min<long long>(p->n_sm, units);
+#define MOC_ROUTE_CASE(KM)                                                                                              \
+    do {                                                                                                                \
+        MOC_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel<D, KM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        route_tc_kernel<D, KM><<<grid, kRtThreads, smem, s>>>(tmQ, tmD, a);                                             \
     } while (0)
         if (p->k <= 8) MOC_ROUTE_CASE(8);
         else if (p->k <= 64) MOC_ROUTE_CASE(64);
@@ -226,15 +438,8 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
 #undef MOC_ROUTE_CASE
         MOC_LAUNCH_CHECK();
     }
-    route_scan_kernel<<<1, 1024, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.gcnt), ws_ptr<int>(ws, p->ws.tile_off),
-                                         ws_ptr<int>(ws, p->ws.qoff), ws_ptr<int>(ws, p->ws.cursor), status, p->H, p->C);
+    route_tiles_kernel<<<1, 1024, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off), status, p->H * p->C);
     MOC_LAUNCH_CHECK();
-    if (p->k > 0) {
-        dim3 grid((unsigned)((p->L + 255) / 256), (unsigned)p->H);
-        route_scatter_kernel<<<grid, 256, 0, s>>>(sel, ws_ptr<int>(ws, p->ws.qoff), ws_ptr<int>(ws, p->ws.cursor),
-                                                  ws_ptr<int32_t>(ws, p->ws.qlist), p->L, p->C, p->k);
-        MOC_LAUNCH_CHECK();
-    }
     return MOC_OK;
 }
 
