@@ -9,17 +9,18 @@
 // accumulated in fp32 in TMEM: every product is exact, only the fp32 accumulation rounds.
 //
 // route_prep_kernel   splits the descriptors, clears the pick counters and the status words.
-// route_tc_kernel     persistent, one CTA per SM, each owning a contiguous range of
-//                     (head, 128-query tile) units:
+// route_tc_kernel     H x (SMs / H) CTAs, each owning a contiguous range of 128-query tiles
+//                     ("units") of one head:
 //     warp 0      TMA producer: Q tiles (ring of stages) and the head's descriptor block;
-//     warp 1      MMA issuer: 3 x d/16 MMAs per 128 chunks into one of two TMEM accumulators;
+//     warps 1, 10 MMA issuers: 3 x d/16 MMAs per 128 chunks into one of two TMEM accumulators
+//                 (warp 1 the even units, warp 10 the odd ones);
 //     warps 2-5 / 6-9   two selection groups (even / odd units), one query per thread (TMEM
 //                 lane = query): read the scores 32 chunks at a time, drop non-candidates,
 //                 keep a sorted top-k in registers, then write sel_idx and append the picks
 //                 to the per-(head, chunk) query lists (tile-local ranks from a shared-memory
 //                 histogram, one global atomic per (tile, chunk) to reserve the range).
-//   The descriptor block of a head stays in shared memory while the CTA's units stay in that
-//   head (C <= 192); with more chunks it is streamed in blocks of 128.
+//   The head's descriptor block stays in shared memory for the CTA's lifetime (C <= 192);
+//   with more chunks it is streamed in blocks of 128 and warp 1 alone issues.
 // route_tiles_kernel  running count of attention tiles over (head, chunk) from the pick counts.
 // Every mbarrier wait is bounded; a wait that runs out flags the workspace status word.
 #include <float.h>
@@ -33,11 +34,29 @@ namespace moc {
 using namespace tc;
 
 constexpr int kRtRows = 128;          // queries per tile
-constexpr int kRtThreads = 320;
+constexpr int kRtThreads = 384;
 constexpr int kRtResident = 192;      // up to this many (padded) chunks the whole block stays resident
 constexpr int kRtBlock = 128;         // otherwise chunks are streamed in blocks of this many
 
+// Optional cycle stamps of one CTA (build with -DMOC_TRACE), read back with moc_trace_read_route().
+// slot 0 start; selection group sg, n-th unit of the group: 100 + 1000 sg + 16 n + {0 unit begins,
+// 1 scores ready, 2 selection done, 3 previous unit's lists written, 4 ranks taken, 5 ranges reserved,
+// 6 scores loaded, 8 + r selection round r done};
+// issuer: 3000 + 4 n + {0 inputs ready, 1 accumulator free, 2 MMAs issued, 3 unit begins}
+#ifdef MOC_TRACE
+__device__ long long g_trace_route[8192];
+#define RTRACE(slot) do { if (blockIdx.x == 70 && (slot) < 8192) g_trace_route[(slot)] = clock64(); } while (0)
+#else
+#define RTRACE(slot) ((void)0)
+#endif
+
 enum RouteWait { RW_QFULL = 32, RW_QEMPTY, RW_DFULL, RW_DEMPTY, RW_ACCFULL, RW_ACCEMPTY, RW_GROUP };
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 
 template <int KMAX>
 struct TopK {
@@ -103,6 +122,7 @@ struct RouteParams {
     int *status;
     int H, L, C, c_pad, k, words, causal;
     int tiles_per_head;     // ceil(L / 128)
+    int ctas_per_head;      // the grid is H * ctas_per_head
     int sb_rows;            // chunks per descriptor block held in shared memory
     int q_stages;
     size_t cap_total;
@@ -112,7 +132,7 @@ struct RouteParams {
 __device__ __forceinline__ int blocks_needed(const RouteParams &p, int t) {
     int c_hi = p.C;
     if (p.causal) c_hi = p.tok_chunk[min(p.L, (t + 1) * kRtRows) - 1];   // picks are strictly earlier chunks
-    return max(1, (c_hi + p.sb_rows - 1) / p.sb_rows);
+    return max(1, (c_hi + p.sb_rows - 1) / p.sb_rows);   // <= 64: C <= 8192, streamed blocks of 128
 }
 
 template <int D, int KMAX>
@@ -135,6 +155,8 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
     const uint32_t sD = sbase;
     const uint32_t sQ = sD + ((3 * SUB * d_sub_bytes + 1023) & ~1023);
     int *hist_base = reinterpret_cast<int *>(gbase + (sQ - sbase) + p.q_stages * Q_TILE_BYTES);
+    int *s_cap = hist_base + 2 * p.C;                                   // copy of cap_off[0 .. C)
+    uint8_t *s_nsb = reinterpret_cast<uint8_t *>(s_cap + p.C);          // descriptor blocks needed by each of this CTA's units
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     constexpr int Q_FULL = 0, Q_EMPTY = kMaxStages, D_FULL = 2 * kMaxStages, D_EMPTY = D_FULL + 1, ACC_FULL = D_FULL + 2,
                   ACC_EMPTY = D_FULL + 4, GROUP = D_FULL + 6;
@@ -161,22 +183,28 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
     volatile int *abort_flag = &s_abort;
+    if (threadIdx.x == 0) RTRACE(0);
 
-    // this CTA's units: a contiguous range of (head, tile), so the descriptor block changes rarely
-    const long long U = (long long)p.H * p.tiles_per_head;
-    const int u0 = (int)(U * blockIdx.x / gridDim.x), u1 = (int)(U * (blockIdx.x + 1) / gridDim.x);
+    // this CTA's units: a contiguous range of 128-query tiles of ONE head (u counts tiles of that head),
+    // so its descriptor block never changes while it fits in shared memory
+    const int h = blockIdx.x / p.ctas_per_head, part = blockIdx.x % p.ctas_per_head;
+    const int u0 = (int)((long long)p.tiles_per_head * part / p.ctas_per_head);
+    const int u1 = (int)((long long)p.tiles_per_head * (part + 1) / p.ctas_per_head);
+    for (int x = threadIdx.x; x < p.C; x += kRtThreads) s_cap[x] = p.cap_off[x];
+    for (int x = threadIdx.x; x < u1 - u0; x += kRtThreads) s_nsb[x] = (uint8_t)blocks_needed(p, u0 + x);
+    __syncthreads();
     constexpr int ACC_COLS = 256;   // TMEM columns per accumulator (sb_rows <= 192)
+    const bool resident = p.sb_rows == p.c_pad;      // one block holds every chunk: loaded once, two MMA issuers
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             prefetch_tensormap(&tmQ);
             prefetch_tensormap(&tmD);
-            int res_h = -1, res_sb = -1, qn = 0, dn = 0;
+            int res_sb = -1, qn = 0, dn = 0;
             bool ok = true;
             for (int u = u0; ok && u < u1; ++u) {
-                const int h = u / p.tiles_per_head, t = u % p.tiles_per_head;
-                const int n_sb = blocks_needed(p, t);
+                const int n_sb = s_nsb[u - u0];
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
                     if (sb == 0) {
                         const int st = qn % p.q_stages;
@@ -185,10 +213,10 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
                         mbar_expect_tx(bar(Q_FULL + st), Q_TILE_BYTES);
 #pragma unroll
                         for (int sub = 0; sub < SUB; ++sub)
-                            tma_load_2d(sQ + st * Q_TILE_BYTES + sub * Q_SUB_BYTES, &tmQ, sub * 64, h * p.L + t * kRtRows, bar(Q_FULL + st));
+                            tma_load_2d(sQ + st * Q_TILE_BYTES + sub * Q_SUB_BYTES, &tmQ, sub * 64, h * p.L + u * kRtRows, bar(Q_FULL + st));
                         ++qn;
                     }
-                    if (h != res_h || sb != res_sb) {
+                    if (sb != res_sb) {
                         ok = mbar_wait(bar(D_EMPTY), (dn & 1) ^ 1, abort_flag, p.status, RW_DEMPTY);
                         if (!ok) break;
                         mbar_expect_tx(bar(D_FULL), 3 * SUB * d_sub_bytes);
@@ -198,7 +226,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
                                 tma_load_2d(sD + (term * SUB + sub) * d_sub_bytes, &tmD, sub * 64,
                                             (h * 3 + term) * p.c_pad + sb * p.sb_rows, bar(D_FULL));
                         ++dn;
-                        res_h = h; res_sb = sb;
+                        res_sb = sb;
                     }
                 }
             }
@@ -212,61 +240,75 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
                 if (dn > 0) mbar_wait(bar(D_FULL), (dn - 1) & 1, &dummy_flag, p.status, RW_DFULL);
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint64_t q_desc0 = smem_desc_sw128(sQ, 16, 1024), d_desc0 = smem_desc_sw128(sD, 16, 1024);
-            int res_h = -1, res_sb = -1, qn = 0, dn = 0, nacc0 = 0, nacc1 = 0;
+    } else if (warp == 1 || warp == 10) {
+        // ------------------------------------------------------------ MMA issuers
+        // With a resident descriptor block, warp 1 serves the even units and warp 10 the odd ones (each
+        // its own accumulator), so one issuer's waits and instruction overhead hide behind the other's
+        // MMAs; when blocks are streamed, warp 1 serves every unit and follows the reloads.
+        const int first = warp == 1 ? 0 : 1, stride = resident ? 2 : 1;
+        if (lane == 0 && (warp == 1 || resident)) {
+            // descriptors are built once: issuing an MMA should cost this thread a few integer instructions
+            const uint64_t q_desc0 = smem_desc_sw128(sQ, 16, 1024);
+            uint64_t d_term[3 * SUB];
+#pragma unroll
+            for (int x = 0; x < 3 * SUB; ++x) d_term[x] = smem_desc_sw128(sD + x * d_sub_bytes, 16, 1024);
+            int res_sb = -1, dn = 0, nacc0 = 0, nacc1 = 0;
             bool ok = true;
-            for (int u = u0; ok && u < u1; ++u) {
-                const int h = u / p.tiles_per_head, t = u % p.tiles_per_head;
-                const int n_sb = blocks_needed(p, t);
+            for (int u = u0 + first; ok && u < u1; u += stride) {
+                const int n_sb = s_nsb[u - u0];
                 const int buf = (u - u0) & 1;
-                const int st = qn % p.q_stages;
+                const int qn = u - u0, st = qn % p.q_stages;
+                RTRACE(3000 + (u - u0) * 4 + 3);
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
                     if (sb == 0) {
                         ok = mbar_wait(bar(Q_FULL + st), (qn / p.q_stages) & 1, abort_flag, p.status, RW_QFULL);
                         if (!ok) break;
                     }
-                    if (h != res_h || sb != res_sb) {
+                    if (sb != res_sb) {
                         ok = mbar_wait(bar(D_FULL), dn & 1, abort_flag, p.status, RW_DFULL);
                         if (!ok) break;
                         ++dn;
-                        res_h = h; res_sb = sb;
+                        res_sb = sb;
                     }
+                    RTRACE(3000 + (u - u0) * 4 + 0);
                     const int uses = buf ? nacc1 : nacc0;
                     ok = mbar_wait(bar(ACC_EMPTY + buf), (uses & 1) ^ 1, abort_flag, p.status, RW_ACCEMPTY);
                     if (!ok) break;
                     tc_fence_after();
+                    RTRACE(3000 + (u - u0) * 4 + 1);
                     const int rows_sb = min(p.sb_rows, p.c_pad - sb * p.sb_rows);
                     const uint64_t qd = q_desc0 + (uint64_t)(st * (Q_TILE_BYTES >> 4));
                     for (int n0 = 0; n0 < rows_sb; n0 += 128) {
                         const int n = min(128, rows_sb - n0);
                         const uint32_t idesc = idesc_bf16_f32(128, n, 0, 0);
                         const uint32_t acc = tmem + buf * ACC_COLS + n0;
+                        const uint32_t nofs = (uint32_t)(n0 * 128) >> 4;
+#pragma unroll
                         for (int term = 0; term < 3; ++term) {
 #pragma unroll
-                            for (int ks = 0; ks < D / 16; ++ks) {
-                                const uint32_t qo = ((ks >> 2) * Q_SUB_BYTES + (ks & 3) * 32) >> 4;
-                                const uint32_t dofs = ((term * SUB + (ks >> 2)) * d_sub_bytes + n0 * 128 + (ks & 3) * 32) >> 4;
-                                mma_ss(acc, qd + qo, d_desc0 + dofs, idesc, (term | ks) != 0);
-                            }
+                            for (int ks = 0; ks < D / 16; ++ks)
+                                mma_ss(acc, qd + (((ks >> 2) * Q_SUB_BYTES + (ks & 3) * 32) >> 4),
+                                       d_term[term * SUB + (ks >> 2)] + nofs + (((ks & 3) * 32) >> 4), idesc, (term | ks) != 0);
                         }
                     }
                     tc_commit(bar(ACC_FULL + buf));
+                    RTRACE(3000 + (u - u0) * 4 + 2);
                     if (buf) ++nacc1; else ++nacc0;
-                    // the next step, if it needs another block, may overwrite this one once these MMAs are done
-                    int nh = h, nsb = sb + 1;
-                    bool more = true;
-                    if (nsb >= n_sb) { nsb = 0; more = u + 1 < u1; nh = more ? (u + 1) / p.tiles_per_head : h; }
-                    if (more && (nh != h || nsb != sb)) tc_commit(bar(D_EMPTY));
+                    // streamed blocks: the next step, if it needs another block, may overwrite this one once
+                    // these MMAs are done
+                    if (!resident) {
+                        int nsb = sb + 1;
+                        bool more = true;
+                        if (nsb >= n_sb) { nsb = 0; more = u + 1 < u1; }
+                        if (more && nsb != sb) tc_commit(bar(D_EMPTY));
+                    }
                 }
-                if (ok) { tc_commit(bar(Q_EMPTY + st)); ++qn; }
+                if (ok) tc_commit(bar(Q_EMPTY + st));
             }
         }
-    } else {
+    } else if (warp < 10) {
         // ------------------------------------------------------------ selection groups
-        const int sg = (warp - 2) >> 2;                        // group; its units are those with (u - u0) & 1 == sg
+        const int sg = (warp - 2) >> 2;                        // group (warps 2-5, 6-9); its units are those with (u - u0) & 1 == sg
         const int gt = threadIdx.x - 64 - sg * 128;            // thread within the group
         const int r = (warp & 3) * 32 + lane;                  // TMEM lane = query row of the tile
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
@@ -280,89 +322,200 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
             ++ngs;
             return o;
         };
+        constexpr bool SMALL = KMAX <= 8;
+        constexpr int KR = SMALL ? KMAX : 1;
+        // With few chunks the list append of a unit is finished after the next unit's selection, so the
+        // round trip of the range-reserving atomics is hidden; `pend` is the unit whose append is open.
+        const bool deferred = SMALL && p.C <= 256;
+        struct Pending { int h, i, j[KR], rank[KR], base0, base1; bool live, open; } pend;
+        pend.open = false; pend.live = false; pend.h = 0; pend.i = 0; pend.base0 = 0; pend.base1 = 0;
+        auto finish_pending = [&]() {          // bases into the histogram, then the list entries
+            if (gt < p.C) hist[gt] = pend.base0;
+            if (gt + 128 < p.C) hist[gt + 128] = pend.base1;
+            bool o = group_sync();
+            if (o && pend.live) {
+                int32_t *list = p.qlist + (size_t)pend.h * p.cap_total;
+#pragma unroll
+                for (int x = 0; x < KR; ++x)
+                    if (x < p.k && pend.j[x] >= 0) list[s_cap[pend.j[x]] + hist[pend.j[x]] + pend.rank[x]] = pend.i * p.k + x;
+            }
+            o = o && group_sync();             // entries written before the histogram is reused
+            pend.open = false;
+            return o;
+        };
+        int nx_ci = 0;
+        uint32_t nx_aw = 0u;
+        if (u0 + sg < u1) {
+            const int i0 = (u0 + sg) * kRtRows + r;
+            nx_ci = i0 < p.L ? p.tok_chunk[i0] : 0;
+            nx_aw = i0 < p.L ? p.anc_bits[(size_t)nx_ci * p.words] : 0u;
+        }
         for (int u = u0 + sg; ok && u < u1; u += 2) {
-            const int h = u / p.tiles_per_head, t = u % p.tiles_per_head;
-            const int n_sb = blocks_needed(p, t);
-            const int i = t * kRtRows + r;
+            const int n_sb = s_nsb[u - u0];
+            const int i = u * kRtRows + r;
             const bool live = i < p.L;
-            const int ci = live ? p.tok_chunk[i] : 0;
+            const int ci = nx_ci;
+            const uint32_t aw_next = nx_aw;
+            const int i2 = (u + 2) * kRtRows + r;
+            const bool live2 = u + 2 < u1 && i2 < p.L;
+            if (live2) nx_ci = p.tok_chunk[i2];       // the next unit's chunk, loaded a unit ahead (its anchor word follows below)
+            [[maybe_unused]] const int tn = 100 + sg * 1000 + ((u - u0) >> 1) * 16;
+            if (gt == 0) RTRACE(tn + 0);
             TopK<KMAX> top;
             top.init();
-            for (int x = gt; x < p.C; x += 128) hist[x] = 0;
+            [[maybe_unused]] float kth = -INFINITY;
             for (int sb = 0; ok && sb < n_sb; ++sb) {
                 ok = mbar_wait(bar(ACC_FULL + sg), nacc & 1, abort_flag, p.status, RW_ACCFULL);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ++nacc;
+                if (gt == 0) RTRACE(tn + 1);
                 tc_fence_after();
                 const int rows_sb = min(p.sb_rows, p.c_pad - sb * p.sb_rows);
                 for (int cc = 0; cc < rows_sb; cc += 32) {
                     uint32_t v[32];
                     tmem_ld32(acc + cc, v);
-                    tmem_wait_ld();
                     const int j0 = sb * p.sb_rows + cc;
-                    if (live) {
-                        const uint32_t aw = p.anc_bits[(size_t)ci * p.words + (j0 >> 5)];
+                    const uint32_t aw = (sb == 0 && cc == 0) ? aw_next : (live ? p.anc_bits[(size_t)ci * p.words + (j0 >> 5)] : 0u);
+                    // candidate bits of this block: a real chunk, not an anchor, strictly earlier if causal
+                    uint32_t cand = ~aw;
+                    const int lim = min(p.C, p.causal ? ci : p.C) - j0;     // chunks j0 .. j0 + lim - 1 may be picked
+                    cand = lim <= 0 ? 0u : (lim >= 32 ? cand : (cand & ((1u << lim) - 1u)));
+                    if (!live) cand = 0u;
+                    tmem_wait_ld();
+                    if (gt == 0) RTRACE(tn + 6);
+                    if (SMALL) {
+                        float f[32];
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            const int j = j0 + c;
-                            const bool cand = j < p.C && !((aw >> c) & 1u) && (!p.causal || j < ci);
-                            if (cand) top.push(__uint_as_float(v[c]), j, p.k);
+                        for (int c = 0; c < 32; ++c) f[c] = ((cand >> c) & 1u) ? __uint_as_float(v[c]) : -INFINITY;
+                        // up to k members of the block can enter the list: take them best first
+#pragma unroll 1
+                        for (int round = 0; round < p.k; ++round) {
+                            float m8[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float a = max3(f[q * 8], f[q * 8 + 1], f[q * 8 + 2]);
+                                const float b = max3(f[q * 8 + 3], f[q * 8 + 4], f[q * 8 + 5]);
+                                m8[q] = max3(a, b, fmaxf(f[q * 8 + 6], f[q * 8 + 7]));
+                            }
+                            const float m = fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3]));
+                            const float thr = kth;                                              // the list's k-th score
+                            const bool want = m > thr;
+                            if (!__any_sync(0xffffffffu, want)) break;
+                            uint32_t eq = 0u;                                                   // lowest index among equals
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) eq |= (f[c] == m) ? (1u << c) : 0u;
+                            const int idx = __ffs(eq) - 1;
+                            if (want) {
+                                // the displaced element sinks through the sorted list (strict '>' keeps equal
+                                // scores in arrival order, which is ascending chunk index)
+                                float cv = m;
+                                int cj = j0 + idx;
+#pragma unroll
+                                for (int x = 0; x < KR; ++x) {
+                                    const bool up = cv > top.s[x];
+                                    const float ts = top.s[x];
+                                    const int tj = top.j[x];
+                                    top.s[x] = up ? cv : ts;
+                                    top.j[x] = up ? cj : tj;
+                                    cv = up ? ts : cv;
+                                    cj = up ? tj : cj;
+                                }
+                                kth = top.s[0];
+#pragma unroll
+                                for (int x = 1; x < KR; ++x) kth = (x < p.k) ? top.s[x] : kth;
+                            }
+                            const uint32_t clr = want ? (1u << idx) : 0u;
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) f[c] = ((clr >> c) & 1u) ? -INFINITY : f[c];
+                            if (gt == 0) RTRACE(tn + 8 + round);
                         }
+                    } else {
+                        for (int c = 0; c < 32; ++c)
+                            if ((cand >> c) & 1u) top.push(__uint_as_float(v[c]), j0 + c, p.k);
                     }
                 }
                 tc_fence_before();
                 mbar_arrive(bar(ACC_EMPTY + sg));
             }
             if (!ok) break;
-            // sel_idx and the empty slots' partial log-sum-exp; tile-local rank of every pick
-            ok = group_sync();                      // histogram cleared
-            if (!ok) break;
-            int rank[KMAX <= 8 ? KMAX : 1];
+            nx_aw = live2 ? p.anc_bits[(size_t)nx_ci * p.words] : 0u;
+            if (gt == 0) RTRACE(tn + 2);
+            // sel_idx and the empty slots' partial log-sum-exp
             int32_t *out = p.sel + ((size_t)h * p.L + i) * p.k;
             float *pl = p.part_lse + ((size_t)h * p.L + i) * p.k;
             if (live) {
-                if (KMAX <= 8) {
+                if (SMALL) {
 #pragma unroll
-                    for (int x = 0; x < (KMAX <= 8 ? KMAX : 1); ++x) {
+                    for (int x = 0; x < KR; ++x)
                         if (x < p.k) {
                             out[x] = top.j[x];
-                            if (top.j[x] >= 0) rank[x] = atomicAdd(&hist[top.j[x]], 1);
-                            else pl[x] = -INFINITY;
+                            if (top.j[x] < 0) pl[x] = -INFINITY;
                         }
-                    }
                 } else {
                     for (int x = 0; x < p.k; ++x) {
-                        const int j = top.j[x];
-                        out[x] = j;
-                        if (j >= 0) top.s[x] = __int_as_float(atomicAdd(&hist[j], 1));   // the score is no longer needed
-                        else pl[x] = -INFINITY;
+                        out[x] = top.j[x];
+                        if (top.j[x] < 0) pl[x] = -INFINITY;
                     }
                 }
             }
-            ok = group_sync();                      // ranks taken
-            if (!ok) break;
-            for (int x = gt; x < p.C; x += 128) {   // reserve this tile's range in each picked chunk's list
-                const int n = hist[x];
-                if (n) hist[x] = atomicAdd(&p.cnt[h * p.C + x], n);
-            }
-            ok = group_sync();                      // bases known
+            if (pend.open) { ok = finish_pending(); if (!ok) break; }
+            if (gt == 0) RTRACE(tn + 3);
+            // tile-local rank of every pick (shared-memory histogram), then one global atomic per picked
+            // chunk reserves this tile's range in that chunk's list
+            for (int x = gt; x < p.C; x += 128) hist[x] = 0;
+            ok = group_sync();
             if (!ok) break;
             if (live) {
-                int32_t *list = p.qlist + (size_t)h * p.cap_total;
-                if (KMAX <= 8) {
+                if (SMALL) {
 #pragma unroll
-                    for (int x = 0; x < (KMAX <= 8 ? KMAX : 1); ++x)
-                        if (x < p.k && top.j[x] >= 0) list[p.cap_off[top.j[x]] + hist[top.j[x]] + rank[x]] = i * p.k + x;
+                    for (int x = 0; x < KR; ++x) {
+                        pend.j[x] = x < p.k ? top.j[x] : -1;
+                        pend.rank[x] = 0;
+                        if (pend.j[x] >= 0) pend.rank[x] = atomicAdd(&hist[pend.j[x]], 1);
+                    }
                 } else {
-                    for (int x = 0; x < p.k; ++x) {
-                        const int j = top.j[x];
-                        if (j >= 0) list[p.cap_off[j] + hist[j] + __float_as_int(top.s[x])] = i * p.k + x;
+                    for (int x = 0; x < p.k; ++x)
+                        if (top.j[x] >= 0) top.s[x] = __int_as_float(atomicAdd(&hist[top.j[x]], 1));   // the score is no longer needed
+                }
+            } else if (SMALL) {
+#pragma unroll
+                for (int x = 0; x < KR; ++x) { pend.j[x] = -1; pend.rank[x] = 0; }
+            }
+            ok = group_sync();
+            if (!ok) break;
+            if (gt == 0) RTRACE(tn + 4);
+            if (deferred) {
+                pend.base0 = 0; pend.base1 = 0;
+                if (gt < p.C && hist[gt]) pend.base0 = atomicAdd(&p.cnt[h * p.C + gt], hist[gt]);
+                if (gt + 128 < p.C && hist[gt + 128]) pend.base1 = atomicAdd(&p.cnt[h * p.C + gt + 128], hist[gt + 128]);
+                pend.h = h; pend.i = i; pend.live = live; pend.open = true;   // each thread re-reads only its own counts
+            } else {
+                for (int x = gt; x < p.C; x += 128) {
+                    const int n = hist[x];
+                    if (n) hist[x] = atomicAdd(&p.cnt[h * p.C + x], n);
+                }
+                ok = group_sync();
+                if (!ok) break;
+                if (live) {
+                    int32_t *list = p.qlist + (size_t)h * p.cap_total;
+                    if (SMALL) {
+#pragma unroll
+                        for (int x = 0; x < KR; ++x)
+                            if (pend.j[x] >= 0) list[s_cap[pend.j[x]] + hist[pend.j[x]] + pend.rank[x]] = i * p.k + x;
+                    } else {
+                        for (int x = 0; x < p.k; ++x) {
+                            const int j = top.j[x];
+                            if (j >= 0) list[s_cap[j] + hist[j] + __float_as_int(top.s[x])] = i * p.k + x;
+                        }
                     }
                 }
+                ok = group_sync();
+                if (!ok) break;
             }
-            ok = group_sync();                      // lists written before the histogram is cleared again
+            if (gt == 0) RTRACE(tn + 5);
         }
+        if (ok && pend.open) finish_pending();
     }
     tc_fence_before();
     __syncthreads();
@@ -396,6 +549,12 @@ __global__ void __launch_bounds__(1024) route_tiles_kernel(const int *__restrict
     if (t == 1023) { gtile[HC] = st[1023]; status[2] = 1; }
 }
 
+#ifdef MOC_TRACE
+extern "C" int moc_trace_read_route(long long *host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_trace_route, sizeof(long long) * (size_t)n);
+}
+#endif
+
 template <int D>
 static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float *desc, int32_t *sel, void *ws,
                           cudaStream_t s) {
@@ -418,21 +577,23 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         a.sb_rows = p->c_pad <= kRtResident ? p->c_pad : kRtBlock;
         a.cap_total = (size_t)p->cap_off[p->C];
         const size_t q_tile = (size_t)kRtRows * D * 2, d_block = ((size_t)3 * a.sb_rows * D * 2 + 1023) & ~(size_t)1023;
-        const size_t hist = 2 * sizeof(int) * (size_t)p->C, budget = 227 * 1024 - 1024;
+        a.ctas_per_head = std::max(1, std::min(p->n_sm / p->H, a.tiles_per_head));
+        const unsigned grid = (unsigned)(p->H * a.ctas_per_head);
+        // two histograms, the list offsets, and one byte per unit of a CTA
+        const size_t hist = 3 * sizeof(int) * (size_t)p->C + (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
         if (d_block + q_tile + hist > budget) return MOC_ERR_SHAPE;
         a.q_stages = (int)std::min<size_t>(4, (budget - d_block - hist) / q_tile);
         const size_t smem = 1024 + d_block + a.q_stages * q_tile + hist;
         CUtensorMap tmQ, tmD;
         if (int r = make_tmap_2d_bf16(&tmQ, Q, (uint64_t)p->H * p->L, D, kRtRows)) return r;
         if (int r = make_tmap_2d_bf16(&tmD, desc3, (uint64_t)p->H * 3 * p->c_pad, D, (uint32_t)a.sb_rows)) return r;
-        const long long units = (long long)p->H * a.tiles_per_head;
-        const unsigned grid = (unsigned)std::min<long long>(p->n_sm, units);
 #define MOC_ROUTE_CASE(KM)                                                                                              \
     do {                                                                                                                \
         MOC_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel<D, KM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
         route_tc_kernel<D, KM><<<grid, kRtThreads, smem, s>>>(tmQ, tmD, a);                                             \
     } while (0)
-        if (p->k <= 8) MOC_ROUTE_CASE(8);
+        if (p->k <= 4) MOC_ROUTE_CASE(4);
+        else if (p->k <= 8) MOC_ROUTE_CASE(8);
         else if (p->k <= 64) MOC_ROUTE_CASE(64);
         else MOC_ROUTE_CASE(512);
 #undef MOC_ROUTE_CASE
