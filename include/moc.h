@@ -101,9 +101,10 @@ int moc_chunk_pool(const moc_plan *plan, const void *K, float *desc, void *ws, v
  * (which may block on the whole device) are forbidden.  The kernel's scratch (per-slice partial
  * sums and per-chunk arrival counters) lives in a fixed array inside the library image: every
  * GPU that loads the library holds those 4 MiB + 64 KiB until the process exits.
- *   Limits: H * ceil-sum(chunk_len / 256) * d * 4 bytes <= 4 MiB and H * C * 4 bytes <= 64 KiB,
- *   otherwise MOC_ERR_TOO_LARGE and nothing is launched (the 33k-token single-shot clip with 24
- *   heads needs 1.8 MiB; longer streams must use moc_chunk_pool with a workspace).
+ *   Limits: H * units * d * 4 bytes <= 4 MiB and H * C * 4 bytes <= 64 KiB, where a unit is a
+ *   256-token slice of a chunk (the last one shorter); beyond that MOC_ERR_TOO_LARGE and nothing is
+ *   launched (24 heads of the 33k-token single-shot clip need 1.8 MiB; longer streams, or more than
+ *   16384 (head, chunk) pairs, must use moc_chunk_pool with a workspace).
  *   K, desc: as for moc_chunk_pool; the caller still owns inputs and outputs.
  *   The call itself allocates nothing (no cudaMalloc / cudaFree, no allocating library call).
  *   The first call on each device looks up the array's device address; make that first call
