@@ -84,6 +84,22 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks_ms(ms: float, world: int, device) -> float:
+    """Slowest rank's time: ranks are independent replicas, so the job's step time is the max."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(flops_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Whole-job TFLOP/s: every rank does `flops_per_rank` per step in `ms_per_step`."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
 def step_flops(wl, pairs: int, with_bwd: bool) -> float:
     return (4.0 + (10.0 if with_bwd else 0.0)) * wl.head_dim * pairs
 
@@ -259,11 +275,8 @@ def main():
     launches = launch_count() - n0
     total_ms = marks_all[0][0].elapsed_time(marks_all[-1][-1])
     seg = [sum(m[i].elapsed_time(m[i + 1]) for m in marks_all) / args.steps for i in range(len(marks_all[0]) - 1)]
-    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_per_step = float(t.item()) / args.steps
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    ms_per_step = max_over_ranks_ms(total_ms, world, "cuda") / args.steps
+    value = job_value(flops, world, ms_per_step)
 
     # ---- end to end: host buffers in, host results out, copies inside the timed region
     e2e = None
@@ -290,12 +303,10 @@ def main():
             e2e_step()
         e1 = _rec()
         barrier()
-        te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        te_ms = max_over_ranks_ms(e0.elapsed_time(e1), world, "cuda")
         h2d = 3 * hq.numel() * 2
         d2h = hO.numel() * 2 + hl.numel() * 4 + sum(g.numel() * 2 for g in hg)
-        e2e = {"value": world * flops / (float(te.item()) / n_e2e * 1e-3) / 1e12, "unit": UNIT,
+        e2e = {"value": job_value(flops, world, te_ms / n_e2e), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e}
 
     if rank != 0:

@@ -101,8 +101,8 @@ int moc_chunk_pool(const moc_plan *plan, const void *K, float *desc, void *ws, v
  * (which may block on the whole device) are forbidden.  The kernel's scratch (per-slice partial
  * sums and per-chunk arrival counters) lives in a fixed array inside the library image: every
  * GPU that loads the library holds those 4 MiB + 64 KiB until the process exits.
- *   Limits: H * units * d * 4 bytes <= 4 MiB and H * C * 4 bytes <= 64 KiB, where a unit is a
- *   256-token slice of a chunk (the last one shorter); beyond that MOC_ERR_TOO_LARGE and nothing is
+ *   Limits: H * units * d * 4 bytes <= 4 MiB and H * C * 4 bytes <= 64 KiB, where the units are the
+ *   256-token slices of the chunks (each chunk's last one shorter); beyond that MOC_ERR_TOO_LARGE and nothing is
  *   launched (24 heads of the 33k-token single-shot clip need 1.8 MiB; longer streams, or more than
  *   16384 (head, chunk) pairs, must use moc_chunk_pool with a workspace).
  *   K, desc: as for moc_chunk_pool; the caller still owns inputs and outputs.

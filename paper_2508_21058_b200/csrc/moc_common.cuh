@@ -11,7 +11,7 @@
 namespace moc {
 
 constexpr int kQTileRows = 256;     // query rows per attention work item (two 128-row MMA tiles)
-constexpr int kPoolSlice = 256;     // tokens per chunk-pool work unit when chunks are cut into slices
+constexpr int kPoolSlice = 256;     // tokens per chunk-pool work unit
 constexpr int kStatusWords = 16;    // status area at the head of the workspace (int32 each)
 
 // One contiguous range of key tokens [t0, t1).
@@ -57,7 +57,6 @@ struct moc_plan {
     std::vector<int32_t> cap_off;            // [C+1] start of chunk c's query list inside a head's list area
     int c_pad;                               // C rounded up to a multiple of 16 (MMA N granularity)
     int n_pool_units;
-    int pool_slice;                          // tokens per pool work unit
     // device tables (one allocation)
     void *d_blob;
     int32_t *d_off, *d_shot, *d_tok_chunk, *d_anc_off, *d_ranc_off, *d_ranc, *d_pool_unit_off, *d_pool_unit_chunk, *d_cap_off;

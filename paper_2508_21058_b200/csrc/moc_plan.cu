@@ -117,16 +117,13 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
         p->ranc_off[j + 1] = (int32_t)p->ranc.size();
     }
     // query tiles (never straddle a chunk) and pool work units
-    // Pool work units: chunks are cut into slices so that the stream of K spreads over all SMs whatever
-    // the chunk sizes; chunks no longer than a slice are single units and need no partial sums.
-    p->pool_slice = kPoolSlice;
     std::vector<int32_t> tok_chunk(L), unit_chunk;
     p->pool_unit_off.assign(C + 1, 0);
     for (int c = 0; c < C; ++c) {
         for (int t = p->off[c]; t < p->off[c + 1]; ++t) tok_chunk[t] = c;
         for (int r = p->off[c]; r < p->off[c + 1]; r += kQTileRows)
             p->qtiles.push_back(QTile{c, r, std::min(kQTileRows, p->off[c + 1] - r), 0});
-        int units = (p->off[c + 1] - p->off[c] + p->pool_slice - 1) / p->pool_slice;
+        int units = (p->off[c + 1] - p->off[c] + kPoolSlice - 1) / kPoolSlice;
         p->pool_unit_off[c + 1] = p->pool_unit_off[c] + units;
         for (int u = 0; u < units; ++u) unit_chunk.push_back(c);
     }

@@ -1,13 +1,12 @@
 // Chunk descriptors: desc[h][c][:] = mean of K[h][t][:] over the chunk's tokens.
 //
-// HBM-bound stream of K.  A work unit is (head, chunk, slice of `slice_len` tokens); a
+// HBM-bound stream of K.  A work unit is (head, chunk, slice of kPoolSlice tokens); a
 // block of 256 threads reads its slice with 128-bit loads (a token row of d bf16 is
 // d/8 lanes wide, so one pass covers 256*8/d rows and every warp reads whole 128-byte
 // lines), accumulates in fp32 registers, folds the row groups through shared memory
 // and writes one partial sum.  The last block to finish a chunk (arrival counter)
 // adds the partials in slice order and scales by 1/n, so the result does not depend
-// on block scheduling.  When every chunk is a single unit (slice_len covers the longest
-// chunk) the block writes the mean itself: no partial sums, no counters.
+// on block scheduling.
 #include <mutex>
 
 #include "moc_common.cuh"
@@ -20,7 +19,7 @@ __global__ void __launch_bounds__(256) chunk_pool_kernel(const __nv_bfloat16 *__
                                                           const int32_t *__restrict__ off,
                                                           const int32_t *__restrict__ unit_off,
                                                           const int32_t *__restrict__ unit_chunk, int L, int C,
-                                                          int n_units, int slice_len) {
+                                                          int n_units) {
     constexpr int LANES = D / 8;          // 16-byte lanes per token row
     constexpr int ROWS = 256 / LANES;     // rows per pass
     __shared__ float red[ROWS][D + 4];
@@ -30,9 +29,8 @@ __global__ void __launch_bounds__(256) chunk_pool_kernel(const __nv_bfloat16 *__
     for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
         const int c = unit_chunk[unit];
         const int slice = unit - unit_off[c];
-        const int t0 = off[c] + slice * slice_len;
-        const int t1 = (int)min((long long)off[c + 1], (long long)t0 + slice_len);
-        const bool whole = n_units == C;      // one unit per chunk
+        const int t0 = off[c] + slice * kPoolSlice;
+        const int t1 = min(off[c + 1], t0 + kPoolSlice);
         float acc[8];
 #pragma unroll
         for (int x = 0; x < 8; ++x) acc[x] = 0.f;
@@ -72,15 +70,10 @@ __global__ void __launch_bounds__(256) chunk_pool_kernel(const __nv_bfloat16 *__
             float s = 0.f;
 #pragma unroll
             for (int r = 0; r < ROWS; ++r) s += red[r][threadIdx.x];
-            if (whole) {
-                desc[((size_t)h * C + c) * D + threadIdx.x] = s / (float)(off[c + 1] - off[c]);
-            } else {
-                mine[threadIdx.x] = s;
-                __threadfence();
-            }
+            mine[threadIdx.x] = s;
+            __threadfence();
         }
         __syncthreads();
-        if (whole) continue;
         if (threadIdx.x == 0) {
             const int n_slices = unit_off[c + 1] - unit_off[c];
             int prev = atomicAdd(&done[h * C + c], 1);
@@ -108,19 +101,17 @@ __global__ void zero_i32_kernel(int *p, size_t n) {
 int launch_chunk_pool(const moc_plan *p, const __nv_bfloat16 *K, float *desc, void *ws, cudaStream_t s) {
     float *part = ws_ptr<float>(ws, p->ws.pool_part);
     int *done = ws_ptr<int>(ws, p->ws.pool_done);
-    if (p->n_pool_units != p->C) {
-        // the arrival counters live in caller-owned scratch whose contents are unknown
-        size_t n = (size_t)p->H * p->C;
-        zero_i32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(done, n);
-        MOC_LAUNCH_CHECK();
-    }
+    // the arrival counters live in caller-owned scratch whose contents are unknown
+    size_t n = (size_t)p->H * p->C;
+    zero_i32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(done, n);
+    MOC_LAUNCH_CHECK();
     dim3 grid((unsigned)std::min(p->n_pool_units, 65535), (unsigned)p->H);
     if (p->d == 128)
         chunk_pool_kernel<128><<<grid, 256, 0, s>>>(K, desc, part, done, p->d_off, p->d_pool_unit_off,
-                                                    p->d_pool_unit_chunk, p->L, p->C, p->n_pool_units, p->pool_slice);
+                                                    p->d_pool_unit_chunk, p->L, p->C, p->n_pool_units);
     else
         chunk_pool_kernel<64><<<grid, 256, 0, s>>>(K, desc, part, done, p->d_off, p->d_pool_unit_off,
-                                                   p->d_pool_unit_chunk, p->L, p->C, p->n_pool_units, p->pool_slice);
+                                                   p->d_pool_unit_chunk, p->L, p->C, p->n_pool_units);
     MOC_LAUNCH_CHECK();
     return MOC_OK;
 }
@@ -181,10 +172,10 @@ extern "C" int moc_chunk_pool_noalloc(const moc_plan *p, const void *K, float *d
     dim3 grid((unsigned)std::min(p->n_pool_units, 65535), (unsigned)p->H);
     if (p->d == 128)
         chunk_pool_kernel<128><<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(K), desc, part, done, p->d_off,
-                                                    p->d_pool_unit_off, p->d_pool_unit_chunk, p->L, p->C, p->n_pool_units, p->pool_slice);
+                                                    p->d_pool_unit_off, p->d_pool_unit_chunk, p->L, p->C, p->n_pool_units);
     else
         chunk_pool_kernel<64><<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(K), desc, part, done, p->d_off,
-                                                   p->d_pool_unit_off, p->d_pool_unit_chunk, p->L, p->C, p->n_pool_units, p->pool_slice);
+                                                   p->d_pool_unit_off, p->d_pool_unit_chunk, p->L, p->C, p->n_pool_units);
     MOC_LAUNCH_CHECK();
     return MOC_OK;
 }

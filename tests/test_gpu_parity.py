@@ -153,12 +153,14 @@ def test_argument_errors_launch_nothing():
     assert launch_count() == n0
 
 
-@pytest.mark.parametrize("name,rows_per_head", [("cfg1", 96)])
-def test_forward_benchmark_size_sampled(name, rows_per_head):
+@pytest.mark.parametrize("name,rows_per_head,heads", [("cfg1", 96, None), ("cfg2", 192, 3)])
+def test_forward_benchmark_size_sampled(name, rows_per_head, heads):
     """The benchmark workload in the launch configuration bench.py times; attention
     checked on sampled rows (frame, caption and shot edges plus uniform picks), indices on
     every row of a sample of heads."""
     wl = W.workload(name)
+    if heads is not None:       # the multi-shot stream at its full length, on a few heads (each head is independent)
+        wl.n_heads = heads
     run = PU.GpuRun(wl).forward()
     x = run.host_inputs()
     orc = Oracle.from_workload(wl)
