@@ -84,6 +84,23 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def measured_traffic(kernel: str, workload: str):
+    """DRAM bytes per call from the committed ncu summary, or None when the kernel source has
+    changed since the counters were taken (profiles/traffic.txt: kernel workload bytes sha1-of-source)."""
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.txt")) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) == 5 and parts[0] == kernel and parts[1] == workload:
+                    with open(os.path.join(ROOT, parts[4]), "rb") as src:
+                        if hashlib.sha1(src.read()).hexdigest() == parts[3]:
+                            return float(parts[2])
+    except Exception:
+        pass
+    return None
+
+
 def max_over_ranks_ms(ms: float, world: int, device) -> float:
     """Slowest rank's time: ranks are independent replicas, so the job's step time is the max."""
     if world <= 1:
@@ -317,12 +334,7 @@ def main():
     peaks, peak_kind = load_peaks()
     t_pool, t_route, t_att = seg[0], seg[1], seg[2]
     att_flops = step_flops(wl, pairs, False)
-    traffic = None
-    try:
-        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
-            traffic = json.load(f).get(f"attend:{wl.name}")
-    except Exception:
-        pass
+    traffic = measured_traffic("moc_attend", wl.name)
     roofline = {"kernel": "moc_attend (tensor-core flash kernel over selected key chunks)" if not args.scalar
                 else "moc_attend (CUDA-core kernels)",
                 "bound": "tensor", "achieved": att_flops / (t_att * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
