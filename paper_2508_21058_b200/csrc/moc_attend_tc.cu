@@ -54,17 +54,13 @@ struct AttendParams {
     float *lse;
     __nv_bfloat16 *part_o;
     float *part_lse;
-    const int32_t *off;
-    const int32_t *anc_off;
-    const KeyRange *anc_rng;
-    const QTile *qtiles;
-    const int *gtile_off;   // [H*C + 1] running count of routed tiles over (head, chunk)
-    const int *cnt;         // [H][C] picks per (head, chunk)
-    const int32_t *cap_off; // [C + 1] start of chunk c's list inside a head's list area
-    const int32_t *qlist;   // [H][cap_total]
+    const KeyRange *rng;        // key ranges the items index: merged anchor ranges, or the chunks
+    const WorkItem *items;      // anchor pass: one head's items (blockIdx.y = head); routed pass: every item
+    const int *n_items_dev;     // routed pass: the item count lives on the device
+    const int32_t *qlist;       // [H][cap_total]
     size_t cap_total;
     int *status;
-    int H, L, C, k;
+    int H, L, k;
     float scale_log2;       // softmax scale * log2(e)
 };
 
@@ -139,7 +135,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     __shared__ uint32_t tmem_slot;
     __shared__ int s_abort;
     __shared__ int w_valid, w_h, w_rows, w_first, w_nrng, w_ntiles;
-    __shared__ KeyRange w_rng0;
+    __shared__ int s_qrow[kQTileRows];              // query row behind each row of the item (-1 = padding)
     __shared__ const KeyRange *w_rng;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -155,36 +151,15 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     if (threadIdx.x == 0) {
         s_abort = 0;
         int valid = (*(volatile int *)p.status == 0);
-        if (ROUTED) {
-            const int HC = p.H * p.C;
-            const int tile = blockIdx.x;
-            if (tile >= p.gtile_off[HC]) valid = 0;
-            if (valid) {
-                int lo = 0, hi = HC;   // largest hc with gtile_off[hc] <= tile
-                while (hi - lo > 1) {
-                    const int mid = (lo + hi) >> 1;
-                    if (p.gtile_off[mid] <= tile) lo = mid; else hi = mid;
-                }
-                const int h = lo / p.C, c = lo % p.C;
-                const int nth = tile - p.gtile_off[lo];
-                w_h = h;
-                w_first = p.cap_off[c] + nth * kQTileRows;
-                w_rows = min(kQTileRows, p.cnt[lo] - nth * kQTileRows);
-                w_rng0 = KeyRange{p.off[c], p.off[c + 1]};
-                w_rng = &w_rng0;
-                w_nrng = 1;
-                w_ntiles = (p.off[c + 1] - p.off[c] + kBN - 1) / kBN;
-            }
-        } else {
-            const QTile qt = p.qtiles[blockIdx.x];
-            w_h = blockIdx.y;
-            w_first = qt.row0;
-            w_rows = qt.rows;
-            w_rng = p.anc_rng + p.anc_off[qt.chunk];
-            w_nrng = p.anc_off[qt.chunk + 1] - p.anc_off[qt.chunk];
-            int nt = 0;
-            for (int r = 0; r < w_nrng; ++r) nt += (w_rng[r].t1 - w_rng[r].t0 + kBN - 1) / kBN;
-            w_ntiles = nt;
+        if (ROUTED && valid && (int)blockIdx.x >= *p.n_items_dev) valid = 0;
+        if (valid) {
+            const WorkItem w = p.items[blockIdx.x];
+            w_h = ROUTED ? w.h : (int)blockIdx.y;
+            w_first = w.first;
+            w_rows = w.rows;
+            w_rng = p.rng + w.rng_off;
+            w_nrng = w.nrng;
+            w_ntiles = w.ntiles;
         }
         w_valid = valid;
         for (int t = 0; t < 2; ++t) {
@@ -239,14 +214,23 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 }
             }
             {
-                const uint4 *src = reinterpret_cast<const uint4 *>(p.Q + ((size_t)h * p.L + (qi >= 0 ? qi : 0)) * D);
-                uint8_t *dstq = gbase + g * TILE_BYTES;
+                // The group stages its Q tile together: consecutive threads take consecutive 16-byte pieces
+                // of a row, so every request covers whole 128-byte lines even when the rows are gathered.
+                s_qrow[g * 128 + r] = qi;
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory");     // the group's 128 threads; nothing can have failed yet
+                constexpr int CH = D / 8, RP = 128 / CH;       // pieces per row, rows per pass
+                const int c16 = r % CH;
+                uint8_t *dstq = gbase + g * TILE_BYTES + (c16 >> 3) * SUB_BYTES;
+                uint4 v[CH];
 #pragma unroll
-                for (int c16 = 0; c16 < D / 8; ++c16) {
-                    uint4 v = make_uint4(0, 0, 0, 0);
-                    if (qi >= 0) v = __ldg(src + c16);
-                    *reinterpret_cast<uint4 *>(dstq + (c16 >> 3) * SUB_BYTES + sw128_offset(r, c16 & 7)) = v;
+                for (int ps = 0; ps < CH; ++ps) {
+                    const int rr = ps * RP + r / CH, q = s_qrow[g * 128 + rr];
+                    v[ps] = make_uint4(0, 0, 0, 0);
+                    if (q >= 0) v[ps] = __ldg(reinterpret_cast<const uint4 *>(p.Q + ((size_t)h * p.L + q) * D) + c16);
                 }
+#pragma unroll
+                for (int ps = 0; ps < CH; ++ps)
+                    *reinterpret_cast<uint4 *>(dstq + sw128_offset(ps * RP + r / CH, c16 & 7)) = v[ps];
             }
             fence_proxy_async_smem();
             mbar_arrive(bar(Q_FULL + g));
@@ -574,14 +558,10 @@ static int attend_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfl
     a.Q = Q; a.O = O; a.lse = lse;
     a.part_o = ws_ptr<__nv_bfloat16>(ws, p->ws.part_o);
     a.part_lse = ws_ptr<float>(ws, p->ws.part_lse);
-    a.off = p->d_off; a.anc_off = p->d_anc_off; a.anc_rng = p->d_anc_rng; a.qtiles = p->d_qtiles;
-    a.gtile_off = ws_ptr<int>(ws, p->ws.tile_off);
-    a.cnt = ws_ptr<int>(ws, p->ws.cnt);
-    a.cap_off = p->d_cap_off;
     a.qlist = ws_ptr<int32_t>(ws, p->ws.qlist);
     a.cap_total = (size_t)p->cap_off[p->C];
     a.status = ws_ptr<int>(ws, p->ws.status);
-    a.H = p->H; a.L = p->L; a.C = p->C; a.k = p->k;
+    a.H = p->H; a.L = p->L; a.k = p->k;
     a.scale_log2 = p->scale * 1.4426950408889634f;
     // always the d = 128 footprint: more than half an SM's shared memory, so CTAs (which each
     // take all 512 TMEM columns) never share an SM
@@ -593,11 +573,19 @@ static int attend_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfl
         attr_done[D == 128] = true;
     }
     if (p->k > 0) {
+        // routed pass: the items and their count were left in the workspace by moc_route; the grid covers
+        // the most there can be
+        a.rng = p->d_chunk_rng;
+        a.items = ws_ptr<WorkItem>(ws, p->ws.rtiles);
+        a.n_items_dev = ws_ptr<int>(ws, p->ws.tile_off) + (size_t)p->H * p->C;
         const long long bound = (long long)p->H * (((long long)p->L * p->k + kQTileRows - 1) / kQTileRows + p->C);
         attend_tc_kernel<D, true><<<(unsigned)bound, kThreads, smem, s>>>(tmK, tmV, a);
         MOC_LAUNCH_CHECK();
     }
-    dim3 grid((unsigned)p->qtiles.size(), (unsigned)p->H);
+    a.rng = p->d_anc_rng;
+    a.items = p->d_qitems;
+    a.n_items_dev = nullptr;
+    dim3 grid((unsigned)p->qitems.size(), (unsigned)p->H);
     attend_tc_kernel<D, false><<<grid, kThreads, smem, s>>>(tmK, tmV, a);
     MOC_LAUNCH_CHECK();
     return MOC_OK;

@@ -17,13 +17,17 @@ constexpr int kStatusWords = 16;    // status area at the head of the workspace 
 // One contiguous range of key tokens [t0, t1).
 struct KeyRange { int32_t t0, t1; };
 
-// A tile of <= kQTileRows consecutive query rows that all live in chunk c.
-struct QTile { int32_t chunk, row0, rows, pad; };
+// One attention work item: up to kQTileRows query rows of head h against the key ranges
+// rng[rng_off .. rng_off + nrng) (ntiles key tiles of 128; [t0, t1) repeats the first range).  Anchor pass: `first` is the first of `rows`
+// consecutive query rows of one chunk (h is implied by the item index).  Routed pass: `first` is the
+// offset, inside the head's list area, of the `rows` entries of one chunk's query list.
+struct WorkItem { int32_t h, first, rows, ntiles, rng_off, nrng, t0, t1; };
 
 struct WsLayout {
     size_t status;      // int32[kStatusWords]: [0] device status, [1] detail, [2] routed-flag
     size_t cnt;         // int32[H][C]     routed picks per (head, chunk); doubles as the list cursor while routing
     size_t tile_off;    // int32[H*C+1]    running count of routed attention tiles over (head, chunk) pairs
+    size_t rtiles;      // WorkItem[H * (ceil(L k / 256) + C)]  routed work items, written after routing
     size_t qlist;       // int32[H][cap_total]  per (head, chunk) list at cap_off[c]: entries i*k+s of the picks of c
     size_t desc3;       // bf16 [H][3][Cpad][d]  descriptors split into three bf16 terms (hi + mid + lo)
     size_t pool_part;   // float[H][n_pool_units][d] partial key sums
@@ -51,7 +55,7 @@ struct moc_plan {
     std::vector<moc::KeyRange> anc_rng;      // merged anchor token ranges per query chunk
     std::vector<int64_t> anc_tokens;         // [C] anchor key tokens per query chunk
     std::vector<int32_t> ranc_off, ranc;     // reverse anchors: key chunk -> query chunks
-    std::vector<moc::QTile> qtiles;
+    std::vector<moc::WorkItem> qitems;       // anchor-pass work items of one head
     std::vector<int32_t> pool_unit_off;      // [C+1] prefix of pool units per chunk
     int words;                               // uint32 words per anchor bitmap row
     std::vector<int32_t> cap_off;            // [C+1] start of chunk c's query list inside a head's list area
@@ -63,7 +67,8 @@ struct moc_plan {
     uint8_t *d_mod;
     uint32_t *d_anc_bits;
     moc::KeyRange *d_anc_rng;
-    moc::QTile *d_qtiles;
+    moc::WorkItem *d_qitems;
+    moc::KeyRange *d_chunk_rng;              // [C] token range of every chunk
     moc::WsLayout ws;
 };
 

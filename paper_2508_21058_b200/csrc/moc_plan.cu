@@ -41,6 +41,7 @@ static void layout_workspace(moc_plan *p) {
     w.status = take(sizeof(int32_t) * kStatusWords);
     w.cnt = take(sizeof(int32_t) * H * C);
     w.tile_off = take(sizeof(int32_t) * (H * C + 1));
+    w.rtiles = take(sizeof(WorkItem) * H * ((L * (k ? k : 1) + kQTileRows - 1) / kQTileRows + C));
     w.qlist = take(sizeof(int32_t) * H * (size_t)std::max(p->cap_off[C], 1));
     w.desc3 = take(sizeof(__nv_bfloat16) * H * 3 * (size_t)p->c_pad * d);
     w.pool_part = take(sizeof(float) * H * (size_t)p->n_pool_units * d);
@@ -118,11 +119,17 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
     }
     // query tiles (never straddle a chunk) and pool work units
     std::vector<int32_t> tok_chunk(L), unit_chunk;
+    std::vector<KeyRange> chunk_rng(C);
+    for (int c = 0; c < C; ++c) chunk_rng[c] = KeyRange{p->off[c], p->off[c + 1]};
     p->pool_unit_off.assign(C + 1, 0);
     for (int c = 0; c < C; ++c) {
         for (int t = p->off[c]; t < p->off[c + 1]; ++t) tok_chunk[t] = c;
+        int anc_tiles = 0;
+        for (int a = p->anc_off[c]; a < p->anc_off[c + 1]; ++a) anc_tiles += (p->anc_rng[a].t1 - p->anc_rng[a].t0 + 127) / 128;
         for (int r = p->off[c]; r < p->off[c + 1]; r += kQTileRows)
-            p->qtiles.push_back(QTile{c, r, std::min(kQTileRows, p->off[c + 1] - r), 0});
+            p->qitems.push_back(WorkItem{0, r, std::min(kQTileRows, p->off[c + 1] - r), anc_tiles, p->anc_off[c],
+                                         p->anc_off[c + 1] - p->anc_off[c], p->anc_rng[p->anc_off[c]].t0,
+                                         p->anc_rng[p->anc_off[c]].t1});
         int units = (p->off[c + 1] - p->off[c] + kPoolSlice - 1) / kPoolSlice;
         p->pool_unit_off[c + 1] = p->pool_unit_off[c] + units;
         for (int u = 0; u < units; ++u) unit_chunk.push_back(c);
@@ -146,8 +153,8 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
     size_t o_off = take(4 * (C + 1)), o_shot = take(4 * C), o_mod = take(C), o_tok = take(4 * (size_t)L);
     size_t o_bits = take(4 * bits.size()), o_aoff = take(4 * (C + 1)), o_arng = take(sizeof(KeyRange) * p->anc_rng.size());
-    size_t o_roff = take(4 * (C + 1)), o_ranc = take(4 * p->ranc.size()), o_qt = take(sizeof(QTile) * p->qtiles.size());
-    size_t o_puo = take(4 * (C + 1)), o_puc = take(4 * unit_chunk.size()), o_cap = take(4 * (C + 1));
+    size_t o_roff = take(4 * (C + 1)), o_ranc = take(4 * p->ranc.size()), o_qt = take(sizeof(WorkItem) * p->qitems.size());
+    size_t o_puo = take(4 * (C + 1)), o_puc = take(4 * unit_chunk.size()), o_cap = take(4 * (C + 1)), o_crng = take(sizeof(KeyRange) * C);
     cudaError_t e = cudaMalloc(&p->d_blob, o);
     if (e != cudaSuccess) { set_cuda_error(e, "cudaMalloc(plan tables)"); delete p; return MOC_ERR_CUDA; }
     char *b = static_cast<char *>(p->d_blob);
@@ -158,17 +165,18 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
                         up(o_tok, tok_chunk.data(), 4 * (size_t)L), up(o_bits, bits.data(), 4 * bits.size()),
                         up(o_aoff, p->anc_off.data(), 4 * (C + 1)), up(o_arng, p->anc_rng.data(), sizeof(KeyRange) * p->anc_rng.size()),
                         up(o_roff, p->ranc_off.data(), 4 * (C + 1)), up(o_ranc, p->ranc.data(), 4 * p->ranc.size()),
-                        up(o_qt, p->qtiles.data(), sizeof(QTile) * p->qtiles.size()),
+                        up(o_qt, p->qitems.data(), sizeof(WorkItem) * p->qitems.size()),
                         up(o_puo, p->pool_unit_off.data(), 4 * (C + 1)), up(o_puc, unit_chunk.data(), 4 * unit_chunk.size()),
-                        up(o_cap, p->cap_off.data(), 4 * (C + 1))};
+                        up(o_cap, p->cap_off.data(), 4 * (C + 1)), up(o_crng, chunk_rng.data(), sizeof(KeyRange) * C)};
     for (cudaError_t x : es)
         if (x != cudaSuccess) { set_cuda_error(x, "cudaMemcpy(plan tables)"); cudaFree(p->d_blob); delete p; return MOC_ERR_CUDA; }
     p->d_off = (int32_t *)(b + o_off); p->d_shot = (int32_t *)(b + o_shot); p->d_mod = (uint8_t *)(b + o_mod);
     p->d_tok_chunk = (int32_t *)(b + o_tok); p->d_anc_bits = (uint32_t *)(b + o_bits);
     p->d_anc_off = (int32_t *)(b + o_aoff); p->d_anc_rng = (KeyRange *)(b + o_arng);
-    p->d_ranc_off = (int32_t *)(b + o_roff); p->d_ranc = (int32_t *)(b + o_ranc); p->d_qtiles = (QTile *)(b + o_qt);
+    p->d_ranc_off = (int32_t *)(b + o_roff); p->d_ranc = (int32_t *)(b + o_ranc); p->d_qitems = (WorkItem *)(b + o_qt);
     p->d_pool_unit_off = (int32_t *)(b + o_puo); p->d_pool_unit_chunk = (int32_t *)(b + o_puc);
     p->d_cap_off = (int32_t *)(b + o_cap);
+    p->d_chunk_rng = (KeyRange *)(b + o_crng);
     *out = p;
     return MOC_OK;
 }

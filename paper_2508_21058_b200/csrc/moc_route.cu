@@ -21,7 +21,8 @@
 //                 histogram, one global atomic per (tile, chunk) to reserve the range).
 //   The head's descriptor block stays in shared memory for the CTA's lifetime (C <= 192);
 //   with more chunks it is streamed in blocks of 128 and warp 1 alone issues.
-// route_tiles_kernel  running count of attention tiles over (head, chunk) from the pick counts.
+// route_tiles_kernel  running count of attention tiles over (head, chunk) from the pick counts;
+// route_items_kernel  the routed attention work items (one per 256 picks of a chunk).
 // Every mbarrier wait is bounded; a wait that runs out flags the workspace status word.
 #include <float.h>
 #include <algorithm>
@@ -549,6 +550,18 @@ __global__ void __launch_bounds__(1024) route_tiles_kernel(const int *__restrict
     if (t == 1023) { gtile[HC] = st[1023]; status[2] = 1; }
 }
 
+// The routed work items of (head, chunk) pair i: one per kQTileRows entries of its query list.
+__global__ void route_items_kernel(const int *__restrict__ cnt, const int *__restrict__ gtile, WorkItem *__restrict__ items,
+                                   const int32_t *__restrict__ off, const int32_t *__restrict__ cap_off, int H, int C) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= H * C) return;
+    const int h = i / C, c = i % C, n = cnt[i];
+    const int key_tiles = (off[c + 1] - off[c] + 127) / 128;
+    int at = gtile[i];
+    for (int e0 = 0; e0 < n; e0 += kQTileRows)
+        items[at++] = WorkItem{h, cap_off[c] + e0, min(kQTileRows, n - e0), key_tiles, c, 1, off[c], off[c + 1]};
+}
+
 #ifdef MOC_TRACE
 extern "C" int moc_trace_read_route(long long *host, int n) {
     return (int)cudaMemcpyFromSymbol(host, g_trace_route, sizeof(long long) * (size_t)n);
@@ -601,6 +614,12 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
     }
     route_tiles_kernel<<<1, 1024, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off), status, p->H * p->C);
     MOC_LAUNCH_CHECK();
+    if (p->k > 0) {
+        route_items_kernel<<<(unsigned)((p->H * p->C + 127) / 128), 128, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off),
+                                                                               ws_ptr<WorkItem>(ws, p->ws.rtiles), p->d_off,
+                                                                               p->d_cap_off, p->H, p->C);
+        MOC_LAUNCH_CHECK();
+    }
     return MOC_OK;
 }
 
