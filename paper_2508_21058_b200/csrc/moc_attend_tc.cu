@@ -234,6 +234,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             }
             fence_proxy_async_smem();
             mbar_arrive(bar(Q_FULL + g));
+            if (!ROUTED && qi >= 0) {
+                // the epilogue will merge this row's routed partials: start them on their way into L2 now
+                const char *po = reinterpret_cast<const char *>(p.part_o + ((size_t)h * p.L + qi) * p.k * D);
+                for (int b = 0; b < p.k * D * 2; b += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(po + b));
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(p.part_lse + ((size_t)h * p.L + qi) * p.k));
+            }
             if (r == 0) TRACE(10 + g);
 
             float m_run = -INFINITY, l_run = 0.f;

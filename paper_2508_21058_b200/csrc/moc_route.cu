@@ -553,13 +553,13 @@ __global__ void __launch_bounds__(1024) route_tiles_kernel(const int *__restrict
 // The routed work items of (head, chunk) pair i: one per kQTileRows entries of its query list.
 __global__ void route_items_kernel(const int *__restrict__ cnt, const int *__restrict__ gtile, WorkItem *__restrict__ items,
                                    const int32_t *__restrict__ off, const int32_t *__restrict__ cap_off, int H, int C) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;     // one warp per pair
     if (i >= H * C) return;
     const int h = i / C, c = i % C, n = cnt[i];
     const int key_tiles = (off[c + 1] - off[c] + 127) / 128;
-    int at = gtile[i];
-    for (int e0 = 0; e0 < n; e0 += kQTileRows)
-        items[at++] = WorkItem{h, cap_off[c] + e0, min(kQTileRows, n - e0), key_tiles, c, 1, off[c], off[c + 1]};
+    const int at = gtile[i];
+    for (int x = lane; x * kQTileRows < n; x += 32)
+        items[at + x] = WorkItem{h, cap_off[c] + x * kQTileRows, min(kQTileRows, n - x * kQTileRows), key_tiles, c, 1, off[c], off[c + 1]};
 }
 
 #ifdef MOC_TRACE
@@ -615,7 +615,7 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
     route_tiles_kernel<<<1, 1024, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off), status, p->H * p->C);
     MOC_LAUNCH_CHECK();
     if (p->k > 0) {
-        route_items_kernel<<<(unsigned)((p->H * p->C + 127) / 128), 128, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off),
+        route_items_kernel<<<(unsigned)((p->H * p->C + 3) / 4), 128, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off),
                                                                                ws_ptr<WorkItem>(ws, p->ws.rtiles), p->d_off,
                                                                                p->d_cap_off, p->H, p->C);
         MOC_LAUNCH_CHECK();
