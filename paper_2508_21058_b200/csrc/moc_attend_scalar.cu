@@ -297,6 +297,15 @@ static int attend_bwd_scalar_d(const moc_plan *p, const __nv_bfloat16 *Q, const 
     return MOC_OK;
 }
 
+int launch_delta(const moc_plan *p, const __nv_bfloat16 *O, const __nv_bfloat16 *dO, float *delta, cudaStream_t s) {
+    const size_t rows = (size_t)p->H * p->L;
+    const unsigned grid = (unsigned)((rows + 3) / 4);
+    if (p->d == 128) delta_kernel<128><<<grid, 128, 0, s>>>(O, dO, delta, rows);
+    else delta_kernel<64><<<grid, 128, 0, s>>>(O, dO, delta, rows);
+    MOC_LAUNCH_CHECK();
+    return MOC_OK;
+}
+
 int launch_attend_bwd_scalar(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
                              const __nv_bfloat16 *O, const float *lse, const __nv_bfloat16 *dO, const int32_t *sel,
                              __nv_bfloat16 *dQ, __nv_bfloat16 *dK, __nv_bfloat16 *dV, void *ws, cudaStream_t s) {

@@ -73,56 +73,6 @@ constexpr float kRescaleThreshold = 8.0f;
 
 enum WaitCode { W_QFULL = 1, W_KFULL, W_VFULL, W_SFULL, W_PFULL, W_OFULL, W_KEMPTY, W_VEMPTY, W_TURN, W_PHALF };
 
-struct TileIter {
-    const KeyRange *rng;
-    int n, ri, t;
-    __device__ TileIter(const KeyRange *r, int n_) : rng(r), n(n_), ri(0), t(n_ > 0 ? r[0].t0 : 0) {}
-    __device__ bool next(int &t0, int &valid) {
-        if (ri >= n) return false;
-        const int end = rng[ri].t1;
-        t0 = t;
-        valid = min(kBN, end - t);
-        t += kBN;
-        if (t >= end) { ++ri; if (ri < n) t = rng[ri].t0; }
-        return true;
-    }
-};
-
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-// two fp32 values in one 64-bit register pair, for the packed fp32 instructions
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-// (lo, hi) -> packed bf16x2, round to nearest even
-__device__ __forceinline__ uint32_t bf16x2(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
 template <int D, bool ROUTED>
 __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                 const __grid_constant__ CUtensorMap tmV,

@@ -23,6 +23,9 @@ struct KeyRange { int32_t t0, t1; };
 // offset, inside the head's list area, of the `rows` entries of one chunk's query list.
 struct WorkItem { int32_t h, first, rows, ntiles, rng_off, nrng, t0, t1; };
 
+// One tile of up to 128 consecutive key tokens of chunk c (backward, key-stationary pass).
+struct KTile { int32_t chunk, t0, valid, pad; };
+
 struct WsLayout {
     size_t status;      // int32[kStatusWords]: [0] device status, [1] detail, [2] routed-flag
     size_t cnt;         // int32[H][C]     routed picks per (head, chunk); doubles as the list cursor while routing
@@ -56,6 +59,7 @@ struct moc_plan {
     std::vector<int64_t> anc_tokens;         // [C] anchor key tokens per query chunk
     std::vector<int32_t> ranc_off, ranc;     // reverse anchors: key chunk -> query chunks
     std::vector<moc::WorkItem> qitems;       // anchor-pass work items of one head
+    std::vector<moc::KTile> ktiles;          // key tiles of one head, chunk by chunk
     std::vector<int32_t> pool_unit_off;      // [C+1] prefix of pool units per chunk
     int words;                               // uint32 words per anchor bitmap row
     std::vector<int32_t> cap_off;            // [C+1] start of chunk c's query list inside a head's list area
@@ -69,6 +73,7 @@ struct moc_plan {
     moc::KeyRange *d_anc_rng;
     moc::WorkItem *d_qitems;
     moc::KeyRange *d_chunk_rng;              // [C] token range of every chunk
+    moc::KTile *d_ktiles;
     moc::WsLayout ws;
 };
 
@@ -101,6 +106,24 @@ static inline T *ws_ptr(void *ws, size_t off) { return reinterpret_cast<T *>(sta
 template <typename T>
 static inline const T *ws_ptr(const void *ws, size_t off) { return reinterpret_cast<const T *>(static_cast<const char *>(ws) + off); }
 
+#ifdef __CUDACC__
+// Walks the 128-key tiles of a list of key ranges (a tile never straddles two ranges).
+struct TileIter {
+    const KeyRange *rng;
+    int n, ri, t;
+    __device__ TileIter(const KeyRange *r, int n_) : rng(r), n(n_), ri(0), t(n_ > 0 ? r[0].t0 : 0) {}
+    __device__ bool next(int &t0, int &valid) {
+        if (ri >= n) return false;
+        const int end = rng[ri].t1;
+        t0 = t;
+        valid = min(128, end - t);
+        t += 128;
+        if (t >= end) { ++ri; if (ri < n) t = rng[ri].t0; }
+        return true;
+    }
+};
+#endif
+
 static inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 // kernels' host launchers (each returns a moc_status)
@@ -111,6 +134,10 @@ int launch_attend_scalar(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_b
 int launch_attend_bwd_scalar(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
                              const __nv_bfloat16 *O, const float *lse, const __nv_bfloat16 *dO, const int32_t *sel,
                              __nv_bfloat16 *dQ, __nv_bfloat16 *dK, __nv_bfloat16 *dV, void *ws, cudaStream_t s);
+int launch_attend_bwd_tc(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
+                         const __nv_bfloat16 *O, const float *lse, const __nv_bfloat16 *dO, const int32_t *sel,
+                         __nv_bfloat16 *dQ, __nv_bfloat16 *dK, __nv_bfloat16 *dV, void *ws, cudaStream_t s);
+int launch_delta(const moc_plan *p, const __nv_bfloat16 *O, const __nv_bfloat16 *dO, float *delta, cudaStream_t s);
 int launch_attend_tc(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
                      const int32_t *sel, __nv_bfloat16 *O, float *lse, void *ws, cudaStream_t s);
 

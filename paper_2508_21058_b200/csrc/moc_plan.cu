@@ -130,6 +130,7 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
             p->qitems.push_back(WorkItem{0, r, std::min(kQTileRows, p->off[c + 1] - r), anc_tiles, p->anc_off[c],
                                          p->anc_off[c + 1] - p->anc_off[c], p->anc_rng[p->anc_off[c]].t0,
                                          p->anc_rng[p->anc_off[c]].t1});
+        for (int t = p->off[c]; t < p->off[c + 1]; t += 128) p->ktiles.push_back(KTile{c, t, std::min(128, p->off[c + 1] - t), 0});
         int units = (p->off[c + 1] - p->off[c] + kPoolSlice - 1) / kPoolSlice;
         p->pool_unit_off[c + 1] = p->pool_unit_off[c] + units;
         for (int u = 0; u < units; ++u) unit_chunk.push_back(c);
@@ -154,7 +155,7 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
     size_t o_off = take(4 * (C + 1)), o_shot = take(4 * C), o_mod = take(C), o_tok = take(4 * (size_t)L);
     size_t o_bits = take(4 * bits.size()), o_aoff = take(4 * (C + 1)), o_arng = take(sizeof(KeyRange) * p->anc_rng.size());
     size_t o_roff = take(4 * (C + 1)), o_ranc = take(4 * p->ranc.size()), o_qt = take(sizeof(WorkItem) * p->qitems.size());
-    size_t o_puo = take(4 * (C + 1)), o_puc = take(4 * unit_chunk.size()), o_cap = take(4 * (C + 1)), o_crng = take(sizeof(KeyRange) * C);
+    size_t o_puo = take(4 * (C + 1)), o_puc = take(4 * unit_chunk.size()), o_cap = take(4 * (C + 1)), o_crng = take(sizeof(KeyRange) * C), o_kt = take(sizeof(KTile) * p->ktiles.size());
     cudaError_t e = cudaMalloc(&p->d_blob, o);
     if (e != cudaSuccess) { set_cuda_error(e, "cudaMalloc(plan tables)"); delete p; return MOC_ERR_CUDA; }
     char *b = static_cast<char *>(p->d_blob);
@@ -167,7 +168,8 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
                         up(o_roff, p->ranc_off.data(), 4 * (C + 1)), up(o_ranc, p->ranc.data(), 4 * p->ranc.size()),
                         up(o_qt, p->qitems.data(), sizeof(WorkItem) * p->qitems.size()),
                         up(o_puo, p->pool_unit_off.data(), 4 * (C + 1)), up(o_puc, unit_chunk.data(), 4 * unit_chunk.size()),
-                        up(o_cap, p->cap_off.data(), 4 * (C + 1)), up(o_crng, chunk_rng.data(), sizeof(KeyRange) * C)};
+                        up(o_cap, p->cap_off.data(), 4 * (C + 1)), up(o_crng, chunk_rng.data(), sizeof(KeyRange) * C),
+                        up(o_kt, p->ktiles.data(), sizeof(KTile) * p->ktiles.size())};
     for (cudaError_t x : es)
         if (x != cudaSuccess) { set_cuda_error(x, "cudaMemcpy(plan tables)"); cudaFree(p->d_blob); delete p; return MOC_ERR_CUDA; }
     p->d_off = (int32_t *)(b + o_off); p->d_shot = (int32_t *)(b + o_shot); p->d_mod = (uint8_t *)(b + o_mod);
@@ -177,6 +179,7 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
     p->d_pool_unit_off = (int32_t *)(b + o_puo); p->d_pool_unit_chunk = (int32_t *)(b + o_puc);
     p->d_cap_off = (int32_t *)(b + o_cap);
     p->d_chunk_rng = (KeyRange *)(b + o_crng);
+    p->d_ktiles = (KTile *)(b + o_kt);
     *out = p;
     return MOC_OK;
 }
@@ -250,9 +253,10 @@ extern "C" int moc_attend_bwd(const moc_plan *p, const void *Q, const void *K, c
     if (p->k > 0) { if (int r = check_dev_ptrs({sel_idx}, 4)) return r; }
     if (!ws) return MOC_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return MOC_ERR_ALIGN;
-    return launch_attend_bwd_scalar(p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V,
-                                    (const __nv_bfloat16 *)O, lse, (const __nv_bfloat16 *)dO, sel_idx,
-                                    (__nv_bfloat16 *)dQ, (__nv_bfloat16 *)dK, (__nv_bfloat16 *)dV, ws, (cudaStream_t)stream);
+    auto bwd = (p->flags & MOC_FLAG_SCALAR_ATTEND) ? launch_attend_bwd_scalar : launch_attend_bwd_tc;
+    return bwd(p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, (const __nv_bfloat16 *)O, lse,
+               (const __nv_bfloat16 *)dO, sel_idx, (__nv_bfloat16 *)dQ, (__nv_bfloat16 *)dK, (__nv_bfloat16 *)dV, ws,
+               (cudaStream_t)stream);
 }
 
 extern "C" int moc_selected_pairs(const moc_plan *p, const void *ws, void *stream, int64_t *pairs) {

@@ -53,15 +53,14 @@ def test_forward_small(name):
     _forward_parity(name, scalar=False, rows_per_head=None if name != "midi2" else 400)
 
 
-@pytest.mark.parametrize("name", ["cfg0", "mini2", "mini4", "mini3"])
-def test_backward_small_scalar_kernels(name):
+def _backward_parity(name, scalar, n_rows=64):
     wl = W.workload(name)
-    run = PU.GpuRun(wl, tensors=("q", "k", "v", "do"), scalar_attend=True).forward().backward()
+    run = PU.GpuRun(wl, tensors=("q", "k", "v", "do"), scalar_attend=scalar).forward().backward()
     x = run.host_inputs()
     orc = Oracle.from_workload(wl)
     sel_gpu = run.sel.cpu().numpy()
     lay = wl.layout
-    rows = W.sample_rows(wl, 64)
+    rows = W.sample_rows(wl, n_rows)
     dQ_g = run.dQ.float().cpu().numpy()
     dK_g, dV_g = run.dK.float().cpu().numpy(), run.dV.float().cpu().numpy()
     for key_head, chunk in ((0, 0), (wl.n_heads - 1, lay.n_chunks // 2), (0, lay.n_chunks - 2)):
@@ -73,6 +72,16 @@ def test_backward_small_scalar_kernels(name):
         # not vacuous: relative L2 as well
         for g, r in ((dQ_g[rows[:, 0], rows[:, 1]], dQ), (dK_g[key_head, t0:t1], dK), (dV_g[key_head, t0:t1], dV)):
             assert np.sqrt(np.sum((g - r) ** 2) / np.sum(r ** 2)) < 2e-2
+
+
+@pytest.mark.parametrize("name", ["cfg0", "mini2", "mini4", "mini3"])
+def test_backward_small_scalar_kernels(name):
+    _backward_parity(name, scalar=True)
+
+
+@pytest.mark.parametrize("name", ["cfg0", "mini1", "mini2", "mini2t", "mini3", "mini4", "mini5", "midi2"])
+def test_backward_small(name):
+    _backward_parity(name, scalar=False, n_rows=64 if name != "midi2" else 200)
 
 
 def test_route_is_deterministic_and_lists_invert_selection():
