@@ -53,8 +53,10 @@ def test_forward_small(name):
     _forward_parity(name, scalar=False, rows_per_head=None if name != "midi2" else 400)
 
 
-def _backward_parity(name, scalar, n_rows=64):
+def _backward_parity(name, scalar, n_rows=64, heads=None):
     wl = W.workload(name)
+    if heads is not None:
+        wl.n_heads = heads
     run = PU.GpuRun(wl, tensors=("q", "k", "v", "do"), scalar_attend=scalar).forward().backward()
     x = run.host_inputs()
     orc = Oracle.from_workload(wl)
@@ -82,6 +84,12 @@ def test_backward_small_scalar_kernels(name):
 @pytest.mark.parametrize("name", ["cfg0", "mini1", "mini2", "mini2t", "mini3", "mini4", "mini5", "midi2"])
 def test_backward_small(name):
     _backward_parity(name, scalar=False, n_rows=64 if name != "midi2" else 200)
+
+
+def test_backward_benchmark_length_sampled():
+    """The single-shot clip at its full length (two heads: heads are independent): dQ on sampled rows, dK / dV
+    of the caption chunk (selected by every query), of a middle frame and of the last-but-one frame."""
+    _backward_parity("cfg1", scalar=False, n_rows=96, heads=2)
 
 
 def test_route_is_deterministic_and_lists_invert_selection():
