@@ -35,7 +35,7 @@ namespace moc {
 using namespace tc;
 
 constexpr int kRtRows = 128;          // queries per tile
-constexpr int kRtThreads = 384;
+__host__ __device__ constexpr int rt_threads(int ng) { return 64 + 128 * ng + 64; }   // producer, issuer | NG selection groups | second issuer, idle
 constexpr int kRtResident = 192;      // up to this many (padded) chunks the whole block stays resident
 constexpr int kRtBlock = 128;         // otherwise chunks are streamed in blocks of this many
 
@@ -130,15 +130,16 @@ __device__ __forceinline__ int blocks_needed(const RouteParams &p, int t) {
     return max(1, (c_hi + p.sb_rows - 1) / p.sb_rows);   // <= 64: C <= 8192, streamed blocks of 128
 }
 
-template <int D, int KMAX>
-__global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
+template <int D, int KMAX, int NG>
+__global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
                                                                  const __grid_constant__ CUtensorMap tmD,
                                                                  const RouteParams p) {
     constexpr int SUB = D / 64;
     constexpr int Q_SUB_BYTES = kRtRows * 128, Q_TILE_BYTES = SUB * Q_SUB_BYTES;
     constexpr int kMaxStages = 4;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * kMaxStages + 8];
+    constexpr int kRtThreads = rt_threads(NG);
+    __shared__ __align__(8) uint64_t bars[2 * kMaxStages + 2 + 3 * NG];
     __shared__ uint32_t tmem_slot;
     __shared__ int s_abort;
 
@@ -150,18 +151,18 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
     const uint32_t sD = sbase;
     const uint32_t sQ = sD + ((3 * SUB * d_sub_bytes + 1023) & ~1023);
     int *hist_base = reinterpret_cast<int *>(gbase + (sQ - sbase) + p.q_stages * Q_TILE_BYTES);
-    int *s_cap = hist_base + 2 * p.C;                                   // copy of cap_off[0 .. C)
+    int *s_cap = hist_base + NG * p.C;                                   // copy of cap_off[0 .. C)
     uint8_t *s_nsb = reinterpret_cast<uint8_t *>(s_cap + p.C);          // descriptor blocks needed by each of this CTA's units
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     constexpr int Q_FULL = 0, Q_EMPTY = kMaxStages, D_FULL = 2 * kMaxStages, D_EMPTY = D_FULL + 1, ACC_FULL = D_FULL + 2,
-                  ACC_EMPTY = D_FULL + 4, GROUP = D_FULL + 6;
+                  ACC_EMPTY = ACC_FULL + NG, GROUP = ACC_EMPTY + NG;
 
     if (threadIdx.x == 0) {
         s_abort = 0;
         for (int t = 0; t < kMaxStages; ++t) { mbar_init(bar(Q_FULL + t), 1); mbar_init(bar(Q_EMPTY + t), 1); }
         mbar_init(bar(D_FULL), 1);
         mbar_init(bar(D_EMPTY), 1);
-        for (int t = 0; t < 2; ++t) {
+        for (int t = 0; t < NG; ++t) {
             mbar_init(bar(ACC_FULL + t), 1);
             mbar_init(bar(ACC_EMPTY + t), 128);
             mbar_init(bar(GROUP + t), 128);
@@ -188,7 +189,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
     for (int x = threadIdx.x; x < p.C; x += kRtThreads) s_cap[x] = p.cap_off[x];
     for (int x = threadIdx.x; x < u1 - u0; x += kRtThreads) s_nsb[x] = (uint8_t)blocks_needed(p, u0 + x);
     __syncthreads();
-    constexpr int ACC_COLS = 256;   // TMEM columns per accumulator (sb_rows <= 192)
+    constexpr int ACC_COLS = 512 / NG;   // TMEM columns per accumulator (NG = 4 only with sb_rows <= 128)
     const bool resident = p.sb_rows == p.c_pad;      // one block holds every chunk: loaded once, two MMA issuers
 
     if (warp == 0) {
@@ -235,10 +236,10 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
                 if (dn > 0) mbar_wait(bar(D_FULL), (dn - 1) & 1, &dummy_flag, p.status, RW_DFULL);
             }
         }
-    } else if (warp == 1 || warp == 10) {
+    } else if (warp == 1 || warp == 2 + 4 * NG) {
         // ------------------------------------------------------------ MMA issuers
-        // With a resident descriptor block, warp 1 serves the even units and warp 10 the odd ones (each
-        // its own accumulator), so one issuer's waits and instruction overhead hide behind the other's
+        // With a resident descriptor block, warp 1 serves the even units and the last warpgroup's first warp
+        // the odd ones (each its own accumulators), so one issuer's waits and instruction overhead hide behind the other's
         // MMAs; when blocks are streamed, warp 1 serves every unit and follows the reloads.
         const int first = warp == 1 ? 0 : 1, stride = resident ? 2 : 1;
         if (lane == 0 && (warp == 1 || resident)) {
@@ -247,11 +248,14 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
             uint64_t d_term[3 * SUB];
 #pragma unroll
             for (int x = 0; x < 3 * SUB; ++x) d_term[x] = smem_desc_sw128(sD + x * d_sub_bytes, 16, 1024);
-            int res_sb = -1, dn = 0, nacc0 = 0, nacc1 = 0;
+            int res_sb = -1, dn = 0;
+            int nacc_total[NG];
+#pragma unroll
+            for (int x = 0; x < NG; ++x) nacc_total[x] = 0;
             bool ok = true;
             for (int u = u0 + first; ok && u < u1; u += stride) {
                 const int n_sb = s_nsb[u - u0];
-                const int buf = (u - u0) & 1;
+                const int buf = (u - u0) % NG;
                 const int qn = u - u0, st = qn % p.q_stages;
                 RTRACE(3000 + (u - u0) * 4 + 3);
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
@@ -266,7 +270,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
                         res_sb = sb;
                     }
                     RTRACE(3000 + (u - u0) * 4 + 0);
-                    const int uses = buf ? nacc1 : nacc0;
+                    const int uses = nacc_total[buf];
                     ok = mbar_wait(bar(ACC_EMPTY + buf), (uses & 1) ^ 1, abort_flag, p.status, RW_ACCEMPTY);
                     if (!ok) break;
                     tc_fence_after();
@@ -288,7 +292,7 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
                     }
                     tc_commit(bar(ACC_FULL + buf));
                     RTRACE(3000 + (u - u0) * 4 + 2);
-                    if (buf) ++nacc1; else ++nacc0;
+                    ++nacc_total[buf];
                     // streamed blocks: the next step, if it needs another block, may overwrite this one once
                     // these MMAs are done
                     if (!resident) {
@@ -301,9 +305,9 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
                 if (ok) tc_commit(bar(Q_EMPTY + st));
             }
         }
-    } else if (warp < 10) {
+    } else if (warp < 2 + 4 * NG) {
         // ------------------------------------------------------------ selection groups
-        const int sg = (warp - 2) >> 2;                        // group (warps 2-5, 6-9); its units are those with (u - u0) & 1 == sg
+        const int sg = (warp - 2) >> 2;                        // group (warps 2-5, 6-9, ...); its units are those with (u - u0) % NG == sg
         const int gt = threadIdx.x - 64 - sg * 128;            // thread within the group
         const int r = (warp & 3) * 32 + lane;                  // TMEM lane = query row of the tile
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
@@ -345,16 +349,16 @@ __global__ void __launch_bounds__(kRtThreads, 1) route_tc_kernel(const __grid_co
             nx_ci = i0 < p.L ? p.tok_chunk[i0] : 0;
             nx_aw = i0 < p.L ? p.anc_bits[(size_t)nx_ci * p.words] : 0u;
         }
-        for (int u = u0 + sg; ok && u < u1; u += 2) {
+        for (int u = u0 + sg; ok && u < u1; u += NG) {
             const int n_sb = s_nsb[u - u0];
             const int i = u * kRtRows + r;
             const bool live = i < p.L;
             const int ci = nx_ci;
             const uint32_t aw_next = nx_aw;
-            const int i2 = (u + 2) * kRtRows + r;
-            const bool live2 = u + 2 < u1 && i2 < p.L;
+            const int i2 = (u + NG) * kRtRows + r;
+            const bool live2 = u + NG < u1 && i2 < p.L;
             if (live2) nx_ci = p.tok_chunk[i2];       // the next unit's chunk, loaded a unit ahead (its anchor word follows below)
-            [[maybe_unused]] const int tn = 100 + sg * 1000 + ((u - u0) >> 1) * 16;
+            [[maybe_unused]] const int tn = 100 + sg * 1000 + ((u - u0) / NG) * 16;
             if (gt == 0) RTRACE(tn + 0);
             TopK<KMAX> top;
             top.init();
@@ -586,23 +590,26 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         const size_t q_tile = (size_t)kRtRows * D * 2, d_block = ((size_t)3 * a.sb_rows * D * 2 + 1023) & ~(size_t)1023;
         a.ctas_per_head = std::max(1, std::min(p->n_sm / p->H, a.tiles_per_head));
         const unsigned grid = (unsigned)(p->H * a.ctas_per_head);
-        // two histograms, the list offsets, and one byte per unit of a CTA
-        const size_t hist = 3 * sizeof(int) * (size_t)p->C + (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
+        // Four selection groups (more warps to hide the selection's latencies) when an accumulator fits
+        // a quarter of TMEM and the top-k list lives in registers; two otherwise.
+        const int ng = (a.sb_rows <= 128 && p->k <= 8) ? 4 : 2;
+        // one histogram per group, the list offsets, and one byte per unit of a CTA
+        const size_t hist = (ng + 1) * sizeof(int) * (size_t)p->C + (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
         if (d_block + q_tile + hist > budget) return MOC_ERR_SHAPE;
         a.q_stages = (int)std::min<size_t>(4, (budget - d_block - hist) / q_tile);
         const size_t smem = 1024 + d_block + a.q_stages * q_tile + hist;
         CUtensorMap tmQ, tmD;
         if (int r = make_tmap_2d_bf16(&tmQ, Q, (uint64_t)p->H * p->L, D, kRtRows)) return r;
         if (int r = make_tmap_2d_bf16(&tmD, desc3, (uint64_t)p->H * 3 * p->c_pad, D, (uint32_t)a.sb_rows)) return r;
-#define MOC_ROUTE_CASE(KM)                                                                                              \
+#define MOC_ROUTE_CASE(KM, NG)                                                                                          \
     do {                                                                                                                \
-        MOC_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel<D, KM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        route_tc_kernel<D, KM><<<grid, kRtThreads, smem, s>>>(tmQ, tmD, a);                                             \
+        MOC_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel<D, KM, NG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        route_tc_kernel<D, KM, NG><<<grid, rt_threads(NG), smem, s>>>(tmQ, tmD, a);                                     \
     } while (0)
-        if (p->k <= 4) MOC_ROUTE_CASE(4);
-        else if (p->k <= 8) MOC_ROUTE_CASE(8);
-        else if (p->k <= 64) MOC_ROUTE_CASE(64);
-        else MOC_ROUTE_CASE(512);
+        if (p->k <= 4) { if (ng == 4) MOC_ROUTE_CASE(4, 4); else MOC_ROUTE_CASE(4, 2); }
+        else if (p->k <= 8) { if (ng == 4) MOC_ROUTE_CASE(8, 4); else MOC_ROUTE_CASE(8, 2); }
+        else if (p->k <= 64) MOC_ROUTE_CASE(64, 2);
+        else MOC_ROUTE_CASE(512, 2);
 #undef MOC_ROUTE_CASE
         MOC_LAUNCH_CHECK();
     }
