@@ -123,11 +123,9 @@ struct RouteParams {
     size_t cap_total;
 };
 
-// number of descriptor blocks a tile needs: those that hold a chunk some row of the tile may pick
-__device__ __forceinline__ int blocks_needed(const RouteParams &p, int t) {
-    int c_hi = p.C;
-    if (p.causal) c_hi = p.tok_chunk[min(p.L, (t + 1) * kRtRows) - 1];   // picks are strictly earlier chunks
-    return max(1, (c_hi + p.sb_rows - 1) / p.sb_rows);   // <= 64: C <= 8192, streamed blocks of 128
+// chunks a tile can pick from: those before the chunk of its last row (causal), else all
+__device__ __forceinline__ int chunks_in_reach(const RouteParams &p, int t) {
+    return p.causal ? p.tok_chunk[min(p.L, (t + 1) * kRtRows) - 1] : p.C;
 }
 
 template <int D, int KMAX, int NG>
@@ -152,7 +150,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     const uint32_t sQ = sD + ((3 * SUB * d_sub_bytes + 1023) & ~1023);
     int *hist_base = reinterpret_cast<int *>(gbase + (sQ - sbase) + p.q_stages * Q_TILE_BYTES);
     int *s_cap = hist_base + NG * p.C;                                   // copy of cap_off[0 .. C)
-    uint8_t *s_nsb = reinterpret_cast<uint8_t *>(s_cap + p.C);          // descriptor blocks needed by each of this CTA's units
+    uint16_t *s_reach = reinterpret_cast<uint16_t *>(s_cap + p.C);      // chunks in reach of each of this CTA's units
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     constexpr int Q_FULL = 0, Q_EMPTY = kMaxStages, D_FULL = 2 * kMaxStages, D_EMPTY = D_FULL + 1, ACC_FULL = D_FULL + 2,
                   ACC_EMPTY = ACC_FULL + NG, GROUP = ACC_EMPTY + NG;
@@ -187,7 +185,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     const int u0 = (int)((long long)p.tiles_per_head * part / p.ctas_per_head);
     const int u1 = (int)((long long)p.tiles_per_head * (part + 1) / p.ctas_per_head);
     for (int x = threadIdx.x; x < p.C; x += kRtThreads) s_cap[x] = p.cap_off[x];
-    for (int x = threadIdx.x; x < u1 - u0; x += kRtThreads) s_nsb[x] = (uint8_t)blocks_needed(p, u0 + x);
+    for (int x = threadIdx.x; x < u1 - u0; x += kRtThreads) s_reach[x] = (uint16_t)chunks_in_reach(p, u0 + x);
     __syncthreads();
     constexpr int ACC_COLS = 512 / NG;   // TMEM columns per accumulator (NG = 4 only with sb_rows <= 128)
     const bool resident = p.sb_rows == p.c_pad;      // one block holds every chunk: loaded once, two MMA issuers
@@ -200,7 +198,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             int res_sb = -1, qn = 0, dn = 0;
             bool ok = true;
             for (int u = u0; ok && u < u1; ++u) {
-                const int n_sb = s_nsb[u - u0];
+                const int reach = s_reach[u - u0], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
                     if (sb == 0) {
                         const int st = qn % p.q_stages;
@@ -254,7 +252,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             for (int x = 0; x < NG; ++x) nacc_total[x] = 0;
             bool ok = true;
             for (int u = u0 + first; ok && u < u1; u += stride) {
-                const int n_sb = s_nsb[u - u0];
+                const int reach = s_reach[u - u0], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
                 const int buf = (u - u0) % NG;
                 const int qn = u - u0, st = qn % p.q_stages;
                 RTRACE(3000 + (u - u0) * 4 + 3);
@@ -275,7 +273,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                     if (!ok) break;
                     tc_fence_after();
                     RTRACE(3000 + (u - u0) * 4 + 1);
-                    const int rows_sb = min(p.sb_rows, p.c_pad - sb * p.sb_rows);
+                    const int rows_sb = max(16, min(min(p.sb_rows, p.c_pad - sb * p.sb_rows), (reach - sb * p.sb_rows + 15) & ~15));
                     const uint64_t qd = q_desc0 + (uint64_t)(st * (Q_TILE_BYTES >> 4));
                     for (int n0 = 0; n0 < rows_sb; n0 += 128) {
                         const int n = min(128, rows_sb - n0);
@@ -350,7 +348,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             nx_aw = i0 < p.L ? p.anc_bits[(size_t)nx_ci * p.words] : 0u;
         }
         for (int u = u0 + sg; ok && u < u1; u += NG) {
-            const int n_sb = s_nsb[u - u0];
+            const int reach = s_reach[u - u0], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
             const int i = u * kRtRows + r;
             const bool live = i < p.L;
             const int ci = nx_ci;
@@ -370,7 +368,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 ++nacc;
                 if (gt == 0) RTRACE(tn + 1);
                 tc_fence_after();
-                const int rows_sb = min(p.sb_rows, p.c_pad - sb * p.sb_rows);
+                const int rows_sb = max(16, min(min(p.sb_rows, p.c_pad - sb * p.sb_rows), (reach - sb * p.sb_rows + 15) & ~15));
                 for (int cc = 0; cc < rows_sb; cc += 32) {
                     uint32_t v[32];
                     tmem_ld32(acc + cc, v);
@@ -594,7 +592,7 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         // a quarter of TMEM and the top-k list lives in registers; two otherwise.
         const int ng = (a.sb_rows <= 128 && p->k <= 8) ? 4 : 2;
         // one histogram per group, the list offsets, and one byte per unit of a CTA
-        const size_t hist = (ng + 1) * sizeof(int) * (size_t)p->C + (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
+        const size_t hist = (ng + 1) * sizeof(int) * (size_t)p->C + 2 * (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
         if (d_block + q_tile + hist > budget) return MOC_ERR_SHAPE;
         a.q_stages = (int)std::min<size_t>(4, (budget - d_block - hist) / q_tile);
         const size_t smem = 1024 + d_block + a.q_stages * q_tile + hist;
