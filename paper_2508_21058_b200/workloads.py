@@ -149,6 +149,10 @@ def workload(name: str, seed: int = 0) -> Workload:
     if name == "mini5":   # non-causal single-shot variant: chunk 256, k=3, self + prompt
         return Workload(name, 2, 64, make_layout(1, 77, 1, 1500, chunk_len=256), 3, 0, 0,
                         causal=False, seed=seed)
+    if name == "mini6":   # many small chunks, k beyond the register-resident top-k list (k = 12)
+        return Workload(name, 2, 128, make_layout(3, 16, 40, 24), 12, 1, 1, seed=seed)
+    if name == "mini7":   # k = 70 of up to 122 candidates, d = 64: the long-list selection path, streamed descriptor blocks
+        return Workload(name, 2, 64, make_layout(3, 16, 80, 16), 70, 1, 1, seed=seed)
     if name == "midi2":   # multi-shot with true 1560-token frames, small enough for a full oracle pass
         return Workload(name, 2, 128, make_layout(2, 256, 4, 1560), 3, 1, 1, seed=seed)
     raise KeyError(name)
