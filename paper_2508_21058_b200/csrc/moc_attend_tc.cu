@@ -38,7 +38,7 @@ using namespace tc;
 // clock64() into a slot of g_trace, read back with moc_trace_read().  Compiled out otherwise.
 #ifdef MOC_TRACE
 __device__ long long g_trace[8192];
-#define TRACE_CTA (blockIdx.x == (ROUTED ? 5000 : 1000) && (ROUTED || blockIdx.y == 3))
+#define TRACE_CTA (blockIdx.x == (ROUTED ? 5000 : 70) && (ROUTED || blockIdx.y == 3))
 #define TRACE(slot) do { if (TRACE_CTA) g_trace[(slot)] = clock64(); } while (0)
 #else
 #define TRACE(slot) ((void)0)
@@ -291,25 +291,44 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             }
             // ---- epilogue
             if (r == 0) TRACE(12 + g);
+            // The merge weights of the routed partials depend only on log-sum-exps: have them ready before
+            // the last P V lands.  wslot[s] = exp(lse_s - lse_total), w_own likewise for this pass's own part.
+            const float inv_l = 1.f / l_run;
+            const float lse_own = (m_run + log2f(l_run)) * kLn2;
+            float w_own = inv_l, big = lse_own, wsum = 1.f;
+            constexpr int KW = 8;                     // slots whose weights live in registers
+            float wslot[KW];
+#pragma unroll
+            for (int s = 0; s < KW; ++s) wslot[s] = 0.f;
+            const float *pl = nullptr;
+            const __nv_bfloat16 *po = nullptr;
+            if (!ROUTED && ok && qi >= 0 && p.k > 0) {
+                pl = p.part_lse + ((size_t)h * p.L + qi) * p.k;
+                po = p.part_o + ((size_t)h * p.L + qi) * p.k * D;
+                if (p.k <= KW) {
+                    float plv[KW];
+#pragma unroll
+                    for (int s = 0; s < KW; ++s) plv[s] = s < p.k ? pl[s] : -INFINITY;
+#pragma unroll
+                    for (int s = 0; s < KW; ++s) big = fmaxf(big, plv[s]);
+                    wsum = __expf(lse_own - big);
+#pragma unroll
+                    for (int s = 0; s < KW; ++s) { wslot[s] = __expf(plv[s] - big); wsum += wslot[s]; }     // exp(-inf) = 0: empty slot
+#pragma unroll
+                    for (int s = 0; s < KW; ++s) wslot[s] /= wsum;
+                } else {
+                    for (int s = 0; s < p.k; ++s) big = fmaxf(big, pl[s]);
+                    wsum = __expf(lse_own - big);
+                    for (int s = 0; s < p.k; ++s) wsum += __expf(pl[s] - big);
+                }
+                w_own = __expf(lse_own - big) / wsum * inv_l;
+            }
             if (ok) {
                 ok = mbar_wait(bar(O_FULL + g), 0, abort_flag, p.status, W_OFULL);
                 ok = __all_sync(0xffffffffu, ok);
             }
             if (ok) {
                 tc_fence_after();
-                const float inv_l = 1.f / l_run;
-                const float lse_own = (m_run + log2f(l_run)) * kLn2;
-                float w_own = inv_l, big = lse_own, wsum = 1.f;
-                const float *pl = nullptr;
-                const __nv_bfloat16 *po = nullptr;
-                if (!ROUTED && qi >= 0 && p.k > 0) {
-                    pl = p.part_lse + ((size_t)h * p.L + qi) * p.k;
-                    po = p.part_o + ((size_t)h * p.L + qi) * p.k * D;
-                    for (int s = 0; s < p.k; ++s) big = fmaxf(big, pl[s]);
-                    wsum = __expf(lse_own - big);
-                    for (int s = 0; s < p.k; ++s) wsum += __expf(pl[s] - big);
-                    w_own = __expf(lse_own - big) / wsum * inv_l;
-                }
 #pragma unroll 1
                 for (int ch = 0; ch < D / 32; ++ch) {
                     uint32_t v[32];
@@ -319,7 +338,35 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                     float acc[32];
 #pragma unroll
                     for (int x = 0; x < 32; ++x) acc[x] = __uint_as_float(v[x]) * w_own;
-                    if (pl) {
+                    if (pl && p.k <= KW) {
+                        // four slots' pieces of this column block are requested together: one round trip, not four
+#pragma unroll
+                        for (int s0 = 0; s0 < KW; s0 += 4) {
+                            if (s0 >= p.k) break;
+                            uint4 raw[4][4];
+#pragma unroll
+                            for (int s = 0; s < 4; ++s)
+#pragma unroll
+                                for (int q4 = 0; q4 < 4; ++q4)
+                                    raw[s][q4] = (s0 + s < p.k && wslot[s0 + s] != 0.f)
+                                                     ? __ldcg(reinterpret_cast<const uint4 *>(po + (size_t)(s0 + s) * D + ch * 32) + q4)
+                                                     : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                            for (int s = 0; s < 4; ++s) {
+                                const float w = wslot[s0 + s];
+#pragma unroll
+                                for (int q4 = 0; q4 < 4; ++q4) {
+                                    const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&raw[s][q4]);
+#pragma unroll
+                                    for (int y = 0; y < 4; ++y) {
+                                        const float2 f = __bfloat1622float2(b[y]);
+                                        acc[q4 * 8 + 2 * y] = fmaf(w, f.x, acc[q4 * 8 + 2 * y]);
+                                        acc[q4 * 8 + 2 * y + 1] = fmaf(w, f.y, acc[q4 * 8 + 2 * y + 1]);
+                                    }
+                                }
+                            }
+                        }
+                    } else if (pl) {
                         for (int s = 0; s < p.k; ++s) {
                             const float ls = pl[s];
                             if (ls == -INFINITY) continue;
