@@ -19,8 +19,9 @@
 //                 keep a sorted top-k in registers, then write sel_idx and append the picks
 //                 to the per-(head, chunk) query lists (tile-local ranks from a shared-memory
 //                 histogram, one global atomic per (tile, chunk) to reserve the range).
-//   The head's descriptor block stays in shared memory for the CTA's lifetime (C <= 192);
-//   with more chunks it is streamed in blocks of 128 and warp 1 alone issues.
+//   The head's descriptors stay in shared memory for the CTA's lifetime (C <= 192) and are scored
+//   in steps of at most 128 chunks; with more chunks they are streamed in blocks of 128 and warp 1
+//   alone issues.
 // route_tiles_kernel  running count of attention tiles over (head, chunk) from the pick counts;
 // route_items_kernel  the routed attention work items (one per 256 picks of a chunk).
 // Every mbarrier wait is bounded; a wait that runs out flags the workspace status word.
@@ -118,7 +119,8 @@ struct RouteParams {
     int H, L, C, c_pad, k, words, causal;
     int tiles_per_head;     // ceil(L / 128)
     int ctas_per_head;      // the grid is H * ctas_per_head
-    int sb_rows;            // chunks per descriptor block held in shared memory
+    int sb_rows;            // chunks per scoring step (one accumulator's worth)
+    int d_rows;             // descriptor rows per term held in shared memory: c_pad (resident) or sb_rows (streamed)
     int q_stages;
     size_t cap_total;
 };
@@ -144,8 +146,8 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gbase = smem_raw + (sbase - smem_u32(smem_raw));
-    // shared memory: descriptor block (3 terms x SUB sub-tiles of sb_rows x 128 bytes) | Q stages | two histograms
-    const int d_sub_bytes = p.sb_rows * 128;
+    // shared memory: descriptor block (3 terms x SUB sub-tiles of d_rows x 128 bytes) | Q stages | histograms
+    const int d_sub_bytes = p.d_rows * 128;
     const uint32_t sD = sbase;
     const uint32_t sQ = sD + ((3 * SUB * d_sub_bytes + 1023) & ~1023);
     int *hist_base = reinterpret_cast<int *>(gbase + (sQ - sbase) + p.q_stages * Q_TILE_BYTES);
@@ -188,7 +190,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     for (int x = threadIdx.x; x < u1 - u0; x += kRtThreads) s_reach[x] = (uint16_t)chunks_in_reach(p, u0 + x);
     __syncthreads();
     constexpr int ACC_COLS = 512 / NG;   // TMEM columns per accumulator (NG = 4 only with sb_rows <= 128)
-    const bool resident = p.sb_rows == p.c_pad;      // one block holds every chunk: loaded once, two MMA issuers
+    const bool resident = p.d_rows == p.c_pad;       // every chunk's descriptor is held: loaded once, two MMA issuers
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -210,7 +212,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                             tma_load_2d(sQ + st * Q_TILE_BYTES + sub * Q_SUB_BYTES, &tmQ, sub * 64, h * p.L + u * kRtRows, bar(Q_FULL + st));
                         ++qn;
                     }
-                    if (sb != res_sb) {
+                    if (resident ? dn == 0 : sb != res_sb) {
                         ok = mbar_wait(bar(D_EMPTY), (dn & 1) ^ 1, abort_flag, p.status, RW_DEMPTY);
                         if (!ok) break;
                         mbar_expect_tx(bar(D_FULL), 3 * SUB * d_sub_bytes);
@@ -218,7 +220,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
 #pragma unroll
                             for (int sub = 0; sub < SUB; ++sub)
                                 tma_load_2d(sD + (term * SUB + sub) * d_sub_bytes, &tmD, sub * 64,
-                                            (h * 3 + term) * p.c_pad + sb * p.sb_rows, bar(D_FULL));
+                                            (h * 3 + term) * p.c_pad + (resident ? 0 : sb * p.sb_rows), bar(D_FULL));
                         ++dn;
                         res_sb = sb;
                     }
@@ -261,7 +263,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                         ok = mbar_wait(bar(Q_FULL + st), (qn / p.q_stages) & 1, abort_flag, p.status, RW_QFULL);
                         if (!ok) break;
                     }
-                    if (sb != res_sb) {
+                    if (resident ? dn == 0 : sb != res_sb) {
                         ok = mbar_wait(bar(D_FULL), dn & 1, abort_flag, p.status, RW_DFULL);
                         if (!ok) break;
                         ++dn;
@@ -279,7 +281,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                         const int n = min(128, rows_sb - n0);
                         const uint32_t idesc = idesc_bf16_f32(128, n, 0, 0);
                         const uint32_t acc = tmem + buf * ACC_COLS + n0;
-                        const uint32_t nofs = (uint32_t)(n0 * 128) >> 4;
+                        const uint32_t nofs = (uint32_t)(((resident ? sb * p.sb_rows : 0) + n0) * 128) >> 4;
 #pragma unroll
                         for (int term = 0; term < 3; ++term) {
 #pragma unroll
@@ -583,9 +585,10 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         a.H = p->H; a.L = p->L; a.C = p->C; a.c_pad = p->c_pad; a.k = p->k; a.words = p->words;
         a.causal = (p->flags & MOC_FLAG_CAUSAL) ? 1 : 0;
         a.tiles_per_head = (p->L + kRtRows - 1) / kRtRows;
-        a.sb_rows = p->c_pad <= kRtResident ? p->c_pad : kRtBlock;
+        a.d_rows = p->c_pad <= kRtResident ? p->c_pad : kRtBlock;
+        a.sb_rows = std::min(a.d_rows, kRtBlock);     // steps of at most 128 chunks: an accumulator is a quarter of TMEM
         a.cap_total = (size_t)p->cap_off[p->C];
-        const size_t q_tile = (size_t)kRtRows * D * 2, d_block = ((size_t)3 * a.sb_rows * D * 2 + 1023) & ~(size_t)1023;
+        const size_t q_tile = (size_t)kRtRows * D * 2, d_block = ((size_t)3 * a.d_rows * D * 2 + 1023) & ~(size_t)1023;
         a.ctas_per_head = std::max(1, std::min(p->n_sm / p->H, a.tiles_per_head));
         const unsigned grid = (unsigned)(p->H * a.ctas_per_head);
         // Four selection groups (more warps to hide the selection's latencies) when an accumulator fits
@@ -598,7 +601,7 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         const size_t smem = 1024 + d_block + a.q_stages * q_tile + hist;
         CUtensorMap tmQ, tmD;
         if (int r = make_tmap_2d_bf16(&tmQ, Q, (uint64_t)p->H * p->L, D, kRtRows)) return r;
-        if (int r = make_tmap_2d_bf16(&tmD, desc3, (uint64_t)p->H * 3 * p->c_pad, D, (uint32_t)a.sb_rows)) return r;
+        if (int r = make_tmap_2d_bf16(&tmD, desc3, (uint64_t)p->H * 3 * p->c_pad, D, (uint32_t)a.d_rows)) return r;
 #define MOC_ROUTE_CASE(KM, NG)                                                                                          \
     do {                                                                                                                \
         MOC_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel<D, KM, NG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
