@@ -117,8 +117,11 @@ int moc_chunk_pool_noalloc(const moc_plan *plan, const void *K, float *desc, voi
 /* Steps 2-5 - routing (Eq. 3; Sec. 3.2 causal mask and fixed selections; Sec. 3.3 forced
  * links before top-k).  For every query i in chunk c(i): candidates are the chunks that
  * are not anchors of c(i) and (causal) lie strictly before c(i); score = q_i . desc_j (raw
- * dot product, fp32); sel_idx gets the min(k, #candidates) best, ties to the lower index.
- * Also rebuilds, in ws, the per-(head, chunk) lists of the queries that picked it. */
+ * dot product: each fp32 descriptor enters as the exact sum of three bf16 terms, products are
+ * exact and the accumulation is fp32); sel_idx gets the min(k, #candidates) best, ties to the
+ * lower index.  Also rebuilds, in ws, the per-(head, chunk) lists of the queries that picked
+ * it and the routed work items of moc_attend / moc_attend_bwd.  MOC_ERR_SHAPE if the chunk
+ * count is beyond what the kernel's shared-memory tables hold (about 8000 chunks). */
 int moc_route(const moc_plan *plan, const void *Q, const float *desc, int32_t *sel_idx, void *ws, void *stream);
 
 /* Step 6 - sparse attention (Eq. 2): O_i = softmax(scale q_i K_Omega^T) V_Omega over the
@@ -129,7 +132,9 @@ int moc_attend(const moc_plan *plan, const void *Q, const void *K, const void *V
 
 /* Backward of step 6 with the selection held constant (Sec. 3.1: top-k is not
  * differentiated, gradients reach Q, K, V only through the attention over selected
- * chunks; none flows through the descriptors or scores).  Needs with_bwd workspace. */
+ * chunks; none flows through the descriptors or scores).  bf16 products (P and dS are rounded
+ * to bf16 before their contractions), fp32 accumulation.  Needs with_bwd workspace, written by
+ * moc_route and moc_attend for the same inputs; overwrites the forward's routed partials. */
 int moc_attend_bwd(const moc_plan *plan, const void *Q, const void *K, const void *V, const void *O,
                    const float *lse, const void *dO, const int32_t *sel_idx, void *dQ, void *dK, void *dV,
                    void *ws, void *stream);
