@@ -5,9 +5,9 @@
 // dS = P (dP - delta_i);  dV_t += P dO_i,  dK_t += scale dS q_i,  dQ_i += scale dS k_t.
 //
 // One kernel, three modes, one tile engine.  A CTA holds a STATIONARY pair of 128-row tiles
-// (X1, X2) in shared memory and streams pairs of 128-row tiles (Y1, Y2) through two stages:
-//     T1 = X1 Y1^T,  T2 = X2 Y2^T        (two MMAs, both operands from shared memory, into TMEM)
-//     threads (one TMEM lane each) turn (T1, T2) into P and dS, written back to TMEM as bf16
+// (X1, X2) in shared memory and streams pairs of 128-row tiles (Y1, Y2) through three and two stages:
+//     T1 = X1 Y1^T,  T2 = X2 Y2^T        (both operands from shared memory, into TMEM)
+//     threads (one TMEM lane each) turn T1 into P, then (P, T2) into dS, written back to TMEM as bf16
 //     ACC1 += dS Y1,  ACC2 += P Y2       (A from TMEM, B the streamed tile as an MN-major operand)
 //   dQ modes (query stationary, the forward's work items, 128 rows per CTA):  X = (Q, dO) rows of
 //     the item, Y = (K, V) tiles of its key ranges by TMA; lse and delta belong to the lane;
@@ -15,10 +15,15 @@
 //     workspace; the anchor mode adds them to its own part and writes dQ.
 //   dK/dV mode (key stationary, one CTA per 128 keys of a chunk):  X = (K, V) rows of the key
 //     tile by TMA, Y = (Q, dO) rows of every query that attends to the chunk - the query rows of
-//     the chunks that have it as an anchor, then the chunk's routed query list - copied by the
-//     producer warp with 16-byte asynchronous copies; lse and delta belong to the column; ACC1 is
+//     the chunks that have it as an anchor, then the chunk's routed query list - copied by four
+//     producer warps with 16-byte asynchronous copies; lse and delta belong to the column; ACC1 is
 //     dK, ACC2 is dV.  Each key tile is owned by one CTA: no atomics, no partial sums.
-// 6 warps: 0-3 the lane threads, 4 the producer, 5 the MMA issuer.  Every mbarrier wait is
+// The tensor pipe and the lanes overlap across tiles.  dK/dV: the issue order is ACC2(j), T1(j+1),
+// ACC1(j), T2(j+1), so that while the lanes form P(j+1) the pipe runs ACC1(j) and T2(j+1), and T1 / T2
+// are rewritten only after the contraction that reads the P / dS stored over them.  dQ: no ACC2, so
+// its columns serve as a second T1 and T1(j+2) is issued as soon as the lanes have finished tile j.
+// 12 warps: 0-3 the lane threads, 4-7 the producers, 8 the MMA issuer, 9-11 idle (they complete the
+// third warpgroup, whose registers go to the lanes).  Every mbarrier wait is
 // bounded; a wait that runs out flags the workspace status word and the CTA drains and leaves.
 #include <algorithm>
 
@@ -30,7 +35,7 @@ namespace moc {
 using namespace tc;
 
 enum BwdMode { DQ_ROUTED = 0, DQ_ANCHOR = 1, DKV = 2 };
-enum BwdWait { BW_XFULL = 64, BW_YFULL, BW_YEMPTY, BW_TFULL, BW_DFULL, BW_ACCFULL };
+enum BwdWait { BW_XFULL = 64, BW_YFULL, BW_YEMPTY, BW_T1FULL, BW_T2FULL, BW_PDONE, BW_DSDONE, BW_ACCFULL, BW_SMEM };
 
 struct BwdParams {
     const __nv_bfloat16 *Q, *K, *V, *dO;
@@ -51,7 +56,8 @@ struct BwdParams {
     float scale, scale_log2;
 };
 
-constexpr int kBwdThreads = 192;
+constexpr int kY1Stages = 3, kY2Stages = 2;   // stages of the streamed tiles Y1 (read twice per tile) and Y2
+constexpr int kBwdThreads = 384;
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D, int MODE>
@@ -62,26 +68,36 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
     constexpr int SUB = D / 64;
     constexpr int SUB_BYTES = 128 * 128;
     constexpr int CH = D / 8;               // 16-byte pieces per row
-    extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[10];
+    constexpr int N_TILES_SMEM = 2 + kY1Stages + kY2Stages;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bars[18];
     __shared__ uint32_t tmem_slot;
     __shared__ int s_abort;
     __shared__ int w_valid, w_h, w_rows, w_first, w_nrng, w_ntiles, w_chunk, w_t0;
     __shared__ const KeyRange *w_rng;
-    __shared__ int s_row[2][128];           // query row behind each row of the staged tile (-1 = none)
-    __shared__ float s_lse[2][128], s_del[2][128];   // dK/dV mode: per streamed query, lse * log2(e) and delta
+    // dK/dV mode: per streamed query, (lse * log2(e), delta), for tiles j and j + 1;
+    // dQ modes: the first 128 words hold the item's query rows while they are staged
+    __shared__ __align__(8) float s_ld[2][2][128];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gbase = smem_raw + (sbase - smem_u32(smem_raw));
-    // shared tiles: X1 X2 | Y1 stage 0,1 | Y2 stage 0,1
-    const uint32_t sX = sbase, sY1 = sbase + 2 * TILE_BYTES, sY2 = sbase + 4 * TILE_BYTES;
+    // shared tiles: X1 X2 | Y1 stages | Y2 stages
+    const uint32_t sX = sbase, sY1 = sbase + 2 * TILE_BYTES, sY2 = sbase + (2 + kY1Stages) * TILE_BYTES;
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
-    constexpr int X_FULL = 0, Y_FULL = 1, Y_EMPTY = 3, T_FULL = 5, D_FULL = 6, ACC_FULL = 7;
+    constexpr int X_FULL = 0, Y1_FULL = 1, Y1_EMPTY = 4, Y2_FULL = 7, Y2_EMPTY = 9, T1_FULL = 11, T2_FULL = 13,
+                  P_DONE = 14, DS_DONE = 15, ACC_FULL = 17;
 
     if (threadIdx.x == 0) {
         s_abort = 0;
         int valid = (*(volatile int *)p.status == 0);
+        uint32_t dyn_bytes;
+        asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_bytes));
+        if (valid && (sbase - smem_u32(smem_raw)) + (uint32_t)N_TILES_SMEM * TILE_BYTES > dyn_bytes) {
+            // the launch gave less shared memory than the tiles need: report, touch nothing
+            if (atomicCAS(p.status, 0, MOC_ERR_TIMEOUT) == 0) p.status[1] = BW_SMEM;
+            valid = 0;
+        }
         if (MODE != DKV) {
             const int item = blockIdx.x >> 1, half = blockIdx.x & 1;
             if (MODE == DQ_ROUTED && valid && item >= *p.n_items_dev) valid = 0;
@@ -114,12 +130,18 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
         }
         w_valid = valid;
         mbar_init(bar(X_FULL), MODE == DKV ? 1 : 128);
-        for (int t = 0; t < 2; ++t) {
-            mbar_init(bar(Y_FULL + t), MODE == DKV ? 32 : 1);
-            mbar_init(bar(Y_EMPTY + t), 1);
+        for (int t = 0; t < kY1Stages; ++t) {
+            mbar_init(bar(Y1_FULL + t), MODE == DKV ? 128 : 1);
+            mbar_init(bar(Y1_EMPTY + t), 1);
         }
-        mbar_init(bar(T_FULL), 1);
-        mbar_init(bar(D_FULL), 128);
+        for (int t = 0; t < kY2Stages; ++t) {
+            mbar_init(bar(Y2_FULL + t), MODE == DKV ? 128 : 1);
+            mbar_init(bar(Y2_EMPTY + t), 1);
+            mbar_init(bar(T1_FULL + t), 1);
+            mbar_init(bar(DS_DONE + t), 128);
+        }
+        mbar_init(bar(T2_FULL), 1);
+        mbar_init(bar(P_DONE), 128);
         mbar_init(bar(ACC_FULL), 1);
         fence_barrier_init();
     }
@@ -133,12 +155,17 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
     __syncthreads();
     tc_fence_after();
 
-    const uint32_t tmem = tmem_slot;      // T1 [0,128)  T2 [128,256)  ACC1 [256,384)  ACC2 [384,512)
+    // TMEM columns: T1 [0,128)  T2 [128,256)  ACC1 [256,384)  ACC2 [384,512); the dQ modes have no ACC2
+    // and use its columns as a second T1, for the odd tiles
+    const uint32_t tmem = tmem_slot;
     const int h = w_h, rows = w_rows, n_tiles = w_ntiles;
     volatile int *abort_flag = &s_abort;
 
     if (warp < 4) {
         // ------------------------------------------------------------ lane threads
+        // a thread keeps the 128 P values of its row between the two halves of a tile: it takes the
+        // registers that the other two warpgroups give up
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         const int r = threadIdx.x;                    // row of the stationary tile = TMEM lane
         const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
         int qi = -1, slot = 0;
@@ -156,7 +183,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 dlt = p.delta[(size_t)h * p.L + qi];
             }
             // stage the item's Q and dO rows together: consecutive threads take consecutive 16-byte pieces
-            s_row[0][r] = qi;
+            int *s_row = reinterpret_cast<int *>(&s_ld[0][0][0]);
+            s_row[r] = qi;
             asm volatile("bar.sync 1, 128;" ::: "memory");
             constexpr int RP = 128 / CH;
             const int c16 = r % CH;
@@ -167,7 +195,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 uint4 v[CH];
 #pragma unroll
                 for (int ps = 0; ps < CH; ++ps) {
-                    const int rr = ps * RP + r / CH, q = s_row[0][rr];
+                    const int rr = ps * RP + r / CH, q = s_row[rr];
                     v[ps] = make_uint4(0, 0, 0, 0);
                     if (q >= 0) v[ps] = __ldg(reinterpret_cast<const uint4 *>(src + ((size_t)h * p.L + q) * D) + c16);
                 }
@@ -180,45 +208,77 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
         const float c = p.scale_log2;
         TileIter it(w_rng, MODE == DKV ? 0 : w_nrng);
         bool ok = true;
+        int s3 = 0, ph3 = 0;                          // Y1 stage of tile jt and its phase
         for (int jt = 0; jt < n_tiles; ++jt) {
             const int st = jt & 1;
             int valid = 128, t0;
             if (MODE != DKV) it.next(t0, valid);
-            ok = mbar_wait(bar(T_FULL), jt & 1, abort_flag, p.status, BW_TFULL);
-            if (MODE == DKV) ok = ok && mbar_wait(bar(Y_FULL + st), (jt >> 1) & 1, abort_flag, p.status, BW_YFULL);
+            ok = mbar_wait(bar(T1_FULL + st), (jt >> 1) & 1, abort_flag, p.status, BW_T1FULL);
+            if (MODE == DKV) ok = ok && mbar_wait(bar(Y1_FULL + s3), ph3, abort_flag, p.status, BW_YFULL);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-#pragma unroll 1
+            // ---- P = exp2(scale log2(e) S - lse log2(e)) from T1
+            const uint32_t t1 = (MODE != DKV && st) ? 384u : 0u;
+            float pv[128];
+#pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
-                uint32_t s[32], dp[32];
-                tmem_ld32(tmem + lane_off + ch * 32, s);
-                tmem_ld32(tmem + lane_off + 128 + ch * 32, dp);
+                uint32_t s[32];
+                tmem_ld32(tmem + lane_off + t1 + ch * 32, s);
                 tmem_wait_ld();
-                uint32_t ups[16], uds[16];
 #pragma unroll
                 for (int x = 0; x < 32; x += 2) {
-                    float l0 = lse2, l1 = lse2, d0 = dlt, d1 = dlt;
+                    float l0 = lse2, l1 = lse2;
                     if (MODE == DKV) {
-                        const float2 l = *reinterpret_cast<const float2 *>(&s_lse[st][ch * 32 + x]);
-                        const float2 d = *reinterpret_cast<const float2 *>(&s_del[st][ch * 32 + x]);
-                        l0 = l.x; l1 = l.y; d0 = d.x; d1 = d.y;
+                        const float2 l = *reinterpret_cast<const float2 *>(&s_ld[st][0][ch * 32 + x]);
+                        l0 = l.x; l1 = l.y;
                     }
                     float p0 = ex2(fmaf(__uint_as_float(s[x]), c, -l0)), p1 = ex2(fmaf(__uint_as_float(s[x + 1]), c, -l1));
                     if (MODE != DKV) {
                         if (ch * 32 + x >= valid) p0 = 0.f;
                         if (ch * 32 + x + 1 >= valid) p1 = 0.f;
                     }
-                    const float ds0 = p0 * (__uint_as_float(dp[x]) - d0), ds1 = p1 * (__uint_as_float(dp[x + 1]) - d1);
-                    ups[x >> 1] = bf16x2(p0, p1);
-                    uds[x >> 1] = bf16x2(ds0, ds1);
+                    pv[ch * 32 + x] = p0;
+                    pv[ch * 32 + x + 1] = p1;
                 }
-                tmem_st16(tmem + lane_off + 128 + ch * 16, uds);          // dS over the T2 columns already read
-                if (MODE == DKV) tmem_st16(tmem + lane_off + ch * 16, ups);   // P over the T1 columns already read
+                if (MODE == DKV) {                                        // P over the T1 columns already read
+                    uint32_t ups[16];
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) ups[x] = bf16x2(pv[ch * 32 + 2 * x], pv[ch * 32 + 2 * x + 1]);
+                    tmem_st16(tmem + lane_off + ch * 16, ups);
+                }
+            }
+            if (MODE == DKV) {
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(P_DONE));
+            }
+            // ---- dS = P (dP - delta) from T2, written over the T2 columns already read
+            ok = mbar_wait(bar(T2_FULL), jt & 1, abort_flag, p.status, BW_T2FULL);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t dp[32], uds[16];
+                tmem_ld32(tmem + lane_off + 128 + ch * 32, dp);
+                tmem_wait_ld();
+#pragma unroll
+                for (int x = 0; x < 32; x += 2) {
+                    float d0 = dlt, d1 = dlt;
+                    if (MODE == DKV) {
+                        const float2 d = *reinterpret_cast<const float2 *>(&s_ld[st][1][ch * 32 + x]);
+                        d0 = d.x; d1 = d.y;
+                    }
+                    uds[x >> 1] = bf16x2(pv[ch * 32 + x] * (__uint_as_float(dp[x]) - d0),
+                                         pv[ch * 32 + x + 1] * (__uint_as_float(dp[x + 1]) - d1));
+                }
+                tmem_st16(tmem + lane_off + 128 + ch * 16, uds);
             }
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bar(D_FULL));
+            mbar_arrive(bar(DS_DONE + st));
+            if (++s3 == kY1Stages) { s3 = 0; ph3 ^= 1; }
         }
         // ---- epilogue
         if (ok) {
@@ -280,34 +340,42 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 }
             }
         }
-    } else if (warp == 4) {
-        // ------------------------------------------------------------ producer
+    } else if (warp < 8) {
+        // ------------------------------------------------------------ producers
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
         if (MODE != DKV) {
-            if (lane == 0) {
+            if (warp == 4 && lane == 0) {
                 prefetch_tensormap(&tmK);
                 prefetch_tensormap(&tmV);
                 TileIter it(w_rng, w_nrng);
-                int t0, valid, jt = 0;
+                int t0, valid, jt = 0, s3 = 0, ph3 = 0, n_k = 0;      // jt counts the V copies issued, n_k the K copies
                 while (it.next(t0, valid)) {
-                    const int st = jt & 1;
-                    if (!mbar_wait(bar(Y_EMPTY + st), ((jt >> 1) & 1) ^ 1, abort_flag, p.status, BW_YEMPTY)) break;
-                    mbar_expect_tx(bar(Y_FULL + st), 2 * TILE_BYTES);
+                    const int s2 = jt & 1;
+                    if (!mbar_wait(bar(Y1_EMPTY + s3), ph3 ^ 1, abort_flag, p.status, BW_YEMPTY)) break;
+                    mbar_expect_tx(bar(Y1_FULL + s3), TILE_BYTES);
 #pragma unroll
-                    for (int sub = 0; sub < SUB; ++sub) {
-                        tma_load_2d(sY1 + st * TILE_BYTES + sub * SUB_BYTES, &tmK, sub * 64, h * p.L + t0, bar(Y_FULL + st));
-                        tma_load_2d(sY2 + st * TILE_BYTES + sub * SUB_BYTES, &tmV, sub * 64, h * p.L + t0, bar(Y_FULL + st));
-                    }
+                    for (int sub = 0; sub < SUB; ++sub)
+                        tma_load_2d(sY1 + s3 * TILE_BYTES + sub * SUB_BYTES, &tmK, sub * 64, h * p.L + t0, bar(Y1_FULL + s3));
+                    ++n_k;
+                    if (!mbar_wait(bar(Y2_EMPTY + s2), ((jt >> 1) & 1) ^ 1, abort_flag, p.status, BW_YEMPTY)) break;
+                    mbar_expect_tx(bar(Y2_FULL + s2), TILE_BYTES);
+#pragma unroll
+                    for (int sub = 0; sub < SUB; ++sub)
+                        tma_load_2d(sY2 + s2 * TILE_BYTES + sub * SUB_BYTES, &tmV, sub * 64, h * p.L + t0, bar(Y2_FULL + s2));
                     ++jt;
+                    if (++s3 == kY1Stages) { s3 = 0; ph3 ^= 1; }
                 }
                 if (*abort_flag) {      // copies already issued must land before the shared memory is released
                     int dummy_flag = 0;
-                    for (int b = 1; b <= 2; ++b)
-                        if (jt - b >= 0) mbar_wait(bar(Y_FULL + ((jt - b) & 1)), ((jt - b) >> 1) & 1, &dummy_flag, p.status, BW_YFULL);
+                    for (int b = 1; b <= kY1Stages; ++b)
+                        if (n_k - b >= 0) mbar_wait(bar(Y1_FULL + ((n_k - b) % kY1Stages)), ((n_k - b) / kY1Stages) & 1, &dummy_flag, p.status, BW_YFULL);
+                    for (int b = 1; b <= kY2Stages; ++b)
+                        if (jt - b >= 0) mbar_wait(bar(Y2_FULL + ((jt - b) & 1)), ((jt - b) >> 1) & 1, &dummy_flag, p.status, BW_YFULL);
                 }
             }
         } else {
             // the key tile itself: K -> X1, V -> X2
-            if (lane == 0) {
+            if (warp == 4 && lane == 0) {
                 mbar_expect_tx(bar(X_FULL), 2 * TILE_BYTES);
 #pragma unroll
                 for (int sub = 0; sub < SUB; ++sub) {
@@ -315,92 +383,132 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     tma_load_2d(sX + TILE_BYTES + sub * SUB_BYTES, &tmV, sub * 64, h * p.L + w_t0, bar(X_FULL));
                 }
             }
-            // the queries that attend to this chunk, 128 at a time: Q rows -> Y1, dO rows -> Y2
+            // the queries that attend to this chunk, 128 at a time: Q rows -> Y1, dO rows -> Y2; each of the
+            // four producer warps copies 32 rows of every tile
+            const int pw = warp - 4;
             const int chunk = w_chunk;
             const int a1 = p.ranc_off[chunk + 1];
             int a = p.ranc_off[chunk], r0 = 0, r1 = 0;       // current row range [r0, r1)
             const int n_list = p.cnt[h * p.C + chunk];
             const int32_t *list = p.qlist + (size_t)h * p.cap_total + p.cap_off[chunk];
             int e0 = 0;                                        // next entry of the routed list
+            int s3 = 0, ph3 = 0;
             bool ok = true;
             for (int jt = 0; ok && jt < n_tiles; ++jt) {
-                const int st = jt & 1;
+                const int s2 = jt & 1;
                 if (r0 >= r1 && a < a1) {                      // next merged range of anchor query rows
                     int qc = p.ranc[a];
                     r0 = p.off[qc]; r1 = p.off[qc + 1];
                     for (++a; a < a1 && p.ranc[a] == qc + 1; ++a) { qc = p.ranc[a]; r1 = p.off[qc + 1]; }
                 }
-                int qrow[4];
-#pragma unroll
-                for (int m = 0; m < 4; ++m) {
-                    const int i = m * 32 + lane;
-                    qrow[m] = -1;
-                    if (r0 < r1) { if (r0 + i < r1) qrow[m] = r0 + i; }
-                    else if (e0 + i < n_list) qrow[m] = list[e0 + i] / p.k;
-                }
+                const int i = pw * 32 + lane;                  // this lane's row of the tile
+                int q = -1;
+                if (r0 < r1) { if (r0 + i < r1) q = r0 + i; }
+                else if (e0 + i < n_list) q = list[e0 + i] / p.k;
                 if (r0 < r1) r0 += 128; else e0 += 128;
-                ok = mbar_wait(bar(Y_EMPTY + st), ((jt >> 1) & 1) ^ 1, abort_flag, p.status, BW_YEMPTY);
+                // a column without a query gets lse = +inf: its P and dS come out as exact zeros
+                const float q_lse = q >= 0 ? p.lse[(size_t)h * p.L + q] * kLog2e : INFINITY;
+                const float q_del = q >= 0 ? p.delta[(size_t)h * p.L + q] : 0.f;
+                ok = mbar_wait(bar(Y1_EMPTY + s3), ph3 ^ 1, abort_flag, p.status, BW_YEMPTY);
+                ok = ok && mbar_wait(bar(Y2_EMPTY + s2), ((jt >> 1) & 1) ^ 1, abort_flag, p.status, BW_YEMPTY);
+                // the lanes have finished with the lse / delta of tile jt - 2
+                if (jt >= 2) ok = ok && mbar_wait(bar(DS_DONE + s2), ((jt - 2) >> 1) & 1, abort_flag, p.status, BW_DSDONE);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-#pragma unroll
-                for (int m = 0; m < 4; ++m) {
-                    const int i = m * 32 + lane, q = qrow[m];
-                    s_row[st][i] = q;
-                    // a column without a query gets lse = +inf: its P and dS come out as exact zeros
-                    s_lse[st][i] = q >= 0 ? p.lse[(size_t)h * p.L + q] * kLog2e : INFINITY;
-                    s_del[st][i] = q >= 0 ? p.delta[(size_t)h * p.L + q] : 0.f;
-                }
-                __syncwarp();
+                s_ld[s2][0][i] = q_lse;
+                s_ld[s2][1][i] = q_del;
                 constexpr int RP = 32 / CH;                    // rows per instruction
                 const int c16 = lane % CH;
 #pragma unroll 4
-                for (int rb = 0; rb < 128; rb += RP) {
-                    const int rr = rb + lane / CH, q = s_row[st][rr];
-                    const size_t src = ((size_t)h * p.L + max(q, 0)) * D + c16 * 8;
-                    const uint32_t dst = st * TILE_BYTES + (c16 >> 3) * SUB_BYTES + sw128_offset(rr, c16 & 7);
-                    cp_async16(sY1 + dst, p.Q + src, q >= 0 ? 16u : 0u);
-                    cp_async16(sY2 + dst, p.dO + src, q >= 0 ? 16u : 0u);
+                for (int rb = 0; rb < 32; rb += RP) {
+                    const int rl = rb + lane / CH, rr = pw * 32 + rl;
+                    const int qq = __shfl_sync(0xffffffffu, q, rl);
+                    const size_t src = ((size_t)h * p.L + max(qq, 0)) * D + c16 * 8;
+                    const uint32_t dst = (c16 >> 3) * SUB_BYTES + sw128_offset(rr, c16 & 7);
+                    cp_async16(sY1 + s3 * TILE_BYTES + dst, p.Q + src, qq >= 0 ? 16u : 0u);
+                    cp_async16(sY2 + s2 * TILE_BYTES + dst, p.dO + src, qq >= 0 ? 16u : 0u);
                 }
                 cp_async_wait_all();
                 fence_proxy_async_smem();
-                mbar_arrive(bar(Y_FULL + st));
+                mbar_arrive(bar(Y1_FULL + s3));
+                mbar_arrive(bar(Y2_FULL + s2));
+                if (++s3 == kY1Stages) { s3 = 0; ph3 ^= 1; }
             }
         }
     } else {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issuer (warp 8; warps 9-11 idle)
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
+        if (warp == 8 && lane == 0) {
             constexpr uint32_t IDESC_T = idesc_bf16_f32(128, 128, 0, 0);      // T = X Y^T, both K-major
             constexpr uint32_t IDESC_ACC = idesc_bf16_f32(128, D, 0, 1);      // ACC += (TMEM) Y, Y MN-major
             constexpr uint64_t STAGE = TILE_BYTES >> 4;
             const uint64_t x1 = smem_desc_sw128(sX, 16, 1024), x2 = smem_desc_sw128(sX + TILE_BYTES, 16, 1024);
             const uint64_t y1k = smem_desc_sw128(sY1, 16, 1024), y2k = smem_desc_sw128(sY2, 16, 1024);
             const uint64_t y1m = smem_desc_sw128(sY1, SUB_BYTES, 1024), y2m = smem_desc_sw128(sY2, SUB_BYTES, 1024);
-            bool ok = mbar_wait(bar(X_FULL), 0, abort_flag, p.status, BW_XFULL);
-            for (int jt = 0; ok && jt < n_tiles; ++jt) {
-                const int st = jt & 1;
-                const uint64_t so = st ? STAGE : 0;
-                if (!(ok = mbar_wait(bar(Y_FULL + st), (jt >> 1) & 1, abort_flag, p.status, BW_YFULL))) break;
+            bool ok = true;
+            // each step waits for what it reads, issues its MMAs and commits to the barriers of what it completes
+            auto t1 = [&](int j) {          // T1(j) = X1 Y1(j)^T
+                const int s3 = j % kY1Stages;
+                if (!(ok = mbar_wait(bar(Y1_FULL + s3), (j / kY1Stages) & 1, abort_flag, p.status, BW_YFULL))) return;
+                tc_fence_after();
+                const uint32_t d = tmem + ((MODE != DKV && (j & 1)) ? 384u : 0u);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t o = ((ks >> 2) * SUB_BYTES + (ks & 3) * 32) >> 4;
+                    mma_ss(d, x1 + o, y1k + s3 * STAGE + o, IDESC_T, ks > 0);
+                }
+                tc_commit(bar(T1_FULL + (j & 1)));
+            };
+            auto t2 = [&](int j) {          // T2(j) = X2 Y2(j)^T
+                const int s2 = j & 1;
+                if (!(ok = mbar_wait(bar(Y2_FULL + s2), (j >> 1) & 1, abort_flag, p.status, BW_YFULL))) return;
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t o = ((ks >> 2) * SUB_BYTES + (ks & 3) * 32) >> 4;
-                    mma_ss(tmem, x1 + o, y1k + so + o, IDESC_T, ks > 0);
+                    mma_ss(tmem + 128, x2 + o, y2k + s2 * STAGE + o, IDESC_T, ks > 0);
                 }
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t o = ((ks >> 2) * SUB_BYTES + (ks & 3) * 32) >> 4;
-                    mma_ss(tmem + 128, x2 + o, y2k + so + o, IDESC_T, ks > 0);
-                }
-                tc_commit(bar(T_FULL));
-                if (!(ok = mbar_wait(bar(D_FULL), jt & 1, abort_flag, p.status, BW_DFULL))) break;
+                tc_commit(bar(T2_FULL));
+                if (MODE != DKV) tc_commit(bar(Y2_EMPTY + s2));      // the dQ modes read V here only
+            };
+            auto acc1 = [&](int j) {        // ACC1 += dS(j) Y1(j)
+                if (!(ok = mbar_wait(bar(DS_DONE + (j & 1)), (j >> 1) & 1, abort_flag, p.status, BW_DSDONE))) return;
                 tc_fence_after();
+                const int s3 = j % kY1Stages;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) mma_ts(tmem + 256, tmem + 128 + ks * 8, y1m + so + ks * (2048 >> 4), IDESC_ACC, jt > 0 || ks > 0);
-                if (MODE == DKV) {
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ts(tmem + 256, tmem + 128 + ks * 8, y1m + s3 * STAGE + ks * (2048 >> 4), IDESC_ACC, j > 0 || ks > 0);
+                tc_commit(bar(Y1_EMPTY + s3));
+            };
+            auto acc2 = [&](int j) {        // ACC2 += P(j) Y2(j)
+                if (!(ok = mbar_wait(bar(P_DONE), j & 1, abort_flag, p.status, BW_PDONE))) return;
+                tc_fence_after();
+                const int s2 = j & 1;
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) mma_ts(tmem + 384, tmem + ks * 8, y2m + so + ks * (2048 >> 4), IDESC_ACC, jt > 0 || ks > 0);
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ts(tmem + 384, tmem + ks * 8, y2m + s2 * STAGE + ks * (2048 >> 4), IDESC_ACC, j > 0 || ks > 0);
+                tc_commit(bar(Y2_EMPTY + s2));
+            };
+            ok = mbar_wait(bar(X_FULL), 0, abort_flag, p.status, BW_XFULL);
+            if (ok && n_tiles > 0) t1(0);
+            if (ok && n_tiles > 0) t2(0);
+            if (MODE == DKV) {
+                // T1(j+1) follows ACC2(j), which reads the P written over T1(j); T2(j+1) follows ACC1(j),
+                // which reads the dS written over T2(j).  The lanes work on P(j+1) while ACC1(j), T2(j+1) run.
+                for (int j = 0; ok && j < n_tiles; ++j) {
+                    acc2(j);
+                    if (ok && j + 1 < n_tiles) t1(j + 1);
+                    if (ok) acc1(j);
+                    if (ok && j + 1 < n_tiles) t2(j + 1);
                 }
-                tc_commit(bar(Y_EMPTY + st));
+            } else {
+                // two T1 buffers: T1(j+2) is issued as soon as the lanes have consumed tile j
+                if (ok && n_tiles > 1) t1(1);
+                for (int j = 0; ok && j < n_tiles; ++j) {
+                    acc1(j);
+                    if (ok && j + 1 < n_tiles) t2(j + 1);
+                    if (ok && j + 2 < n_tiles) t1(j + 2);
+                }
             }
             if (ok) tc_commit(bar(ACC_FULL));
         }
@@ -430,28 +538,41 @@ static int attend_bwd_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv
     a.status = ws_ptr<int>(ws, p->ws.status);
     a.H = p->H; a.L = p->L; a.C = p->C; a.k = p->k;
     a.scale = p->scale; a.scale_log2 = p->scale * kLog2e;
-    const size_t smem = 6 * (size_t)128 * 128 * 2 + 1024;     // the d = 128 footprint: one CTA (512 TMEM columns) per SM
-    static bool attr_done[2] = {false, false};
-    if (!attr_done[D == 128]) {
-        MOC_CUDA_TRY(cudaFuncSetAttribute(attend_bwd_tc_kernel<D, DQ_ROUTED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        MOC_CUDA_TRY(cudaFuncSetAttribute(attend_bwd_tc_kernel<D, DQ_ANCHOR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        MOC_CUDA_TRY(cudaFuncSetAttribute(attend_bwd_tc_kernel<D, DKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_done[D == 128] = true;
+    // seven tiles (X1 X2, three Y1 stages, two Y2 stages) and the slack that aligns them to 1024 bytes; at
+    // d = 128 that is all an SM has, so the request is what the kernel's static variables leave of the limit
+    const size_t tiles = (size_t)(2 + kY1Stages + kY2Stages) * 128 * D * 2;
+    static size_t smem_mode[2][3] = {{0, 0, 0}, {0, 0, 0}};
+    if (!smem_mode[D == 128][0]) {
+        int dev = 0, optin = 0;
+        MOC_CUDA_TRY(cudaGetDevice(&dev));
+        MOC_CUDA_TRY(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+        const void *fn[3] = {(const void *)attend_bwd_tc_kernel<D, DQ_ROUTED>, (const void *)attend_bwd_tc_kernel<D, DQ_ANCHOR>,
+                             (const void *)attend_bwd_tc_kernel<D, DKV>};
+        size_t got[3];
+        for (int m = 0; m < 3; ++m) {
+            cudaFuncAttributes fa;
+            MOC_CUDA_TRY(cudaFuncGetAttributes(&fa, fn[m]));
+            got[m] = std::min(tiles + 1024, (size_t)optin - fa.sharedSizeBytes);
+            if (got[m] < tiles) return MOC_ERR_SHAPE;
+            MOC_CUDA_TRY(cudaFuncSetAttribute(fn[m], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)got[m]));
+        }
+        for (int m = 2; m >= 0; --m) smem_mode[D == 128][m] = got[m];
     }
+    const size_t *smem = smem_mode[D == 128];
     if (p->k > 0) {
         a.rng = p->d_chunk_rng;
         a.items = ws_ptr<WorkItem>(ws, p->ws.rtiles);
         a.n_items_dev = ws_ptr<int>(ws, p->ws.tile_off) + (size_t)p->H * p->C;
         const long long bound = (long long)p->H * (((long long)p->L * p->k + kQTileRows - 1) / kQTileRows + p->C);
-        attend_bwd_tc_kernel<D, DQ_ROUTED><<<(unsigned)(2 * bound), kBwdThreads, smem, s>>>(tmK, tmV, a);
+        attend_bwd_tc_kernel<D, DQ_ROUTED><<<(unsigned)(2 * bound), kBwdThreads, smem[DQ_ROUTED], s>>>(tmK, tmV, a);
         MOC_LAUNCH_CHECK();
     }
     a.rng = p->d_anc_rng;
     a.items = p->d_qitems;
     a.n_items_dev = nullptr;
-    attend_bwd_tc_kernel<D, DQ_ANCHOR><<<dim3((unsigned)(2 * p->qitems.size()), (unsigned)p->H), kBwdThreads, smem, s>>>(tmK, tmV, a);
+    attend_bwd_tc_kernel<D, DQ_ANCHOR><<<dim3((unsigned)(2 * p->qitems.size()), (unsigned)p->H), kBwdThreads, smem[DQ_ANCHOR], s>>>(tmK, tmV, a);
     MOC_LAUNCH_CHECK();
-    attend_bwd_tc_kernel<D, DKV><<<dim3((unsigned)p->ktiles.size(), (unsigned)p->H), kBwdThreads, smem, s>>>(tmK, tmV, a);
+    attend_bwd_tc_kernel<D, DKV><<<dim3((unsigned)p->ktiles.size(), (unsigned)p->H), kBwdThreads, smem[DKV], s>>>(tmK, tmV, a);
     MOC_LAUNCH_CHECK();
     return MOC_OK;
 }
