@@ -20,10 +20,11 @@
 //     dK, ACC2 is dV.  Each key tile is owned by one CTA: no atomics, no partial sums.
 // The tensor pipe and the lanes overlap across tiles.  dK/dV: the issue order is ACC2(j), T1(j+1),
 // ACC1(j), T2(j+1), so that while the lanes form P(j+1) the pipe runs ACC1(j) and T2(j+1), and T1 / T2
-// are rewritten only after the contraction that reads the P / dS stored over them.  dQ: no ACC2, so
-// its columns serve as a second T1 and T1(j+2) is issued as soon as the lanes have finished tile j.
-// 12 warps: 0-3 the lane threads, 4-7 the producers, 8 the MMA issuer, 9-11 idle (they complete the
-// third warpgroup, whose registers go to the lanes).  Every mbarrier wait is
+// are rewritten only after the contraction that reads the P / dS stored over them; ACC2(j) starts on the
+// first half of P(j) while the lanes form the second.  dQ: no ACC2, so its columns serve as a second T2:
+// T1(j+1) and T2(j+1) are issued once the lanes have read T1(j) and run while they form dS(j).
+// 12 warps: 0-3 the lane threads, 4-7 the producers, 8 and 9 the MMA issuers, 10-11 idle (they complete
+// the third warpgroup, whose registers go to the lanes).  Every mbarrier wait is
 // bounded; a wait that runs out flags the workspace status word and the CTA drains and leaves.
 #include <algorithm>
 
@@ -57,6 +58,21 @@ struct BwdParams {
 };
 
 constexpr int kY1Stages = 3, kY2Stages = 2;   // stages of the streamed tiles Y1 (read twice per tile) and Y2
+// Optional cycle-stamp tracing of one CTA per mode (build with -DMOC_TRACE): each hook stores clock64()
+// into a slot of g_trace_bwd, read back with moc_trace_read_bwd().  Compiled out otherwise.
+// slot map: 0 start, 1 TMEM ready, 2 X staged, 3 epilogue begins, 4 epilogue done; lanes, tile j: 16 + 8 j +
+// {0 T1 ready, 1 P done, 2 T2 ready, 3 dS done}; issuer, tile j: 1024 + 8 j + {0 T1, 1 T2, 2 ACC1, 3 ACC2}
+// (stamped after the step's wait); producer, tile j: 1536 + 4 j + {0 stages free, 1 copies done or issued}.
+#ifdef MOC_TRACE
+__device__ long long g_trace_bwd[3][2048];
+#define BTRACE_CTA (MODE == DQ_ROUTED ? blockIdx.x == 5000 : MODE == DQ_ANCHOR ? (blockIdx.x == 70 && blockIdx.y == 3) : (blockIdx.x == 100 && blockIdx.y == 3))
+#define BTRACE(slot) do { if (BTRACE_CTA) g_trace_bwd[MODE][(slot)] = clock64(); } while (0)
+#define BTRACE_J(base, stride, j, k) do { if ((j) < 60) BTRACE((base) + (stride) * (j) + (k)); } while (0)
+#else
+#define BTRACE(slot) ((void)0)
+#define BTRACE_J(base, stride, j, k) ((void)0)
+#endif
+
 constexpr int kBwdThreads = 384;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -70,7 +86,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
     constexpr int CH = D / 8;               // 16-byte pieces per row
     constexpr int N_TILES_SMEM = 2 + kY1Stages + kY2Stages;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[18];
+    __shared__ __align__(8) uint64_t bars[21];
     __shared__ uint32_t tmem_slot;
     __shared__ int s_abort;
     __shared__ int w_valid, w_h, w_rows, w_first, w_nrng, w_ntiles, w_chunk, w_t0;
@@ -86,8 +102,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
     const uint32_t sX = sbase, sY1 = sbase + 2 * TILE_BYTES, sY2 = sbase + (2 + kY1Stages) * TILE_BYTES;
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     constexpr int X_FULL = 0, Y1_FULL = 1, Y1_EMPTY = 4, Y2_FULL = 7, Y2_EMPTY = 9, T1_FULL = 11, T2_FULL = 13,
-                  P_DONE = 14, DS_DONE = 15, ACC_FULL = 17;
+                  P_HALF = 15, P_DONE = 16, DS_DONE = 17, ACC_FULL = 19, T1_ISSUED = 20;
 
+    if (threadIdx.x == 0) BTRACE(0);
     if (threadIdx.x == 0) {
         s_abort = 0;
         int valid = (*(volatile int *)p.status == 0);
@@ -136,13 +153,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
         }
         for (int t = 0; t < kY2Stages; ++t) {
             mbar_init(bar(Y2_FULL + t), MODE == DKV ? 128 : 1);
-            mbar_init(bar(Y2_EMPTY + t), 1);
+            mbar_init(bar(Y2_EMPTY + t), MODE == DKV ? 2 : 1);     // dK/dV: T2 and ACC2 both read the stage
             mbar_init(bar(T1_FULL + t), 1);
+            mbar_init(bar(T2_FULL + t), 1);
             mbar_init(bar(DS_DONE + t), 128);
         }
-        mbar_init(bar(T2_FULL), 1);
+        mbar_init(bar(P_HALF), 128);
         mbar_init(bar(P_DONE), 128);
-        mbar_init(bar(ACC_FULL), 1);
+        mbar_init(bar(T1_ISSUED), 1);
+        mbar_init(bar(ACC_FULL), 2);                                // both issuers
         fence_barrier_init();
     }
     __syncthreads();
@@ -156,8 +175,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
     tc_fence_after();
 
     // TMEM columns: T1 [0,128)  T2 [128,256)  ACC1 [256,384)  ACC2 [384,512); the dQ modes have no ACC2
-    // and use its columns as a second T1, for the odd tiles
+    // and use its columns as a second T2, for the odd tiles
     const uint32_t tmem = tmem_slot;
+    if (threadIdx.x == 0) BTRACE(1);
     const int h = w_h, rows = w_rows, n_tiles = w_ntiles;
     volatile int *abort_flag = &s_abort;
 
@@ -204,6 +224,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             }
             fence_proxy_async_smem();
             mbar_arrive(bar(X_FULL));
+            if (r == 0) BTRACE(2);
         }
         const float c = p.scale_log2;
         TileIter it(w_rng, MODE == DKV ? 0 : w_nrng);
@@ -213,18 +234,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             const int st = jt & 1;
             int valid = 128, t0;
             if (MODE != DKV) it.next(t0, valid);
-            ok = mbar_wait(bar(T1_FULL + st), (jt >> 1) & 1, abort_flag, p.status, BW_T1FULL);
+            ok = mbar_wait_spin(bar(T1_FULL + st), (jt >> 1) & 1, abort_flag, p.status, BW_T1FULL);
             if (MODE == DKV) ok = ok && mbar_wait(bar(Y1_FULL + s3), ph3, abort_flag, p.status, BW_YFULL);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
+            if (r == 0) BTRACE_J(16, 8, jt, 0);
             // ---- P = exp2(scale log2(e) S - lse log2(e)) from T1
-            const uint32_t t1 = (MODE != DKV && st) ? 384u : 0u;
+            const uint32_t t2c = (MODE != DKV && st) ? 384u : 128u;       // T2 (then dS) of this tile
             float pv[128];
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
                 uint32_t s[32];
-                tmem_ld32(tmem + lane_off + t1 + ch * 32, s);
+                tmem_ld32(tmem + lane_off + ch * 32, s);
                 tmem_wait_ld();
 #pragma unroll
                 for (int x = 0; x < 32; x += 2) {
@@ -246,22 +268,28 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
 #pragma unroll
                     for (int x = 0; x < 16; ++x) ups[x] = bf16x2(pv[ch * 32 + 2 * x], pv[ch * 32 + 2 * x + 1]);
                     tmem_st16(tmem + lane_off + ch * 16, ups);
+                    if (ch == 1) {                                        // the first 64 columns of P can be contracted
+                        tmem_wait_st();
+                        tc_fence_before();
+                        mbar_arrive(bar(P_HALF));
+                    }
                 }
             }
-            if (MODE == DKV) {
-                tmem_wait_st();
-                tc_fence_before();
-                mbar_arrive(bar(P_DONE));
-            }
+            // dK/dV: P is complete; dQ: T1 has been read and may be overwritten
+            if (MODE == DKV) tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar(P_DONE));
+            if (r == 0) BTRACE_J(16, 8, jt, 1);
             // ---- dS = P (dP - delta) from T2, written over the T2 columns already read
-            ok = mbar_wait(bar(T2_FULL), jt & 1, abort_flag, p.status, BW_T2FULL);
+            ok = mbar_wait_spin(bar(T2_FULL + st), (jt >> 1) & 1, abort_flag, p.status, BW_T2FULL);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
+            if (r == 0) BTRACE_J(16, 8, jt, 2);
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
                 uint32_t dp[32], uds[16];
-                tmem_ld32(tmem + lane_off + 128 + ch * 32, dp);
+                tmem_ld32(tmem + lane_off + t2c + ch * 32, dp);
                 tmem_wait_ld();
 #pragma unroll
                 for (int x = 0; x < 32; x += 2) {
@@ -273,11 +301,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     uds[x >> 1] = bf16x2(pv[ch * 32 + x] * (__uint_as_float(dp[x]) - d0),
                                          pv[ch * 32 + x + 1] * (__uint_as_float(dp[x + 1]) - d1));
                 }
-                tmem_st16(tmem + lane_off + 128 + ch * 16, uds);
+                tmem_st16(tmem + lane_off + t2c + ch * 16, uds);
             }
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(DS_DONE + st));
+            if (r == 0) BTRACE_J(16, 8, jt, 3);
             if (++s3 == kY1Stages) { s3 = 0; ph3 ^= 1; }
         }
         // ---- epilogue
@@ -287,6 +316,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
         }
         if (ok) {
             tc_fence_after();
+            if (r == 0) BTRACE(3);
 #pragma unroll 1
             for (int ch = 0; ch < D / 32; ++ch) {
                 uint32_t v[32];
@@ -340,6 +370,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 }
             }
         }
+        if (r == 0) BTRACE(4);
     } else if (warp < 8) {
         // ------------------------------------------------------------ producers
         asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
@@ -352,6 +383,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 while (it.next(t0, valid)) {
                     const int s2 = jt & 1;
                     if (!mbar_wait(bar(Y1_EMPTY + s3), ph3 ^ 1, abort_flag, p.status, BW_YEMPTY)) break;
+                    BTRACE_J(1536, 4, jt, 0);
                     mbar_expect_tx(bar(Y1_FULL + s3), TILE_BYTES);
 #pragma unroll
                     for (int sub = 0; sub < SUB; ++sub)
@@ -362,6 +394,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
 #pragma unroll
                     for (int sub = 0; sub < SUB; ++sub)
                         tma_load_2d(sY2 + s2 * TILE_BYTES + sub * SUB_BYTES, &tmV, sub * 64, h * p.L + t0, bar(Y2_FULL + s2));
+                    BTRACE_J(1536, 4, jt, 1);
                     ++jt;
                     if (++s3 == kY1Stages) { s3 = 0; ph3 ^= 1; }
                 }
@@ -415,6 +448,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 if (jt >= 2) ok = ok && mbar_wait(bar(DS_DONE + s2), ((jt - 2) >> 1) & 1, abort_flag, p.status, BW_DSDONE);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+                if (warp == 4 && lane == 0) BTRACE_J(1536, 4, jt, 0);
                 s_ld[s2][0][i] = q_lse;
                 s_ld[s2][1][i] = q_del;
                 constexpr int RP = 32 / CH;                    // rows per instruction
@@ -432,13 +466,18 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 fence_proxy_async_smem();
                 mbar_arrive(bar(Y1_FULL + s3));
                 mbar_arrive(bar(Y2_FULL + s2));
+                if (warp == 4 && lane == 0) BTRACE_J(1536, 4, jt, 1);
                 if (++s3 == kY1Stages) { s3 = 0; ph3 ^= 1; }
             }
         }
     } else {
-        // ------------------------------------------------------------ MMA issuer (warp 8; warps 9-11 idle)
+        // ------------------------------------------------------------ MMA issuers: warp 8 owns the T1 / P side
+        // (T1, ACC2), warp 9 the T2 / dS side (T2, ACC1); each side's TMEM columns are touched by its issuer only,
+        // so the two instruction streams need no ordering between them and one's waits and commits are
+        // covered by the other's MMAs.  Warps 10 and 11 idle.
         asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
-        if (warp == 8 && lane == 0) {
+        if (warp <= 9 && lane == 0) {
+            const bool side1 = warp == 8;
             constexpr uint32_t IDESC_T = idesc_bf16_f32(128, 128, 0, 0);      // T = X Y^T, both K-major
             constexpr uint32_t IDESC_ACC = idesc_bf16_f32(128, D, 0, 1);      // ACC += (TMEM) Y, Y MN-major
             constexpr uint64_t STAGE = TILE_BYTES >> 4;
@@ -446,68 +485,114 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             const uint64_t y1k = smem_desc_sw128(sY1, 16, 1024), y2k = smem_desc_sw128(sY2, 16, 1024);
             const uint64_t y1m = smem_desc_sw128(sY1, SUB_BYTES, 1024), y2m = smem_desc_sw128(sY2, SUB_BYTES, 1024);
             bool ok = true;
-            // each step waits for what it reads, issues its MMAs and commits to the barriers of what it completes
+            auto wait = [&](int b, int parity, int code) { ok = ok && mbar_wait_spin(bar(b), parity, abort_flag, p.status, code); };
+            // the MMA groups, without their waits and commits
             auto t1 = [&](int j) {          // T1(j) = X1 Y1(j)^T
                 const int s3 = j % kY1Stages;
-                if (!(ok = mbar_wait(bar(Y1_FULL + s3), (j / kY1Stages) & 1, abort_flag, p.status, BW_YFULL))) return;
-                tc_fence_after();
-                const uint32_t d = tmem + ((MODE != DKV && (j & 1)) ? 384u : 0u);
+                BTRACE_J(1024, 8, j, 0);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t o = ((ks >> 2) * SUB_BYTES + (ks & 3) * 32) >> 4;
-                    mma_ss(d, x1 + o, y1k + s3 * STAGE + o, IDESC_T, ks > 0);
+                    mma_ss(tmem, x1 + o, y1k + s3 * STAGE + o, IDESC_T, ks > 0);
                 }
-                tc_commit(bar(T1_FULL + (j & 1)));
+                BTRACE_J(1024, 8, j, 4);
             };
             auto t2 = [&](int j) {          // T2(j) = X2 Y2(j)^T
                 const int s2 = j & 1;
-                if (!(ok = mbar_wait(bar(Y2_FULL + s2), (j >> 1) & 1, abort_flag, p.status, BW_YFULL))) return;
-                tc_fence_after();
+                BTRACE_J(1024, 8, j, 1);
+                const uint32_t d = tmem + ((MODE != DKV && s2) ? 384u : 128u);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t o = ((ks >> 2) * SUB_BYTES + (ks & 3) * 32) >> 4;
-                    mma_ss(tmem + 128, x2 + o, y2k + s2 * STAGE + o, IDESC_T, ks > 0);
+                    mma_ss(d, x2 + o, y2k + s2 * STAGE + o, IDESC_T, ks > 0);
                 }
-                tc_commit(bar(T2_FULL));
-                if (MODE != DKV) tc_commit(bar(Y2_EMPTY + s2));      // the dQ modes read V here only
             };
             auto acc1 = [&](int j) {        // ACC1 += dS(j) Y1(j)
-                if (!(ok = mbar_wait(bar(DS_DONE + (j & 1)), (j >> 1) & 1, abort_flag, p.status, BW_DSDONE))) return;
-                tc_fence_after();
+                BTRACE_J(1024, 8, j, 2);
                 const int s3 = j % kY1Stages;
+                const uint32_t ds = tmem + ((MODE != DKV && (j & 1)) ? 384u : 128u);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    mma_ts(tmem + 256, tmem + 128 + ks * 8, y1m + s3 * STAGE + ks * (2048 >> 4), IDESC_ACC, j > 0 || ks > 0);
-                tc_commit(bar(Y1_EMPTY + s3));
+                    mma_ts(tmem + 256, ds + ks * 8, y1m + s3 * STAGE + ks * (2048 >> 4), IDESC_ACC, j > 0 || ks > 0);
             };
-            auto acc2 = [&](int j) {        // ACC2 += P(j) Y2(j)
-                if (!(ok = mbar_wait(bar(P_DONE), j & 1, abort_flag, p.status, BW_PDONE))) return;
-                tc_fence_after();
+            auto acc2 = [&](int j, int half) {   // ACC2 += P(j) Y2(j), the K steps of one half of P
                 const int s2 = j & 1;
+                if (half == 0) BTRACE_J(1024, 8, j, 3);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ts(tmem + 384, tmem + ks * 8, y2m + s2 * STAGE + ks * (2048 >> 4), IDESC_ACC, j > 0 || ks > 0);
-                tc_commit(bar(Y2_EMPTY + s2));
+                for (int ks = 0; ks < 4; ++ks)
+                    mma_ts(tmem + 384, tmem + (half * 4 + ks) * 8, y2m + s2 * STAGE + (half * 4 + ks) * (2048 >> 4), IDESC_ACC,
+                           j > 0 || half > 0 || ks > 0);
             };
-            ok = mbar_wait(bar(X_FULL), 0, abort_flag, p.status, BW_XFULL);
-            if (ok && n_tiles > 0) t1(0);
-            if (ok && n_tiles > 0) t2(0);
-            if (MODE == DKV) {
-                // T1(j+1) follows ACC2(j), which reads the P written over T1(j); T2(j+1) follows ACC1(j),
-                // which reads the dS written over T2(j).  The lanes work on P(j+1) while ACC1(j), T2(j+1) run.
+            // A wait, a fence or a commit between two groups leaves the pipe idle for longer than it takes, so each
+            // side waits early for the tiles it will read, fences once per hand-over from the lanes, and commits
+            // after the last group it has to issue at that point.
+            wait(X_FULL, 0, BW_XFULL);
+            if (side1) {
+                // dK/dV: ACC2(j) starts on the first half of P(j); T1(j+1) follows ACC2(j), which reads the P
+                // written over T1(j).  dQ: T1(j+1) follows the lanes' read of T1(j).
+                if (n_tiles > 0) {
+                    wait(Y1_FULL, 0, BW_YFULL);
+                    if (ok) {
+                        tc_fence_after();
+                        t1(0);
+                        tc_commit(bar(T1_FULL));
+                    }
+                }
                 for (int j = 0; ok && j < n_tiles; ++j) {
-                    acc2(j);
-                    if (ok && j + 1 < n_tiles) t1(j + 1);
-                    if (ok) acc1(j);
-                    if (ok && j + 1 < n_tiles) t2(j + 1);
+                    const bool more = j + 1 < n_tiles;
+                    if (MODE == DKV) {
+                        wait(P_HALF, j & 1, BW_PDONE);
+                        if (!ok) break;
+                        tc_fence_after();
+                        acc2(j, 0);
+                    }
+                    if (more) wait(Y1_FULL + (j + 1) % kY1Stages, ((j + 1) / kY1Stages) & 1, BW_YFULL);
+                    if (MODE == DKV || more) wait(P_DONE, j & 1, BW_PDONE);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (MODE == DKV) acc2(j, 1);
+                    if (more) {
+                        t1(j + 1);
+                        tc_commit(bar(T1_FULL + ((j + 1) & 1)));
+                        BTRACE_J(1024, 8, j + 1, 5);
+                    }
+                    if (MODE == DKV) {
+                        tc_commit(bar(Y2_EMPTY + (j & 1)));                 // the second of two arrivals
+                        if (more) mbar_arrive(bar(T1_ISSUED));              // the other side may use the pipe again
+                    }
                 }
             } else {
-                // two T1 buffers: T1(j+2) is issued as soon as the lanes have consumed tile j
-                if (ok && n_tiles > 1) t1(1);
+                // The lanes wait for T1(j+1) as soon as dS(j) is done, so this side keeps out of the pipe while the
+                // other issues it.  dK/dV: ACC1(j) waits for that issue, and T2(j+1) follows ACC1(j), which reads the
+                // dS written over T2(j).  dQ: two T2 buffers; ACC1(j) then T2(j+2), both while the lanes form P(j+1).
+                constexpr int AHEAD = MODE == DKV ? 1 : 2;
+                for (int j = 0; ok && j < AHEAD && j < n_tiles; ++j) {
+                    wait(Y2_FULL + (j & 1), 0, BW_YFULL);
+                    if (!ok) break;
+                    tc_fence_after();
+                    t2(j);
+                    tc_commit(bar(T2_FULL + (j & 1)));
+                    tc_commit(bar(Y2_EMPTY + (j & 1)));
+                }
                 for (int j = 0; ok && j < n_tiles; ++j) {
+                    const int jn = j + AHEAD;
+                    const bool more = jn < n_tiles;
+                    // one look at the next Y2 tile before the hand-over; ACC1(j) never waits for it
+                    const bool y2_ready = more && mbar_test_wait(bar(Y2_FULL + (jn & 1)), (jn >> 1) & 1);
+                    if (MODE == DKV && j + 1 < n_tiles) wait(T1_ISSUED, j & 1, BW_T1FULL);
+                    wait(DS_DONE + (j & 1), (j >> 1) & 1, BW_DSDONE);
+                    if (!ok) break;
+                    tc_fence_after();
                     acc1(j);
-                    if (ok && j + 1 < n_tiles) t2(j + 1);
-                    if (ok && j + 2 < n_tiles) t1(j + 2);
+                    if (!y2_ready) tc_commit(bar(Y1_EMPTY + j % kY1Stages));
+                    if (more) {
+                        if (!y2_ready) wait(Y2_FULL + (jn & 1), (jn >> 1) & 1, BW_YFULL);
+                        if (!ok) break;
+                        t2(jn);
+                        tc_commit(bar(T2_FULL + (jn & 1)));
+                        tc_commit(bar(Y2_EMPTY + (jn & 1)));    // dQ modes: V is read here only; dK/dV: the first of two arrivals
+                    }
+                    if (y2_ready) tc_commit(bar(Y1_EMPTY + j % kY1Stages));
                 }
             }
             if (ok) tc_commit(bar(ACC_FULL));
@@ -576,6 +661,12 @@ static int attend_bwd_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv
     MOC_LAUNCH_CHECK();
     return MOC_OK;
 }
+
+#ifdef MOC_TRACE
+extern "C" int moc_trace_read_bwd(long long *host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_trace_bwd, sizeof(long long) * (size_t)n);
+}
+#endif
 
 int launch_attend_bwd_tc(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
                          const __nv_bfloat16 *O, const float *lse, const __nv_bfloat16 *dO, const int32_t *sel,
