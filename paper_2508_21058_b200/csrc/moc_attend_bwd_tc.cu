@@ -7,7 +7,7 @@
 // One kernel, three modes, one tile engine.  A CTA holds a STATIONARY pair of 128-row tiles
 // (X1, X2) in shared memory and streams pairs of 128-row tiles (Y1, Y2) through three and two stages:
 //     T1 = X1 Y1^T,  T2 = X2 Y2^T        (both operands from shared memory, into TMEM)
-//     threads (one TMEM lane each) turn T1 into P, then (P, T2) into dS, written back to TMEM as bf16
+//     threads (two per TMEM lane) turn T1 into P, then (P, T2) into dS, written back to TMEM as bf16
 //     ACC1 += dS Y1,  ACC2 += P Y2       (A from TMEM, B the streamed tile as an MN-major operand)
 //   dQ modes (query stationary, the forward's work items, 128 rows per CTA):  X = (Q, dO) rows of
 //     the item, Y = (K, V) tiles of its key ranges by TMA; lse and delta belong to the lane;
@@ -23,8 +23,8 @@
 // are rewritten only after the contraction that reads the P / dS stored over them; ACC2(j) starts on the
 // first half of P(j) while the lanes form the second.  dQ: no ACC2, so its columns serve as a second T2:
 // T1(j+1) and T2(j+1) are issued once the lanes have read T1(j) and run while they form dS(j).
-// 12 warps: 0-3 the lane threads, 4-7 the producers, 8 and 9 the MMA issuers, 10-11 idle (they complete
-// the third warpgroup, whose registers go to the lanes).  Every mbarrier wait is
+// 16 warps: 0-7 the lane threads (two per TMEM lane), 8-11 the producers, 12 and 13 the MMA issuers,
+// 14-15 idle (they complete the fourth warpgroup; the lanes take the registers the others give up).  Every mbarrier wait is
 // bounded; a wait that runs out flags the workspace status word and the CTA drains and leaves.
 #include <algorithm>
 
@@ -73,7 +73,7 @@ __device__ long long g_trace_bwd[3][2048];
 #define BTRACE_J(base, stride, j, k) ((void)0)
 #endif
 
-constexpr int kBwdThreads = 384;
+constexpr int kBwdThreads = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D, int MODE>
@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             w_ntiles = nt;
         }
         w_valid = valid;
-        mbar_init(bar(X_FULL), MODE == DKV ? 1 : 128);
+        mbar_init(bar(X_FULL), MODE == DKV ? 1 : 256);
         for (int t = 0; t < kY1Stages; ++t) {
             mbar_init(bar(Y1_FULL + t), MODE == DKV ? 128 : 1);
             mbar_init(bar(Y1_EMPTY + t), 1);
@@ -156,17 +156,17 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             mbar_init(bar(Y2_EMPTY + t), MODE == DKV ? 2 : 1);     // dK/dV: T2 and ACC2 both read the stage
             mbar_init(bar(T1_FULL + t), 1);
             mbar_init(bar(T2_FULL + t), 1);
-            mbar_init(bar(DS_DONE + t), 128);
+            mbar_init(bar(DS_DONE + t), 256);
         }
-        mbar_init(bar(P_HALF), 128);
-        mbar_init(bar(P_DONE), 128);
+        mbar_init(bar(P_HALF), 256);
+        mbar_init(bar(P_DONE), 256);
         mbar_init(bar(T1_ISSUED), 1);
         mbar_init(bar(ACC_FULL), 2);                                // both issuers
         fence_barrier_init();
     }
     __syncthreads();
     if (!w_valid) return;
-    if (warp == 4) {
+    if (warp == 8) {
         tmem_alloc(smem_u32(&tmem_slot), 512);
         tmem_relinquish();
     }
@@ -181,13 +181,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
     const int h = w_h, rows = w_rows, n_tiles = w_ntiles;
     volatile int *abort_flag = &s_abort;
 
-    if (warp < 4) {
-        // ------------------------------------------------------------ lane threads
-        // a thread keeps the 128 P values of its row between the two halves of a tile: it takes the
-        // registers that the other two warpgroups give up
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
-        const int r = threadIdx.x;                    // row of the stationary tile = TMEM lane
-        const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    if (warp < 8) {
+        // ------------------------------------------------------------ lane threads: two per TMEM lane (warps w and
+        // w + 4 reach the same lanes).  Of the four 32-column chunks of a tile, thread `half` takes chunks half and
+        // 2 + half, so that the first two chunks - the first half of P for ACC2 - are finished first.  A thread
+        // keeps its 64 P values between the two halves of a tile.
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 168;");
+        const int r = threadIdx.x & 127;              // row of the stationary tile = TMEM lane
+        const int half = warp >> 2;
+        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
         int qi = -1, slot = 0;
         float lse2 = INFINITY, dlt = 0.f;             // dQ modes: this lane's query
         if (MODE != DKV) {
@@ -202,16 +204,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 lse2 = p.lse[(size_t)h * p.L + qi] * kLog2e;
                 dlt = p.delta[(size_t)h * p.L + qi];
             }
-            // stage the item's Q and dO rows together: consecutive threads take consecutive 16-byte pieces
+            // stage the item's rows, one half Q and the other dO: consecutive threads take consecutive 16-byte pieces
             int *s_row = reinterpret_cast<int *>(&s_ld[0][0][0]);
-            s_row[r] = qi;
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (half == 0) s_row[r] = qi;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             constexpr int RP = 128 / CH;
             const int c16 = r % CH;
-#pragma unroll
-            for (int which = 0; which < 2; ++which) {
-                const __nv_bfloat16 *src = which ? p.dO : p.Q;
-                uint8_t *dst = gbase + which * TILE_BYTES + (c16 >> 3) * SUB_BYTES;
+            {
+                const __nv_bfloat16 *src = half ? p.dO : p.Q;
+                uint8_t *dst = gbase + half * TILE_BYTES + (c16 >> 3) * SUB_BYTES;
                 uint4 v[CH];
 #pragma unroll
                 for (int ps = 0; ps < CH; ++ps) {
@@ -224,7 +225,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             }
             fence_proxy_async_smem();
             mbar_arrive(bar(X_FULL));
-            if (r == 0) BTRACE(2);
+            if (threadIdx.x == 0) BTRACE(2);
         }
         const float c = p.scale_log2;
         TileIter it(w_rng, MODE == DKV ? 0 : w_nrng);
@@ -239,15 +240,18 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            if (r == 0) BTRACE_J(16, 8, jt, 0);
+            if (threadIdx.x == 0) BTRACE_J(16, 8, jt, 0);
             // ---- P = exp2(scale log2(e) S - lse log2(e)) from T1
             const uint32_t t2c = (MODE != DKV && st) ? 384u : 128u;       // T2 (then dS) of this tile
-            float pv[128];
+            float pv[64];
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
+            for (int rd = 0; rd < 2; ++rd) {
+                const int ch = rd * 2 + half;
                 uint32_t s[32];
                 tmem_ld32(tmem + lane_off + ch * 32, s);
                 tmem_wait_ld();
+                // dK/dV: P goes over T1 columns that the other thread of the lane reads in its first round
+                if (MODE == DKV && rd == 0) asm volatile("bar.sync 2, 256;" ::: "memory");
 #pragma unroll
                 for (int x = 0; x < 32; x += 2) {
                     float l0 = lse2, l1 = lse2;
@@ -260,37 +264,37 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                         if (ch * 32 + x >= valid) p0 = 0.f;
                         if (ch * 32 + x + 1 >= valid) p1 = 0.f;
                     }
-                    pv[ch * 32 + x] = p0;
-                    pv[ch * 32 + x + 1] = p1;
+                    pv[rd * 32 + x] = p0;
+                    pv[rd * 32 + x + 1] = p1;
                 }
-                if (MODE == DKV) {                                        // P over the T1 columns already read
+                if (MODE == DKV) {
                     uint32_t ups[16];
 #pragma unroll
-                    for (int x = 0; x < 16; ++x) ups[x] = bf16x2(pv[ch * 32 + 2 * x], pv[ch * 32 + 2 * x + 1]);
+                    for (int x = 0; x < 16; ++x) ups[x] = bf16x2(pv[rd * 32 + 2 * x], pv[rd * 32 + 2 * x + 1]);
                     tmem_st16(tmem + lane_off + ch * 16, ups);
-                    if (ch == 1) {                                        // the first 64 columns of P can be contracted
-                        tmem_wait_st();
-                        tc_fence_before();
-                        mbar_arrive(bar(P_HALF));
-                    }
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(bar(rd == 0 ? P_HALF : P_DONE));      // the first, then the second 64 columns of P
                 }
             }
-            // dK/dV: P is complete; dQ: T1 has been read and may be overwritten
-            if (MODE == DKV) tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(P_DONE));
-            if (r == 0) BTRACE_J(16, 8, jt, 1);
-            // ---- dS = P (dP - delta) from T2, written over the T2 columns already read
+            if (MODE != DKV) {                                            // T1 has been read and may be overwritten
+                tc_fence_before();
+                mbar_arrive(bar(P_DONE));
+            }
+            if (threadIdx.x == 0) BTRACE_J(16, 8, jt, 1);
+            // ---- dS = P (dP - delta) from T2, written over T2 columns that have been read
             ok = mbar_wait_spin(bar(T2_FULL + st), (jt >> 1) & 1, abort_flag, p.status, BW_T2FULL);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            if (r == 0) BTRACE_J(16, 8, jt, 2);
+            if (threadIdx.x == 0) BTRACE_J(16, 8, jt, 2);
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
+            for (int rd = 0; rd < 2; ++rd) {
+                const int ch = rd * 2 + half;
                 uint32_t dp[32], uds[16];
                 tmem_ld32(tmem + lane_off + t2c + ch * 32, dp);
                 tmem_wait_ld();
+                if (rd == 0) asm volatile("bar.sync 3, 256;" ::: "memory");
 #pragma unroll
                 for (int x = 0; x < 32; x += 2) {
                     float d0 = dlt, d1 = dlt;
@@ -298,15 +302,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                         const float2 d = *reinterpret_cast<const float2 *>(&s_ld[st][1][ch * 32 + x]);
                         d0 = d.x; d1 = d.y;
                     }
-                    uds[x >> 1] = bf16x2(pv[ch * 32 + x] * (__uint_as_float(dp[x]) - d0),
-                                         pv[ch * 32 + x + 1] * (__uint_as_float(dp[x + 1]) - d1));
+                    uds[x >> 1] = bf16x2(pv[rd * 32 + x] * (__uint_as_float(dp[x]) - d0),
+                                         pv[rd * 32 + x + 1] * (__uint_as_float(dp[x + 1]) - d1));
                 }
                 tmem_st16(tmem + lane_off + t2c + ch * 16, uds);
             }
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(DS_DONE + st));
-            if (r == 0) BTRACE_J(16, 8, jt, 3);
+            if (threadIdx.x == 0) BTRACE_J(16, 8, jt, 3);
             if (++s3 == kY1Stages) { s3 = 0; ph3 ^= 1; }
         }
         // ---- epilogue
@@ -316,9 +320,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
         }
         if (ok) {
             tc_fence_after();
-            if (r == 0) BTRACE(3);
+            if (threadIdx.x == 0) BTRACE(3);
 #pragma unroll 1
-            for (int ch = 0; ch < D / 32; ++ch) {
+            for (int ch = half; ch < D / 32; ch += 2) {
                 uint32_t v[32];
                 __syncwarp();
                 tmem_ld32(tmem + lane_off + 256 + ch * 32, v);
@@ -370,12 +374,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 }
             }
         }
-        if (r == 0) BTRACE(4);
-    } else if (warp < 8) {
+        if (threadIdx.x == 0) BTRACE(4);
+    } else if (warp < 12) {
         // ------------------------------------------------------------ producers
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
         if (MODE != DKV) {
-            if (warp == 4 && lane == 0) {
+            if (warp == 8 && lane == 0) {
                 prefetch_tensormap(&tmK);
                 prefetch_tensormap(&tmV);
                 TileIter it(w_rng, w_nrng);
@@ -408,7 +412,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             }
         } else {
             // the key tile itself: K -> X1, V -> X2
-            if (warp == 4 && lane == 0) {
+            if (warp == 8 && lane == 0) {
                 mbar_expect_tx(bar(X_FULL), 2 * TILE_BYTES);
 #pragma unroll
                 for (int sub = 0; sub < SUB; ++sub) {
@@ -418,7 +422,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             }
             // the queries that attend to this chunk, 128 at a time: Q rows -> Y1, dO rows -> Y2; each of the
             // four producer warps copies 32 rows of every tile
-            const int pw = warp - 4;
+            const int pw = warp - 8;
             const int chunk = w_chunk;
             const int a1 = p.ranc_off[chunk + 1];
             int a = p.ranc_off[chunk], r0 = 0, r1 = 0;       // current row range [r0, r1)
@@ -427,33 +431,40 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             int e0 = 0;                                        // next entry of the routed list
             int s3 = 0, ph3 = 0;
             bool ok = true;
-            for (int jt = 0; ok && jt < n_tiles; ++jt) {
-                const int s2 = jt & 1;
+            const int i = pw * 32 + lane;                      // this lane's row of every tile
+            // the query behind this lane's row of the next tile, with its lse and delta; loaded one tile ahead so
+            // that these dependent loads are never waited for
+            int q = -1;
+            float q_lse = INFINITY, q_del = 0.f;
+            auto next_rows = [&]() {
                 if (r0 >= r1 && a < a1) {                      // next merged range of anchor query rows
                     int qc = p.ranc[a];
                     r0 = p.off[qc]; r1 = p.off[qc + 1];
                     for (++a; a < a1 && p.ranc[a] == qc + 1; ++a) { qc = p.ranc[a]; r1 = p.off[qc + 1]; }
                 }
-                const int i = pw * 32 + lane;                  // this lane's row of the tile
-                int q = -1;
+                q = -1;
                 if (r0 < r1) { if (r0 + i < r1) q = r0 + i; }
                 else if (e0 + i < n_list) q = list[e0 + i] / p.k;
                 if (r0 < r1) r0 += 128; else e0 += 128;
                 // a column without a query gets lse = +inf: its P and dS come out as exact zeros
-                const float q_lse = q >= 0 ? p.lse[(size_t)h * p.L + q] * kLog2e : INFINITY;
-                const float q_del = q >= 0 ? p.delta[(size_t)h * p.L + q] : 0.f;
+                q_lse = q >= 0 ? p.lse[(size_t)h * p.L + q] * kLog2e : INFINITY;
+                q_del = q >= 0 ? p.delta[(size_t)h * p.L + q] : 0.f;
+            };
+            if (n_tiles > 0) next_rows();
+            for (int jt = 0; ok && jt < n_tiles; ++jt) {
+                const int s2 = jt & 1;
                 ok = mbar_wait(bar(Y1_EMPTY + s3), ph3 ^ 1, abort_flag, p.status, BW_YEMPTY);
                 ok = ok && mbar_wait(bar(Y2_EMPTY + s2), ((jt >> 1) & 1) ^ 1, abort_flag, p.status, BW_YEMPTY);
                 // the lanes have finished with the lse / delta of tile jt - 2
                 if (jt >= 2) ok = ok && mbar_wait(bar(DS_DONE + s2), ((jt - 2) >> 1) & 1, abort_flag, p.status, BW_DSDONE);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (warp == 4 && lane == 0) BTRACE_J(1536, 4, jt, 0);
+                if (warp == 8 && lane == 0) BTRACE_J(1536, 4, jt, 0);
                 s_ld[s2][0][i] = q_lse;
                 s_ld[s2][1][i] = q_del;
                 constexpr int RP = 32 / CH;                    // rows per instruction
                 const int c16 = lane % CH;
-#pragma unroll 4
+#pragma unroll
                 for (int rb = 0; rb < 32; rb += RP) {
                     const int rl = rb + lane / CH, rr = pw * 32 + rl;
                     const int qq = __shfl_sync(0xffffffffu, q, rl);
@@ -462,22 +473,23 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     cp_async16(sY1 + s3 * TILE_BYTES + dst, p.Q + src, qq >= 0 ? 16u : 0u);
                     cp_async16(sY2 + s2 * TILE_BYTES + dst, p.dO + src, qq >= 0 ? 16u : 0u);
                 }
+                if (jt + 1 < n_tiles) next_rows();
                 cp_async_wait_all();
                 fence_proxy_async_smem();
                 mbar_arrive(bar(Y1_FULL + s3));
                 mbar_arrive(bar(Y2_FULL + s2));
-                if (warp == 4 && lane == 0) BTRACE_J(1536, 4, jt, 1);
+                if (warp == 8 && lane == 0) BTRACE_J(1536, 4, jt, 1);
                 if (++s3 == kY1Stages) { s3 = 0; ph3 ^= 1; }
             }
         }
     } else {
-        // ------------------------------------------------------------ MMA issuers: warp 8 owns the T1 / P side
-        // (T1, ACC2), warp 9 the T2 / dS side (T2, ACC1); each side's TMEM columns are touched by its issuer only,
+        // ------------------------------------------------------------ MMA issuers: warp 12 owns the T1 / P side
+        // (T1, ACC2), warp 13 the T2 / dS side (T2, ACC1); each side's TMEM columns are touched by its issuer only,
         // so the two instruction streams need no ordering between them and one's waits and commits are
-        // covered by the other's MMAs.  Warps 10 and 11 idle.
+        // covered by the other's MMAs.  Warps 14 and 15 idle.
         asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
-        if (warp <= 9 && lane == 0) {
-            const bool side1 = warp == 8;
+        if (warp <= 13 && lane == 0) {
+            const bool side1 = warp == 12;
             constexpr uint32_t IDESC_T = idesc_bf16_f32(128, 128, 0, 0);      // T = X Y^T, both K-major
             constexpr uint32_t IDESC_ACC = idesc_bf16_f32(128, D, 0, 1);      // ACC += (TMEM) Y, Y MN-major
             constexpr uint64_t STAGE = TILE_BYTES >> 4;
@@ -549,8 +561,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     if (more) wait(Y1_FULL + (j + 1) % kY1Stages, ((j + 1) / kY1Stages) & 1, BW_YFULL);
                     if (MODE == DKV || more) wait(P_DONE, j & 1, BW_PDONE);
                     if (!ok) break;
+                    BTRACE_J(1024, 8, j, 6);
                     tc_fence_after();
                     if (MODE == DKV) acc2(j, 1);
+                    BTRACE_J(1024, 8, j, 7);
                     if (more) {
                         t1(j + 1);
                         tc_commit(bar(T1_FULL + ((j + 1) & 1)));
@@ -600,7 +614,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) tmem_dealloc(tmem, 512);
+    if (warp == 8) tmem_dealloc(tmem, 512);
 }
 
 template <int D>
