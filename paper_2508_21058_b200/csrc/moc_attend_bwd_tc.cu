@@ -591,22 +591,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 for (int j = 0; ok && j < n_tiles; ++j) {
                     const int jn = j + AHEAD;
                     const bool more = jn < n_tiles;
-                    // one look at the next Y2 tile before the hand-over; ACC1(j) never waits for it
-                    const bool y2_ready = more && mbar_test_wait(bar(Y2_FULL + (jn & 1)), (jn >> 1) & 1);
                     if (MODE == DKV && j + 1 < n_tiles) wait(T1_ISSUED, j & 1, BW_T1FULL);
                     wait(DS_DONE + (j & 1), (j >> 1) & 1, BW_DSDONE);
                     if (!ok) break;
                     tc_fence_after();
                     acc1(j);
-                    if (!y2_ready) tc_commit(bar(Y1_EMPTY + j % kY1Stages));
+                    tc_commit(bar(Y1_EMPTY + j % kY1Stages));       // at once: the next K tile waits for this stage
                     if (more) {
-                        if (!y2_ready) wait(Y2_FULL + (jn & 1), (jn >> 1) & 1, BW_YFULL);
+                        wait(Y2_FULL + (jn & 1), (jn >> 1) & 1, BW_YFULL);
                         if (!ok) break;
                         t2(jn);
                         tc_commit(bar(T2_FULL + (jn & 1)));
                         tc_commit(bar(Y2_EMPTY + (jn & 1)));    // dQ modes: V is read here only; dK/dV: the first of two arrivals
                     }
-                    if (y2_ready) tc_commit(bar(Y1_EMPTY + j % kY1Stages));
                 }
             }
             if (ok) tc_commit(bar(ACC_FULL));
