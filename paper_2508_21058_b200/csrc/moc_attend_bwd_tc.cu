@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
         const int r = threadIdx.x & 127;              // row of the stationary tile = TMEM lane
         const int half = warp >> 2;
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-        int qi = -1, slot = 0;
+        int qi = -1, slot = 0, n_sel = 0;             // n_sel: routed picks of the query (anchor mode)
         float lse2 = INFINITY, dlt = 0.f;             // dQ modes: this lane's query
         if (MODE != DKV) {
             if (r < rows) {
@@ -203,6 +203,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 }
                 lse2 = p.lse[(size_t)h * p.L + qi] * kLog2e;
                 dlt = p.delta[(size_t)h * p.L + qi];
+                if (MODE == DQ_ANCHOR) {               // picks come first, -1 padding after them
+                    const int32_t *sel = p.sel + ((size_t)h * p.L + qi) * p.k;
+                    for (int s = 0; s < p.k; ++s) n_sel += sel[s] >= 0;
+                }
             }
             // stage the item's rows, one half Q and the other dO: consecutive threads take consecutive 16-byte pieces
             int *s_row = reinterpret_cast<int *>(&s_ld[0][0][0]);
@@ -345,20 +349,27 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     if (qi >= 0) store_row(p.part + (((size_t)h * p.L + qi) * p.k + slot) * D + ch * 32);
                 } else if (MODE == DQ_ANCHOR) {
                     if (qi >= 0) {
-                        for (int s = 0; s < p.k; ++s) {
-                            if (p.sel[((size_t)h * p.L + qi) * p.k + s] < 0) continue;
-                            const uint4 *src = reinterpret_cast<const uint4 *>(p.part + (((size_t)h * p.L + qi) * p.k + s) * D + ch * 32);
+                        // the routed partials of this query, four slots requested together
+                        const uint4 *src = reinterpret_cast<const uint4 *>(p.part + ((size_t)h * p.L + qi) * p.k * D + ch * 32);
+                        for (int s0 = 0; s0 < n_sel; s0 += 4) {
+                            uint4 raw[4][4];
 #pragma unroll
-                            for (int q4 = 0; q4 < 4; ++q4) {
-                                const uint4 raw = __ldcg(src + q4);
-                                const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+                            for (int u = 0; u < 4; ++u)
 #pragma unroll
-                                for (int y = 0; y < 4; ++y) {
-                                    const float2 f = __bfloat1622float2(b[y]);
-                                    acc[q4 * 8 + 2 * y] += f.x;
-                                    acc[q4 * 8 + 2 * y + 1] += f.y;
+                                for (int q4 = 0; q4 < 4; ++q4)
+                                    raw[u][q4] = s0 + u < n_sel ? __ldcg(src + (size_t)(s0 + u) * (D / 8) + q4) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                                for (int q4 = 0; q4 < 4; ++q4) {
+                                    const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&raw[u][q4]);
+#pragma unroll
+                                    for (int y = 0; y < 4; ++y) {
+                                        const float2 f = __bfloat1622float2(b[y]);
+                                        acc[q4 * 8 + 2 * y] += f.x;
+                                        acc[q4 * 8 + 2 * y + 1] += f.y;
+                                    }
                                 }
-                            }
                         }
                         store_row(p.dQ + ((size_t)h * p.L + qi) * D + ch * 32);
                     }
