@@ -130,7 +130,10 @@ __device__ __forceinline__ int chunks_in_reach(const RouteParams &p, int t) {
     return p.causal ? p.tok_chunk[min(p.L, (t + 1) * kRtRows) - 1] : p.C;
 }
 
-template <int D, int KMAX, int NG>
+// FEW (at most 32 padded chunks, k <= 8): the three descriptor terms form one B operand of 3 c_pad rows, so a
+// tile costs one MMA chain instead of three (an MMA costs the same for any N <= 128); the selection adds the
+// three column groups and lets every candidate in reach sink through the sorted list in one pass.
+template <int D, int KMAX, int NG, bool FEW>
 __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
                                                                  const __grid_constant__ CUtensorMap tmD,
                                                                  const RouteParams p) {
@@ -219,7 +222,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                         for (int term = 0; term < 3; ++term)
 #pragma unroll
                             for (int sub = 0; sub < SUB; ++sub)
-                                tma_load_2d(sD + (term * SUB + sub) * d_sub_bytes, &tmD, sub * 64,
+                                tma_load_2d(sD + (sub * 3 + term) * d_sub_bytes, &tmD, sub * 64,
                                             (h * 3 + term) * p.c_pad + (resident ? 0 : sb * p.sb_rows), bar(D_FULL));
                         ++dn;
                         res_sb = sb;
@@ -247,7 +250,8 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             const uint64_t q_desc0 = smem_desc_sw128(sQ, 16, 1024);
             uint64_t d_term[3 * SUB];
 #pragma unroll
-            for (int x = 0; x < 3 * SUB; ++x) d_term[x] = smem_desc_sw128(sD + x * d_sub_bytes, 16, 1024);
+            for (int x = 0; x < 3 * SUB; ++x)            // the three terms of a 64-column slice lie one after another
+                d_term[x] = smem_desc_sw128(sD + ((x % SUB) * 3 + x / SUB) * d_sub_bytes, 16, 1024);
             int res_sb = -1, dn = 0;
             int nacc_total[NG];
 #pragma unroll
@@ -277,6 +281,15 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                     RTRACE(3000 + (u - u0) * 4 + 1);
                     const int rows_sb = max(16, min(min(p.sb_rows, p.c_pad - sb * p.sb_rows), (reach - sb * p.sb_rows + 15) & ~15));
                     const uint64_t qd = q_desc0 + (uint64_t)(st * (Q_TILE_BYTES >> 4));
+                    if (FEW) {
+                        // one chain: B = the 3 c_pad rows (hi, mid, lo terms) of the block, three column groups out
+                        const uint32_t idesc = idesc_bf16_f32(128, 3 * p.c_pad, 0, 0);
+                        const uint32_t acc = tmem + buf * ACC_COLS;
+#pragma unroll
+                        for (int ks = 0; ks < D / 16; ++ks)
+                            mma_ss(acc, qd + (((ks >> 2) * Q_SUB_BYTES + (ks & 3) * 32) >> 4),
+                                   d_term[ks >> 2] + (((ks & 3) * 32) >> 4), idesc, ks != 0);
+                    } else
                     for (int n0 = 0; n0 < rows_sb; n0 += 128) {
                         const int n = min(128, rows_sb - n0);
                         const uint32_t idesc = idesc_bf16_f32(128, n, 0, 0);
@@ -317,7 +330,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
         bool ok = true;
         auto group_sync = [&]() {     // all 128 threads of the group, bounded
             mbar_arrive(bar(GROUP + sg));
-            bool o = mbar_wait(bar(GROUP + sg), ngs & 1, abort_flag, p.status, RW_GROUP);
+            bool o = mbar_wait_spin(bar(GROUP + sg), ngs & 1, abort_flag, p.status, RW_GROUP);   // polled: a parked thread wakes late
             ++ngs;
             return o;
         };
@@ -364,13 +377,57 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             top.init();
             [[maybe_unused]] float kth = -INFINITY;
             for (int sb = 0; ok && sb < n_sb; ++sb) {
-                ok = mbar_wait(bar(ACC_FULL + sg), nacc & 1, abort_flag, p.status, RW_ACCFULL);
+                ok = mbar_wait_spin(bar(ACC_FULL + sg), nacc & 1, abort_flag, p.status, RW_ACCFULL);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ++nacc;
                 if (gt == 0) RTRACE(tn + 1);
                 tc_fence_after();
                 const int rows_sb = max(16, min(min(p.sb_rows, p.c_pad - sb * p.sb_rows), (reach - sb * p.sb_rows + 15) & ~15));
+                if (FEW) {
+                    // at most 32 chunks, all in this block.  Candidate bits: a real chunk, not an anchor, strictly
+                    // earlier if causal.  The scores of the chunks in the tile's reach come eight at a time, each the
+                    // sum of its three terms (hi, mid, lo, in that order), and sink through the sorted list (strict
+                    // '>' keeps equal scores in arrival order, which is ascending chunk index).
+                    uint32_t cand = ~aw_next;
+                    const int lim = min(p.C, p.causal ? ci : p.C);
+                    cand = lim <= 0 ? 0u : (lim >= 32 ? cand : (cand & ((1u << lim) - 1u)));
+                    if (!live) cand = 0u;
+                    uint32_t a[8], b[8], c3[8];
+                    tmem_ld8(acc, a);
+                    tmem_ld8(acc + p.c_pad, b);
+                    tmem_ld8(acc + 2 * p.c_pad, c3);
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        if (g * 8 < rows_sb) {
+                            tmem_wait_ld();
+                            float f[8];
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) f[c] = (__uint_as_float(a[c]) + __uint_as_float(b[c])) + __uint_as_float(c3[c]);
+                            if (g < 3 && (g + 1) * 8 < rows_sb) {       // the next eight, in flight behind this group's work
+                                tmem_ld8(acc + (g + 1) * 8, a);
+                                tmem_ld8(acc + p.c_pad + (g + 1) * 8, b);
+                                tmem_ld8(acc + 2 * p.c_pad + (g + 1) * 8, c3);
+                            }
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) {
+                                float cv = ((cand >> (g * 8 + c)) & 1u) ? f[c] : -INFINITY;
+                                int cj = g * 8 + c;
+#pragma unroll
+                                for (int x = 0; x < KR; ++x) {
+                                    const bool up = cv > top.s[x];
+                                    const float ts = top.s[x];
+                                    const int tj = top.j[x];
+                                    top.s[x] = up ? cv : ts;
+                                    top.j[x] = up ? cj : tj;
+                                    cv = up ? ts : cv;
+                                    cj = up ? tj : cj;
+                                }
+                            }
+                        }
+                    }
+                    if (gt == 0) RTRACE(tn + 8);
+                } else
                 for (int cc = 0; cc < rows_sb; cc += 32) {
                     uint32_t v[32];
                     tmem_ld32(acc + cc, v);
@@ -602,15 +659,16 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         CUtensorMap tmQ, tmD;
         if (int r = make_tmap_2d_bf16(&tmQ, Q, (uint64_t)p->H * p->L, D, kRtRows)) return r;
         if (int r = make_tmap_2d_bf16(&tmD, desc3, (uint64_t)p->H * 3 * p->c_pad, D, (uint32_t)a.d_rows)) return r;
-#define MOC_ROUTE_CASE(KM, NG)                                                                                          \
+#define MOC_ROUTE_CASE(KM, NG, FW)                                                                                          \
     do {                                                                                                                \
-        MOC_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel<D, KM, NG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        route_tc_kernel<D, KM, NG><<<grid, rt_threads(NG), smem, s>>>(tmQ, tmD, a);                                     \
+        MOC_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel<D, KM, NG, FW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        route_tc_kernel<D, KM, NG, FW><<<grid, rt_threads(NG), smem, s>>>(tmQ, tmD, a);                                     \
     } while (0)
-        if (p->k <= 4) { if (ng == 4) MOC_ROUTE_CASE(4, 4); else MOC_ROUTE_CASE(4, 2); }
-        else if (p->k <= 8) { if (ng == 4) MOC_ROUTE_CASE(8, 4); else MOC_ROUTE_CASE(8, 2); }
-        else if (p->k <= 64) MOC_ROUTE_CASE(64, 2);
-        else MOC_ROUTE_CASE(512, 2);
+        const bool few = p->c_pad <= 32 && p->k <= 8;       // then ng == 4 as well
+        if (p->k <= 4) { if (few) MOC_ROUTE_CASE(4, 4, true); else if (ng == 4) MOC_ROUTE_CASE(4, 4, false); else MOC_ROUTE_CASE(4, 2, false); }
+        else if (p->k <= 8) { if (few) MOC_ROUTE_CASE(8, 4, true); else if (ng == 4) MOC_ROUTE_CASE(8, 4, false); else MOC_ROUTE_CASE(8, 2, false); }
+        else if (p->k <= 64) MOC_ROUTE_CASE(64, 2, false);
+        else MOC_ROUTE_CASE(512, 2, false);
 #undef MOC_ROUTE_CASE
         MOC_LAUNCH_CHECK();
     }
