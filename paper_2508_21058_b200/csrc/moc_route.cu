@@ -154,7 +154,10 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     const uint32_t sD = sbase;
     const uint32_t sQ = sD + ((3 * SUB * d_sub_bytes + 1023) & ~1023);
     int *hist_base = reinterpret_cast<int *>(gbase + (sQ - sbase) + p.q_stages * Q_TILE_BYTES);
-    int *s_cap = hist_base + NG * p.C;                                   // copy of cap_off[0 .. C)
+    // per selection group: one histogram of C counters, or (deferred list append) two alternating histograms and
+    // two alternating tables of list bases
+    const int hist_ints = (KMAX <= 8 && p.C <= 256 ? 4 : 1) * p.C;
+    int *s_cap = hist_base + NG * hist_ints;                             // copy of cap_off[0 .. C)
     uint16_t *s_reach = reinterpret_cast<uint16_t *>(s_cap + p.C);      // chunks in reach of each of this CTA's units
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     constexpr int Q_FULL = 0, Q_EMPTY = kMaxStages, D_FULL = 2 * kMaxStages, D_EMPTY = D_FULL + 1, ACC_FULL = D_FULL + 2,
@@ -187,10 +190,12 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     // this CTA's units: a contiguous range of 128-query tiles of ONE head (u counts tiles of that head),
     // so its descriptor block never changes while it fits in shared memory
     const int h = blockIdx.x / p.ctas_per_head, part = blockIdx.x % p.ctas_per_head;
-    const int u0 = (int)((long long)p.tiles_per_head * part / p.ctas_per_head);
-    const int u1 = (int)((long long)p.tiles_per_head * (part + 1) / p.ctas_per_head);
+    // the head's tiles are dealt round-robin to its CTAs: a tile's work grows with the chunks in its causal
+    // reach, i.e. with its position, and contiguous ranges would leave the last CTA of a head the slowest
+    const int nu = (p.tiles_per_head - part + p.ctas_per_head - 1) / p.ctas_per_head;      // units of this CTA
+    auto unit_of = [&](int n) { return part + n * p.ctas_per_head; };
     for (int x = threadIdx.x; x < p.C; x += kRtThreads) s_cap[x] = p.cap_off[x];
-    for (int x = threadIdx.x; x < u1 - u0; x += kRtThreads) s_reach[x] = (uint16_t)chunks_in_reach(p, u0 + x);
+    for (int x = threadIdx.x; x < nu; x += kRtThreads) s_reach[x] = (uint16_t)chunks_in_reach(p, unit_of(x));
     __syncthreads();
     constexpr int ACC_COLS = 512 / NG;   // TMEM columns per accumulator (NG = 4 only with sb_rows <= 128)
     const bool resident = p.d_rows == p.c_pad;       // every chunk's descriptor is held: loaded once, two MMA issuers
@@ -202,8 +207,9 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             prefetch_tensormap(&tmD);
             int res_sb = -1, qn = 0, dn = 0;
             bool ok = true;
-            for (int u = u0; ok && u < u1; ++u) {
-                const int reach = s_reach[u - u0], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
+            for (int n = 0; ok && n < nu; ++n) {
+                const int u = unit_of(n);
+                const int reach = s_reach[n], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
                     if (sb == 0) {
                         const int st = qn % p.q_stages;
@@ -257,11 +263,11 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
 #pragma unroll
             for (int x = 0; x < NG; ++x) nacc_total[x] = 0;
             bool ok = true;
-            for (int u = u0 + first; ok && u < u1; u += stride) {
-                const int reach = s_reach[u - u0], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
-                const int buf = (u - u0) % NG;
-                const int qn = u - u0, st = qn % p.q_stages;
-                RTRACE(3000 + (u - u0) * 4 + 3);
+            for (int n = first; ok && n < nu; n += stride) {
+                const int reach = s_reach[n], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
+                const int buf = n % NG;
+                const int qn = n, st = qn % p.q_stages;
+                RTRACE(3000 + n * 4 + 3);
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
                     if (sb == 0) {
                         ok = mbar_wait(bar(Q_FULL + st), (qn / p.q_stages) & 1, abort_flag, p.status, RW_QFULL);
@@ -273,12 +279,12 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                         ++dn;
                         res_sb = sb;
                     }
-                    RTRACE(3000 + (u - u0) * 4 + 0);
+                    RTRACE(3000 + n * 4 + 0);
                     const int uses = nacc_total[buf];
                     ok = mbar_wait(bar(ACC_EMPTY + buf), (uses & 1) ^ 1, abort_flag, p.status, RW_ACCEMPTY);
                     if (!ok) break;
                     tc_fence_after();
-                    RTRACE(3000 + (u - u0) * 4 + 1);
+                    RTRACE(3000 + n * 4 + 1);
                     const int rows_sb = max(16, min(min(p.sb_rows, p.c_pad - sb * p.sb_rows), (reach - sb * p.sb_rows + 15) & ~15));
                     const uint64_t qd = q_desc0 + (uint64_t)(st * (Q_TILE_BYTES >> 4));
                     if (FEW) {
@@ -304,14 +310,14 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                         }
                     }
                     tc_commit(bar(ACC_FULL + buf));
-                    RTRACE(3000 + (u - u0) * 4 + 2);
+                    RTRACE(3000 + n * 4 + 2);
                     ++nacc_total[buf];
                     // streamed blocks: the next step, if it needs another block, may overwrite this one once
                     // these MMAs are done
                     if (!resident) {
                         int nsb = sb + 1;
                         bool more = true;
-                        if (nsb >= n_sb) { nsb = 0; more = u + 1 < u1; }
+                        if (nsb >= n_sb) { nsb = 0; more = n + 1 < nu; }
                         if (more && nsb != sb) tc_commit(bar(D_EMPTY));
                     }
                 }
@@ -320,12 +326,12 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
         }
     } else if (warp < 2 + 4 * NG) {
         // ------------------------------------------------------------ selection groups
-        const int sg = (warp - 2) >> 2;                        // group (warps 2-5, 6-9, ...); its units are those with (u - u0) % NG == sg
+        const int sg = (warp - 2) >> 2;                        // group (warps 2-5, 6-9, ...); its units are those with n % NG == sg
         const int gt = threadIdx.x - 64 - sg * 128;            // thread within the group
         const int r = (warp & 3) * 32 + lane;                  // TMEM lane = query row of the tile
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t acc = tmem + sg * ACC_COLS + lane_off;
-        int *hist = hist_base + sg * p.C;
+        int *hist = hist_base + sg * hist_ints;
         int nacc = 0, ngs = 0;
         bool ok = true;
         auto group_sync = [&]() {     // all 128 threads of the group, bounded
@@ -341,37 +347,49 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
         const bool deferred = SMALL && p.C <= 256;
         struct Pending { int h, i, j[KR], rank[KR], base0, base1; bool live, open; } pend;
         pend.open = false; pend.live = false; pend.h = 0; pend.i = 0; pend.base0 = 0; pend.base1 = 0;
-        auto finish_pending = [&]() {          // bases into the histogram, then the list entries
-            if (gt < p.C) hist[gt] = pend.base0;
-            if (gt + 128 < p.C) hist[gt + 128] = pend.base1;
-            bool o = group_sync();
-            if (o && pend.live) {
+        // Deferred append, one group barrier per unit.  Unit n uses histogram n & 1 and base table n & 1:
+        //   before the barrier: the bases that unit n - 1's range-reserving atomics returned go into the table,
+        //     and unit n's picks take their tile-local ranks from the histogram;
+        //   after it: unit n - 1's list entries are written (base + rank), and each thread reserves, for the
+        //     chunk it owns, unit n's range in that chunk's list and clears the counter it has just read.
+        // The same histogram and table are next written two units later, with unit n + 1's barrier in between.
+        int ndef = 0;                          // units this group has appended so far
+        auto write_bases = [&]() {
+            int *baseb = hist + (2 + (ndef & 1)) * p.C;
+            if (gt < p.C) baseb[gt] = pend.base0;
+            if (gt + 128 < p.C) baseb[gt + 128] = pend.base1;
+        };
+        auto write_entries = [&]() {
+            const int *baseb = hist + (2 + (ndef & 1)) * p.C;
+            if (pend.live) {
                 int32_t *list = p.qlist + (size_t)pend.h * p.cap_total;
 #pragma unroll
-                for (int x = 0; x < KR; ++x)
-                    if (x < p.k && pend.j[x] >= 0) list[s_cap[pend.j[x]] + hist[pend.j[x]] + pend.rank[x]] = pend.i * p.k + x;
+                for (int x = 0; x < KR; ++x)           // j holds (chunk << 8 | rank) here: a tile has 128 rows
+                    if (x < p.k && pend.j[x] >= 0) list[s_cap[pend.j[x] >> 8] + baseb[pend.j[x] >> 8] + (pend.j[x] & 255)] = pend.i * p.k + x;
             }
-            o = o && group_sync();             // entries written before the histogram is reused
-            pend.open = false;
-            return o;
         };
+        if (deferred) {
+            for (int x = gt; x < 2 * p.C; x += 128) hist[x] = 0;
+            ok = group_sync();
+        }
         int nx_ci = 0;
         uint32_t nx_aw = 0u;
-        if (u0 + sg < u1) {
-            const int i0 = (u0 + sg) * kRtRows + r;
+        if (sg < nu) {
+            const int i0 = unit_of(sg) * kRtRows + r;
             nx_ci = i0 < p.L ? p.tok_chunk[i0] : 0;
             nx_aw = i0 < p.L ? p.anc_bits[(size_t)nx_ci * p.words] : 0u;
         }
-        for (int u = u0 + sg; ok && u < u1; u += NG) {
-            const int reach = s_reach[u - u0], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
+        for (int n = sg; ok && n < nu; n += NG) {
+            const int u = unit_of(n);
+            const int reach = s_reach[n], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
             const int i = u * kRtRows + r;
             const bool live = i < p.L;
             const int ci = nx_ci;
             const uint32_t aw_next = nx_aw;
-            const int i2 = (u + NG) * kRtRows + r;
-            const bool live2 = u + NG < u1 && i2 < p.L;
+            const int i2 = unit_of(n + NG) * kRtRows + r;
+            const bool live2 = n + NG < nu && i2 < p.L;
             if (live2) nx_ci = p.tok_chunk[i2];       // the next unit's chunk, loaded a unit ahead (its anchor word follows below)
-            [[maybe_unused]] const int tn = 100 + sg * 1000 + ((u - u0) / NG) * 16;
+            [[maybe_unused]] const int tn = 100 + sg * 1000 + (n / NG) * 16;
             if (gt == 0) RTRACE(tn + 0);
             TopK<KMAX> top;
             top.init();
@@ -515,7 +533,35 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                     }
                 }
             }
-            if (pend.open) { ok = finish_pending(); if (!ok) break; }
+            if (deferred) {
+                int *cntb = hist + (ndef & 1) * p.C;
+                if (pend.open) write_bases();
+                int njr[KR];                           // chunk << 8 | tile-local rank, or -1
+#pragma unroll
+                for (int x = 0; x < KR; ++x) {
+                    const int j = (live && x < p.k) ? top.j[x] : -1;
+                    njr[x] = j >= 0 ? ((j << 8) | atomicAdd(&cntb[j], 1)) : -1;
+                }
+                ok = group_sync();
+                if (!ok) break;
+                if (gt == 0) RTRACE(tn + 3);
+                if (pend.open) write_entries();
+                pend.base0 = 0; pend.base1 = 0;
+                if (gt < p.C) {
+                    const int n = cntb[gt];
+                    if (n) { pend.base0 = atomicAdd(&p.cnt[h * p.C + gt], n); cntb[gt] = 0; }
+                }
+                if (gt + 128 < p.C) {
+                    const int n = cntb[gt + 128];
+                    if (n) { pend.base1 = atomicAdd(&p.cnt[h * p.C + gt + 128], n); cntb[gt + 128] = 0; }
+                }
+#pragma unroll
+                for (int x = 0; x < KR; ++x) pend.j[x] = njr[x];
+                pend.h = h; pend.i = i; pend.live = live; pend.open = true;
+                ++ndef;
+                if (gt == 0) RTRACE(tn + 5);
+                continue;
+            }
             if (gt == 0) RTRACE(tn + 3);
             // tile-local rank of every pick (shared-memory histogram), then one global atomic per picked
             // chunk reserves this tile's range in that chunk's list
@@ -541,12 +587,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             ok = group_sync();
             if (!ok) break;
             if (gt == 0) RTRACE(tn + 4);
-            if (deferred) {
-                pend.base0 = 0; pend.base1 = 0;
-                if (gt < p.C && hist[gt]) pend.base0 = atomicAdd(&p.cnt[h * p.C + gt], hist[gt]);
-                if (gt + 128 < p.C && hist[gt + 128]) pend.base1 = atomicAdd(&p.cnt[h * p.C + gt + 128], hist[gt + 128]);
-                pend.h = h; pend.i = i; pend.live = live; pend.open = true;   // each thread re-reads only its own counts
-            } else {
+            {
                 for (int x = gt; x < p.C; x += 128) {
                     const int n = hist[x];
                     if (n) hist[x] = atomicAdd(&p.cnt[h * p.C + x], n);
@@ -571,7 +612,10 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             }
             if (gt == 0) RTRACE(tn + 5);
         }
-        if (ok && pend.open) finish_pending();
+        if (ok && pend.open) {                 // the last unit's entries
+            write_bases();
+            if (group_sync()) write_entries();
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -652,7 +696,7 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         // a quarter of TMEM and the top-k list lives in registers; two otherwise.
         const int ng = (a.sb_rows <= 128 && p->k <= 8) ? 4 : 2;
         // one histogram per group, the list offsets, and one byte per unit of a CTA
-        const size_t hist = (ng + 1) * sizeof(int) * (size_t)p->C + 2 * (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
+        const size_t hist = (ng * (p->k <= 8 && p->C <= 256 ? 4 : 1) + 1) * sizeof(int) * (size_t)p->C + 2 * (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
         if (d_block + q_tile + hist > budget) return MOC_ERR_SHAPE;
         a.q_stages = (int)std::min<size_t>(4, (budget - d_block - hist) / q_tile);
         const size_t smem = 1024 + d_block + a.q_stages * q_tile + hist;
