@@ -9,8 +9,8 @@
 // accumulated in fp32 in TMEM: every product is exact, only the fp32 accumulation rounds.
 //
 // route_prep_kernel   splits the descriptors, clears the pick counters and the status words.
-// route_tc_kernel     H x (SMs / H) CTAs, each owning a contiguous range of 128-query tiles
-//                     ("units") of one head:
+// route_tc_kernel     H x (SMs / H) CTAs; the 128-query tiles ("units") of a head are dealt round-robin
+//                     to the head's CTAs:
 //     warp 0      TMA producer: Q tiles (ring of stages) and the head's descriptor block;
 //     warps 1, 10 MMA issuers: 3 x d/16 MMAs per 128 chunks into one of two TMEM accumulators
 //                 (warp 1 the even units, warp 10 the odd ones);
@@ -22,6 +22,9 @@
 //   The head's descriptors stay in shared memory for the CTA's lifetime (C <= 192) and are scored
 //   in steps of at most 128 chunks; with more chunks they are streamed in blocks of 128 and warp 1
 //   alone issues.
+//   With at most 32 padded chunks (and k <= 8) the three terms of the split descriptors form one MMA
+//   operand, the selection adds the three column groups and every candidate sinks through the sorted
+//   list in one pass (template parameter FEW).
 // route_tiles_kernel  running count of attention tiles over (head, chunk) from the pick counts;
 // route_items_kernel  the routed attention work items (one per 256 picks of a chunk).
 // Every mbarrier wait is bounded; a wait that runs out flags the workspace status word.
@@ -187,8 +190,8 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     volatile int *abort_flag = &s_abort;
     if (threadIdx.x == 0) RTRACE(0);
 
-    // this CTA's units: a contiguous range of 128-query tiles of ONE head (u counts tiles of that head),
-    // so its descriptor block never changes while it fits in shared memory
+    // this CTA's units: 128-query tiles of ONE head (u counts tiles of that head), so its descriptor block
+    // never changes while it fits in shared memory
     const int h = blockIdx.x / p.ctas_per_head, part = blockIdx.x % p.ctas_per_head;
     // the head's tiles are dealt round-robin to its CTAs: a tile's work grows with the chunks in its causal
     // reach, i.e. with its position, and contiguous ranges would leave the last CTA of a head the slowest
