@@ -153,6 +153,10 @@ def workload(name: str, seed: int = 0) -> Workload:
         return Workload(name, 2, 128, make_layout(3, 16, 40, 24), 12, 1, 1, seed=seed)
     if name == "mini7":   # k = 70 of up to 122 candidates, d = 64: the long-list selection path, streamed descriptor blocks
         return Workload(name, 2, 64, make_layout(3, 16, 80, 16), 70, 1, 1, seed=seed)
+    if name == "mini8":   # few chunks (one scoring operand for the three descriptor terms) with k above 4
+        return Workload(name, 2, 128, make_layout(2, 32, 10, 160), 6, 1, 1, seed=seed)
+    if name == "mini9":   # more than 32 chunks with k <= 4: the selection by extraction rounds, short list
+        return Workload(name, 2, 64, make_layout(3, 16, 14, 96), 4, 1, 1, seed=seed)
     if name == "midi2":   # multi-shot with true 1560-token frames, small enough for a full oracle pass
         return Workload(name, 2, 128, make_layout(2, 256, 4, 1560), 3, 1, 1, seed=seed)
     raise KeyError(name)
