@@ -38,7 +38,11 @@ using namespace tc;
 // clock64() into a slot of g_trace, read back with moc_trace_read().  Compiled out otherwise.
 #ifdef MOC_TRACE
 __device__ long long g_trace[8192];
-#define TRACE_CTA (blockIdx.x == (ROUTED ? 5000 : 70) && (ROUTED || blockIdx.y == 3))
+// -DMOC_TRACE_PASS=1 stamps the routed pass only, =0 the anchor pass only; by default both write (the anchor pass last)
+#ifndef MOC_TRACE_PASS
+#define MOC_TRACE_PASS 2
+#endif
+#define TRACE_CTA (blockIdx.x == (ROUTED ? 5000 : 70) && (ROUTED || blockIdx.y == 3) && (MOC_TRACE_PASS == 2 || (int)ROUTED == MOC_TRACE_PASS))
 #define TRACE(slot) do { if (TRACE_CTA) g_trace[(slot)] = clock64(); } while (0)
 #else
 #define TRACE(slot) ((void)0)
@@ -507,12 +511,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 tc_fence_after();
                 if (steps > half) issue_pv(g, st, half, steps, true);
                 TRACE(2100 + g * 1000 + jt * 8 + 4);
-                tc_commit(bar(V_EMPTY + st));
+                // a commit between two groups of MMAs leaves the pipe idle: the next S goes out first, then all commits
                 if (more) {
                     issue_qk(g, sn, valid_next);
                     tc_commit(bar(S_FULL + g));
+                    tc_commit(bar(V_EMPTY + st));
                     tc_commit(bar(K_EMPTY + sn));
                 } else {
+                    tc_commit(bar(V_EMPTY + st));
                     tc_commit(bar(O_FULL + g));
                 }
                 TRACE(2100 + g * 1000 + jt * 8 + 5);
