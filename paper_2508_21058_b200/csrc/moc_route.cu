@@ -62,7 +62,7 @@ struct TopK {
     float s[KMAX];
     int j[KMAX];
     __device__ __forceinline__ void init() {
-#pragma unroll(KMAX <= 8 ? KMAX : 1)
+#pragma unroll(KMAX <= 64 ? KMAX : 1)
         for (int x = 0; x < KMAX; ++x) { s[x] = -INFINITY; j[x] = -1; }
     }
     // candidates arrive in ascending chunk index, so strict '>' keeps equal scores in index order
@@ -253,8 +253,9 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
         // With a resident descriptor block, warp 1 serves the even units and the last warpgroup's first warp
         // the odd ones (each its own accumulators), so one issuer's waits and instruction overhead hide behind the other's
         // MMAs; when blocks are streamed, warp 1 serves every unit and follows the reloads.
-        const int first = warp == 1 ? 0 : 1, stride = resident ? 2 : 1;
-        if (lane == 0 && (warp == 1 || resident)) {
+        const bool dual = resident && NG > 1;          // one selection group has one accumulator: one issuer
+        const int first = warp == 1 ? 0 : 1, stride = dual ? 2 : 1;
+        if (lane == 0 && (warp == 1 || dual)) {
             // descriptors are built once: issuing an MMA should cost this thread a few integer instructions
             const uint64_t q_desc0 = smem_desc_sw128(sQ, 16, 1024);
             uint64_t d_term[3 * SUB];
@@ -343,11 +344,11 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             ++ngs;
             return o;
         };
-        constexpr bool SMALL = KMAX <= 8;
+        constexpr bool SMALL = KMAX <= 64;      // the sorted list lives in registers (64 entries: one selection group)
         constexpr int KR = SMALL ? KMAX : 1;
         // With few chunks the list append of a unit is finished after the next unit's selection, so the
         // round trip of the range-reserving atomics is hidden; `pend` is the unit whose append is open.
-        const bool deferred = SMALL && p.C <= 256;
+        const bool deferred = KMAX <= 8 && p.C <= 256;
         struct Pending { int h, i, j[KR], rank[KR], base0, base1; bool live, open; } pend;
         pend.open = false; pend.live = false; pend.h = 0; pend.i = 0; pend.base0 = 0; pend.base1 = 0;
         // Deferred append, one group barrier per unit.  Unit n uses histogram n & 1 and base table n & 1:
@@ -696,8 +697,8 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         a.ctas_per_head = std::max(1, std::min(p->n_sm / p->H, a.tiles_per_head));
         const unsigned grid = (unsigned)(p->H * a.ctas_per_head);
         // Four selection groups (more warps to hide the selection's latencies) when an accumulator fits
-        // a quarter of TMEM and the top-k list lives in registers; two otherwise.
-        const int ng = (a.sb_rows <= 128 && p->k <= 8) ? 4 : 2;
+        // a quarter of TMEM and k <= 8; one when the 64-entry list takes nearly all of a thread's registers; two otherwise.
+        const int ng = (a.sb_rows <= 128 && p->k <= 8) ? 4 : (p->k > 32 && p->k <= 64) ? 1 : 2;
         // one histogram per group, the list offsets, and one byte per unit of a CTA
         const size_t hist = (ng * (p->k <= 8 && p->C <= 256 ? 4 : 1) + 1) * sizeof(int) * (size_t)p->C + 2 * (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
         if (d_block + q_tile + hist > budget) return MOC_ERR_SHAPE;
@@ -714,7 +715,9 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         const bool few = p->c_pad <= 32 && p->k <= 8;       // then ng == 4 as well
         if (p->k <= 4) { if (few) MOC_ROUTE_CASE(4, 4, true); else if (ng == 4) MOC_ROUTE_CASE(4, 4, false); else MOC_ROUTE_CASE(4, 2, false); }
         else if (p->k <= 8) { if (few) MOC_ROUTE_CASE(8, 4, true); else if (ng == 4) MOC_ROUTE_CASE(8, 4, false); else MOC_ROUTE_CASE(8, 2, false); }
-        else if (p->k <= 64) MOC_ROUTE_CASE(64, 2, false);
+        else if (p->k <= 16) MOC_ROUTE_CASE(16, 2, false);
+        else if (p->k <= 32) MOC_ROUTE_CASE(32, 2, false);
+        else if (p->k <= 64) MOC_ROUTE_CASE(64, 1, false);
         else MOC_ROUTE_CASE(512, 2, false);
 #undef MOC_ROUTE_CASE
         MOC_LAUNCH_CHECK();

@@ -157,6 +157,10 @@ def workload(name: str, seed: int = 0) -> Workload:
         return Workload(name, 2, 128, make_layout(2, 32, 10, 160), 6, 1, 1, seed=seed)
     if name == "mini9":   # more than 32 chunks with k <= 4: the selection by extraction rounds, short list
         return Workload(name, 2, 64, make_layout(3, 16, 14, 96), 4, 1, 1, seed=seed)
+    if name == "mini10":  # k = 20 of up to 80 candidates: the largest register-resident list
+        return Workload(name, 2, 128, make_layout(2, 16, 40, 32), 20, 1, 1, seed=seed)
+    if name == "mini11":  # k = 40 of up to 120 candidates: the 64-entry register list, one selection group
+        return Workload(name, 2, 64, make_layout(2, 16, 60, 32), 40, 1, 1, seed=seed)
     if name == "midi2":   # multi-shot with true 1560-token frames, small enough for a full oracle pass
         return Workload(name, 2, 128, make_layout(2, 256, 4, 1560), 3, 1, 1, seed=seed)
     raise KeyError(name)

@@ -12,7 +12,7 @@ import parity_utils as PU
 
 pytestmark = pytest.mark.gpu
 
-SMALL = ["cfg0", "mini1", "mini2", "mini2t", "mini3", "mini4", "mini5", "mini6", "mini7", "mini8", "mini9", "midi2"]
+SMALL = ["cfg0", "mini1", "mini2", "mini2t", "mini3", "mini4", "mini5", "mini6", "mini7", "mini8", "mini9", "mini10", "mini11", "midi2"]
 
 
 def _forward_parity(name, scalar, rows_per_head=None):
@@ -81,7 +81,7 @@ def test_backward_small_scalar_kernels(name):
     _backward_parity(name, scalar=True)
 
 
-@pytest.mark.parametrize("name", ["cfg0", "mini1", "mini2", "mini2t", "mini3", "mini4", "mini5", "mini6", "mini7", "mini8", "mini9", "midi2"])
+@pytest.mark.parametrize("name", ["cfg0", "mini1", "mini2", "mini2t", "mini3", "mini4", "mini5", "mini6", "mini7", "mini8", "mini9", "mini10", "mini11", "midi2"])
 def test_backward_small(name):
     _backward_parity(name, scalar=False, n_rows=64 if name != "midi2" else 200)
 
