@@ -14,9 +14,10 @@
 //     warp 0      TMA producer: Q tiles (ring of stages) and the head's descriptor block;
 //     warps 1, 10 MMA issuers: 3 x d/16 MMAs per 128 chunks into one of two TMEM accumulators
 //                 (warp 1 the even units, warp 10 the odd ones);
-//     warps 2-5 / 6-9   two selection groups (even / odd units), one query per thread (TMEM
+//     warps 2-5 / 6-9   selection groups (one, two or four: the units in turn), one query per thread (TMEM
 //                 lane = query): read the scores 32 chunks at a time, drop non-candidates,
-//                 keep a sorted top-k in registers, then write sel_idx and append the picks
+//                 keep a sorted top-k in registers (at most 64 entries; more picks are taken in
+//                 passes of 64 over recomputed scores), then write sel_idx and append the picks
 //                 to the per-(head, chunk) query lists (tile-local ranks from a shared-memory
 //                 histogram, one global atomic per (tile, chunk) to reserve the range).
 //   The head's descriptors stay in shared memory for the CTA's lifetime (C <= 192) and are scored
@@ -62,27 +63,8 @@ struct TopK {
     float s[KMAX];
     int j[KMAX];
     __device__ __forceinline__ void init() {
-#pragma unroll(KMAX <= 64 ? KMAX : 1)
-        for (int x = 0; x < KMAX; ++x) { s[x] = -INFINITY; j[x] = -1; }
-    }
-    // candidates arrive in ascending chunk index, so strict '>' keeps equal scores in index order
-    __device__ __forceinline__ void push(float v, int idx, int k) {
-        if (KMAX <= 8) {
-            if (!(v > s[KMAX - 1])) return;
 #pragma unroll
-            for (int x = KMAX - 1; x >= 0; --x) {
-                bool shift = (x > 0) && (v > s[x > 0 ? x - 1 : 0]);
-                bool place = (v > s[x]) && !shift;
-                float ns = shift ? s[x > 0 ? x - 1 : 0] : (place ? v : s[x]);
-                int nj = shift ? j[x > 0 ? x - 1 : 0] : (place ? idx : j[x]);
-                s[x] = ns; j[x] = nj;
-            }
-        } else {
-            if (!(v > s[k - 1])) return;
-            int x = k - 1;
-            while (x > 0 && v > s[x - 1]) { s[x] = s[x - 1]; j[x] = j[x - 1]; --x; }
-            s[x] = v; j[x] = idx;
-        }
+        for (int x = 0; x < KMAX; ++x) { s[x] = -INFINITY; j[x] = -1; }
     }
 };
 
@@ -125,6 +107,7 @@ struct RouteParams {
     int sb_rows;            // chunks per scoring step (one accumulator's worth)
     int d_rows;             // descriptor rows per term held in shared memory: c_pad (resident) or sb_rows (streamed)
     int q_stages;
+    int n_pass;             // selection passes over a tile's scores: 64 picks each (the scores are recomputed per pass)
     size_t cap_total;
 };
 
@@ -213,8 +196,9 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             for (int n = 0; ok && n < nu; ++n) {
                 const int u = unit_of(n);
                 const int reach = s_reach[n], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
+                for (int rep = 0; ok && rep < p.n_pass; ++rep)
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
-                    if (sb == 0) {
+                    if (sb == 0 && rep == 0) {
                         const int st = qn % p.q_stages;
                         ok = mbar_wait(bar(Q_EMPTY + st), ((qn / p.q_stages) & 1) ^ 1, abort_flag, p.status, RW_QEMPTY);
                         if (!ok) break;
@@ -272,8 +256,9 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 const int buf = n % NG;
                 const int qn = n, st = qn % p.q_stages;
                 RTRACE(3000 + n * 4 + 3);
+                for (int rep = 0; ok && rep < p.n_pass; ++rep)
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
-                    if (sb == 0) {
+                    if (sb == 0 && rep == 0) {
                         ok = mbar_wait(bar(Q_FULL + st), (qn / p.q_stages) & 1, abort_flag, p.status, RW_QFULL);
                         if (!ok) break;
                     }
@@ -321,7 +306,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                     if (!resident) {
                         int nsb = sb + 1;
                         bool more = true;
-                        if (nsb >= n_sb) { nsb = 0; more = n + 1 < nu; }
+                        if (nsb >= n_sb) { nsb = 0; more = rep + 1 < p.n_pass || n + 1 < nu; }
                         if (more && nsb != sb) tc_commit(bar(D_EMPTY));
                     }
                 }
@@ -344,8 +329,8 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             ++ngs;
             return o;
         };
-        constexpr bool SMALL = KMAX <= 64;      // the sorted list lives in registers (64 entries: one selection group)
-        constexpr int KR = SMALL ? KMAX : 1;
+        // the sorted list of this pass's picks lives in registers (a 64-entry list leaves room for one selection group)
+        constexpr int KR = KMAX;
         // With few chunks the list append of a unit is finished after the next unit's selection, so the
         // round trip of the range-reserving atomics is hidden; `pend` is the unit whose append is open.
         const bool deferred = KMAX <= 8 && p.C <= 256;
@@ -395,6 +380,13 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             if (live2) nx_ci = p.tok_chunk[i2];       // the next unit's chunk, loaded a unit ahead (its anchor word follows below)
             [[maybe_unused]] const int tn = 100 + sg * 1000 + (n / NG) * 16;
             if (gt == 0) RTRACE(tn + 0);
+            // More than 64 picks are taken 64 at a time: every pass sees the tile's scores again (the issuer
+            // recomputes them) and considers only the chunks that come after the previous pass's last pick in
+            // the order of the result (score descending, then chunk index ascending).
+            [[maybe_unused]] float prev_s = INFINITY;
+            [[maybe_unused]] int prev_j = -1;
+            for (int pass = 0; ok && pass < p.n_pass; ++pass) {
+            const int kp = min(p.k - pass * 64, KMAX);      // picks of this pass
             TopK<KMAX> top;
             top.init();
             [[maybe_unused]] float kth = -INFINITY;
@@ -462,13 +454,20 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                     if (!live) cand = 0u;
                     tmem_wait_ld();
                     if (gt == 0) RTRACE(tn + 6);
-                    if (SMALL) {
+                    {
                         float f[32];
 #pragma unroll
                         for (int c = 0; c < 32; ++c) f[c] = ((cand >> c) & 1u) ? __uint_as_float(v[c]) : -INFINITY;
+                        if (KMAX == 64 && pass > 0) {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) {
+                                const bool after = f[c] < prev_s || (f[c] == prev_s && j0 + c > prev_j);
+                                f[c] = after ? f[c] : -INFINITY;
+                            }
+                        }
                         // up to k members of the block can enter the list: take them best first
 #pragma unroll 1
-                        for (int round = 0; round < p.k; ++round) {
+                        for (int round = 0; round < kp; ++round) {
                             float m8[4];
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
@@ -501,16 +500,13 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                                 }
                                 kth = top.s[0];
 #pragma unroll
-                                for (int x = 1; x < KR; ++x) kth = (x < p.k) ? top.s[x] : kth;
+                                for (int x = 1; x < KR; ++x) kth = (x < kp) ? top.s[x] : kth;
                             }
                             const uint32_t clr = want ? (1u << idx) : 0u;
 #pragma unroll
                             for (int c = 0; c < 32; ++c) f[c] = ((clr >> c) & 1u) ? -INFINITY : f[c];
                             if (gt == 0) RTRACE(tn + 8 + round);
                         }
-                    } else {
-                        for (int c = 0; c < 32; ++c)
-                            if ((cand >> c) & 1u) top.push(__uint_as_float(v[c]), j0 + c, p.k);
                     }
                 }
                 tc_fence_before();
@@ -520,22 +516,20 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             nx_aw = live2 ? p.anc_bits[(size_t)nx_ci * p.words] : 0u;
             if (gt == 0) RTRACE(tn + 2);
             // sel_idx and the empty slots' partial log-sum-exp
-            int32_t *out = p.sel + ((size_t)h * p.L + i) * p.k;
-            float *pl = p.part_lse + ((size_t)h * p.L + i) * p.k;
+            int32_t *out = p.sel + ((size_t)h * p.L + i) * p.k + pass * 64;
+            float *pl = p.part_lse + ((size_t)h * p.L + i) * p.k + pass * 64;
             if (live) {
-                if (SMALL) {
 #pragma unroll
-                    for (int x = 0; x < KR; ++x)
-                        if (x < p.k) {
-                            out[x] = top.j[x];
-                            if (top.j[x] < 0) pl[x] = -INFINITY;
-                        }
-                } else {
-                    for (int x = 0; x < p.k; ++x) {
+                for (int x = 0; x < KR; ++x)
+                    if (x < kp) {
                         out[x] = top.j[x];
                         if (top.j[x] < 0) pl[x] = -INFINITY;
                     }
-                }
+            }
+            if (KMAX == 64) {                           // the next pass starts after this pass's last pick
+#pragma unroll
+                for (int x = 0; x < KR; ++x)
+                    if (x == kp - 1) { prev_s = top.s[x]; prev_j = top.j[x]; }
             }
             if (deferred) {
                 int *cntb = hist + (ndef & 1) * p.C;
@@ -543,7 +537,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 int njr[KR];                           // chunk << 8 | tile-local rank, or -1
 #pragma unroll
                 for (int x = 0; x < KR; ++x) {
-                    const int j = (live && x < p.k) ? top.j[x] : -1;
+                    const int j = (live && x < kp) ? top.j[x] : -1;
                     njr[x] = j >= 0 ? ((j << 8) | atomicAdd(&cntb[j], 1)) : -1;
                 }
                 ok = group_sync();
@@ -573,18 +567,13 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             ok = group_sync();
             if (!ok) break;
             if (live) {
-                if (SMALL) {
 #pragma unroll
-                    for (int x = 0; x < KR; ++x) {
-                        pend.j[x] = x < p.k ? top.j[x] : -1;
-                        pend.rank[x] = 0;
-                        if (pend.j[x] >= 0) pend.rank[x] = atomicAdd(&hist[pend.j[x]], 1);
-                    }
-                } else {
-                    for (int x = 0; x < p.k; ++x)
-                        if (top.j[x] >= 0) top.s[x] = __int_as_float(atomicAdd(&hist[top.j[x]], 1));   // the score is no longer needed
+                for (int x = 0; x < KR; ++x) {
+                    pend.j[x] = x < kp ? top.j[x] : -1;
+                    pend.rank[x] = 0;
+                    if (pend.j[x] >= 0) pend.rank[x] = atomicAdd(&hist[pend.j[x]], 1);
                 }
-            } else if (SMALL) {
+            } else {
 #pragma unroll
                 for (int x = 0; x < KR; ++x) { pend.j[x] = -1; pend.rank[x] = 0; }
             }
@@ -600,21 +589,15 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 if (!ok) break;
                 if (live) {
                     int32_t *list = p.qlist + (size_t)h * p.cap_total;
-                    if (SMALL) {
 #pragma unroll
-                        for (int x = 0; x < KR; ++x)
-                            if (pend.j[x] >= 0) list[s_cap[pend.j[x]] + hist[pend.j[x]] + pend.rank[x]] = i * p.k + x;
-                    } else {
-                        for (int x = 0; x < p.k; ++x) {
-                            const int j = top.j[x];
-                            if (j >= 0) list[s_cap[j] + hist[j] + __float_as_int(top.s[x])] = i * p.k + x;
-                        }
-                    }
+                    for (int x = 0; x < KR; ++x)
+                        if (pend.j[x] >= 0) list[s_cap[pend.j[x]] + hist[pend.j[x]] + pend.rank[x]] = i * p.k + pass * 64 + x;
                 }
                 ok = group_sync();
                 if (!ok) break;
             }
             if (gt == 0) RTRACE(tn + 5);
+            }   // pass
         }
         if (ok && pend.open) {                 // the last unit's entries
             write_bases();
@@ -698,7 +681,8 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         const unsigned grid = (unsigned)(p->H * a.ctas_per_head);
         // Four selection groups (more warps to hide the selection's latencies) when an accumulator fits
         // a quarter of TMEM and k <= 8; one when the 64-entry list takes nearly all of a thread's registers; two otherwise.
-        const int ng = (a.sb_rows <= 128 && p->k <= 8) ? 4 : (p->k > 32 && p->k <= 64) ? 1 : 2;
+        const int ng = (a.sb_rows <= 128 && p->k <= 8) ? 4 : p->k > 32 ? 1 : 2;
+        a.n_pass = p->k > 64 ? (p->k + 63) / 64 : 1;
         // one histogram per group, the list offsets, and one byte per unit of a CTA
         const size_t hist = (ng * (p->k <= 8 && p->C <= 256 ? 4 : 1) + 1) * sizeof(int) * (size_t)p->C + 2 * (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
         if (d_block + q_tile + hist > budget) return MOC_ERR_SHAPE;
@@ -717,8 +701,7 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         else if (p->k <= 8) { if (few) MOC_ROUTE_CASE(8, 4, true); else if (ng == 4) MOC_ROUTE_CASE(8, 4, false); else MOC_ROUTE_CASE(8, 2, false); }
         else if (p->k <= 16) MOC_ROUTE_CASE(16, 2, false);
         else if (p->k <= 32) MOC_ROUTE_CASE(32, 2, false);
-        else if (p->k <= 64) MOC_ROUTE_CASE(64, 1, false);
-        else MOC_ROUTE_CASE(512, 2, false);
+        else MOC_ROUTE_CASE(64, 1, false);                 // beyond 64 picks: several passes of 64
 #undef MOC_ROUTE_CASE
         MOC_LAUNCH_CHECK();
     }
