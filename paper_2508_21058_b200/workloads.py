@@ -149,15 +149,15 @@ def workload(name: str, seed: int = 0) -> Workload:
     if name == "mini5":   # non-causal single-shot variant: chunk 256, k=3, self + prompt
         return Workload(name, 2, 64, make_layout(1, 77, 1, 1500, chunk_len=256), 3, 0, 0,
                         causal=False, seed=seed)
-    if name == "mini6":   # many small chunks, k beyond the register-resident top-k list (k = 12)
+    if name == "mini6":   # many small chunks, k = 12: the 16-entry pick list, two selection groups
         return Workload(name, 2, 128, make_layout(3, 16, 40, 24), 12, 1, 1, seed=seed)
-    if name == "mini7":   # k = 70 of up to 122 candidates, d = 64: the long-list selection path, streamed descriptor blocks
+    if name == "mini7":   # k = 70 of up to 122 candidates, d = 64: two selection passes of 64 picks, streamed descriptor blocks
         return Workload(name, 2, 64, make_layout(3, 16, 80, 16), 70, 1, 1, seed=seed)
     if name == "mini8":   # few chunks (one scoring operand for the three descriptor terms) with k above 4
         return Workload(name, 2, 128, make_layout(2, 32, 10, 160), 6, 1, 1, seed=seed)
     if name == "mini9":   # more than 32 chunks with k <= 4: the selection by extraction rounds, short list
         return Workload(name, 2, 64, make_layout(3, 16, 14, 96), 4, 1, 1, seed=seed)
-    if name == "mini10":  # k = 20 of up to 80 candidates: the largest register-resident list
+    if name == "mini10":  # k = 20 of up to 80 candidates: the 32-entry pick list
         return Workload(name, 2, 128, make_layout(2, 16, 40, 32), 20, 1, 1, seed=seed)
     if name == "mini11":  # k = 40 of up to 120 candidates: the 64-entry register list, one selection group
         return Workload(name, 2, 64, make_layout(2, 16, 60, 32), 40, 1, 1, seed=seed)
