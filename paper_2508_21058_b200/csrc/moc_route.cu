@@ -184,6 +184,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     for (int x = threadIdx.x; x < nu; x += kRtThreads) s_reach[x] = (uint16_t)chunks_in_reach(p, unit_of(x));
     __syncthreads();
     constexpr int ACC_COLS = 512 / NG;   // TMEM columns per accumulator (NG = 4 only with sb_rows <= 128)
+    const int n_pass = KMAX == 64 ? p.n_pass : 1;     // only the 64-entry list is used for more picks than it holds
     const bool resident = p.d_rows == p.c_pad;       // every chunk's descriptor is held: loaded once, two MMA issuers
 
     if (warp == 0) {
@@ -196,7 +197,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             for (int n = 0; ok && n < nu; ++n) {
                 const int u = unit_of(n);
                 const int reach = s_reach[n], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
-                for (int rep = 0; ok && rep < p.n_pass; ++rep)
+                for (int rep = 0; ok && rep < n_pass; ++rep)
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
                     if (sb == 0 && rep == 0) {
                         const int st = qn % p.q_stages;
@@ -256,7 +257,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 const int buf = n % NG;
                 const int qn = n, st = qn % p.q_stages;
                 RTRACE(3000 + n * 4 + 3);
-                for (int rep = 0; ok && rep < p.n_pass; ++rep)
+                for (int rep = 0; ok && rep < n_pass; ++rep)
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
                     if (sb == 0 && rep == 0) {
                         ok = mbar_wait(bar(Q_FULL + st), (qn / p.q_stages) & 1, abort_flag, p.status, RW_QFULL);
@@ -306,7 +307,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                     if (!resident) {
                         int nsb = sb + 1;
                         bool more = true;
-                        if (nsb >= n_sb) { nsb = 0; more = rep + 1 < p.n_pass || n + 1 < nu; }
+                        if (nsb >= n_sb) { nsb = 0; more = rep + 1 < n_pass || n + 1 < nu; }
                         if (more && nsb != sb) tc_commit(bar(D_EMPTY));
                     }
                 }
@@ -385,7 +386,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             // the order of the result (score descending, then chunk index ascending).
             [[maybe_unused]] float prev_s = INFINITY;
             [[maybe_unused]] int prev_j = -1;
-            for (int pass = 0; ok && pass < p.n_pass; ++pass) {
+            for (int pass = 0; ok && pass < n_pass; ++pass) {
             const int kp = min(p.k - pass * 64, KMAX);      // picks of this pass
             TopK<KMAX> top;
             top.init();
