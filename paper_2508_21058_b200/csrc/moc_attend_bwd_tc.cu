@@ -36,7 +36,7 @@ namespace moc {
 using namespace tc;
 
 enum BwdMode { DQ_ROUTED = 0, DQ_ANCHOR = 1, DKV = 2 };
-enum BwdWait { BW_XFULL = 64, BW_YFULL, BW_YEMPTY, BW_T1FULL, BW_T2FULL, BW_PDONE, BW_DSDONE, BW_ACCFULL, BW_SMEM };
+enum BwdWait { BW_XFULL = 64, BW_YFULL, BW_YEMPTY, BW_T1FULL, BW_T2FULL, BW_PDONE, BW_DSDONE, BW_ACCFULL, BW_SMEM, BW_READ };
 
 struct BwdParams {
     const __nv_bfloat16 *Q, *K, *V, *dO;
@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
     constexpr int CH = D / 8;               // 16-byte pieces per row
     constexpr int N_TILES_SMEM = 2 + kY1Stages + kY2Stages;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[21];
+    __shared__ __align__(8) uint64_t bars[23];
     __shared__ uint32_t tmem_slot;
     __shared__ int s_abort;
     __shared__ int w_valid, w_h, w_rows, w_first, w_nrng, w_ntiles, w_chunk, w_t0;
@@ -102,7 +102,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
     const uint32_t sX = sbase, sY1 = sbase + 2 * TILE_BYTES, sY2 = sbase + (2 + kY1Stages) * TILE_BYTES;
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     constexpr int X_FULL = 0, Y1_FULL = 1, Y1_EMPTY = 4, Y2_FULL = 7, Y2_EMPTY = 9, T1_FULL = 11, T2_FULL = 13,
-                  P_HALF = 15, P_DONE = 16, DS_DONE = 17, ACC_FULL = 19, T1_ISSUED = 20;
+                  P_HALF = 15, P_DONE = 16, DS_DONE = 17, ACC_FULL = 19, T1_ISSUED = 20, RD1 = 21, RD2 = 22;
 
     if (threadIdx.x == 0) BTRACE(0);
     if (threadIdx.x == 0) {
@@ -161,6 +161,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
         mbar_init(bar(P_HALF), 256);
         mbar_init(bar(P_DONE), 256);
         mbar_init(bar(T1_ISSUED), 1);
+        mbar_init(bar(RD1), 256);
+        mbar_init(bar(RD2), 256);
         mbar_init(bar(ACC_FULL), 2);                                // both issuers
         fence_barrier_init();
     }
@@ -254,8 +256,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 uint32_t s[32];
                 tmem_ld32(tmem + lane_off + ch * 32, s);
                 tmem_wait_ld();
-                // dK/dV: P goes over T1 columns that the other thread of the lane reads in its first round
-                if (MODE == DKV && rd == 0) asm volatile("bar.sync 2, 256;" ::: "memory");
+                // dK/dV: P goes over T1 columns that the other thread of the lane reads in its first round; that
+                // read is announced here and waited for (bounded, like every wait) just before the first store
+                if (MODE == DKV && rd == 0) mbar_arrive(bar(RD1));
 #pragma unroll
                 for (int x = 0; x < 32; x += 2) {
                     float l0 = lse2, l1 = lse2;
@@ -275,12 +278,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     uint32_t ups[16];
 #pragma unroll
                     for (int x = 0; x < 16; ++x) ups[x] = bf16x2(pv[rd * 32 + 2 * x], pv[rd * 32 + 2 * x + 1]);
-                    tmem_st16(tmem + lane_off + ch * 16, ups);
-                    tmem_wait_st();
-                    tc_fence_before();
-                    mbar_arrive(bar(rd == 0 ? P_HALF : P_DONE));      // the first, then the second 64 columns of P
+                    if (rd == 0) {
+                        ok = mbar_wait_spin(bar(RD1), jt & 1, abort_flag, p.status, BW_READ);
+                        ok = __all_sync(0xffffffffu, ok);
+                    }
+                    if (ok) {
+                        tmem_st16(tmem + lane_off + ch * 16, ups);
+                        tmem_wait_st();
+                        tc_fence_before();
+                        mbar_arrive(bar(rd == 0 ? P_HALF : P_DONE));      // the first, then the second 64 columns of P
+                    }
                 }
             }
+            if (!ok) break;
             if (MODE != DKV) {                                            // T1 has been read and may be overwritten
                 tc_fence_before();
                 mbar_arrive(bar(P_DONE));
@@ -298,7 +308,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 uint32_t dp[32], uds[16];
                 tmem_ld32(tmem + lane_off + t2c + ch * 32, dp);
                 tmem_wait_ld();
-                if (rd == 0) asm volatile("bar.sync 3, 256;" ::: "memory");
+                if (rd == 0) mbar_arrive(bar(RD2));                     // this thread's first-round columns have been read
 #pragma unroll
                 for (int x = 0; x < 32; x += 2) {
                     float d0 = dlt, d1 = dlt;
@@ -309,8 +319,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     uds[x >> 1] = bf16x2(pv[rd * 32 + x] * (__uint_as_float(dp[x]) - d0),
                                          pv[rd * 32 + x + 1] * (__uint_as_float(dp[x + 1]) - d1));
                 }
-                tmem_st16(tmem + lane_off + t2c + ch * 16, uds);
+                if (rd == 0) {
+                    ok = mbar_wait_spin(bar(RD2), jt & 1, abort_flag, p.status, BW_READ);
+                    ok = __all_sync(0xffffffffu, ok);
+                }
+                if (ok) tmem_st16(tmem + lane_off + t2c + ch * 16, uds);
             }
+            if (!ok) break;
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(DS_DONE + st));
