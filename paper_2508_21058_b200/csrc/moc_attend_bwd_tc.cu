@@ -522,6 +522,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             const uint64_t x1 = smem_desc_sw128(sX, 16, 1024), x2 = smem_desc_sw128(sX + TILE_BYTES, 16, 1024);
             const uint64_t y1k = smem_desc_sw128(sY1, 16, 1024), y2k = smem_desc_sw128(sY2, 16, 1024);
             const uint64_t y1m = smem_desc_sw128(sY1, SUB_BYTES, 1024), y2m = smem_desc_sw128(sY2, SUB_BYTES, 1024);
+            // only the start-address field (low word) of a descriptor moves: 32-bit arithmetic, never a carry out of it
+            auto lo = [](uint64_t d) { return (uint32_t)d; };
+            auto hi = [](uint64_t d) { return (uint32_t)(d >> 32); };
             bool ok = true;
             auto wait = [&](int b, int parity, int code) { ok = ok && mbar_wait_spin(bar(b), parity, abort_flag, p.status, code); };
             // the MMA groups, without their waits and commits
@@ -531,7 +534,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t o = ((ks >> 2) * SUB_BYTES + (ks & 3) * 32) >> 4;
-                    mma_ss(tmem, x1 + o, y1k + s3 * STAGE + o, IDESC_T, ks > 0);
+                    mma_ss_lo(tmem, lo(x1) + o, hi(x1), lo(y1k) + s3 * (uint32_t)STAGE + o, hi(y1k), IDESC_T, ks > 0);
                 }
                 BTRACE_J(1024, 8, j, 4);
             };
@@ -542,7 +545,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t o = ((ks >> 2) * SUB_BYTES + (ks & 3) * 32) >> 4;
-                    mma_ss(d, x2 + o, y2k + s2 * STAGE + o, IDESC_T, ks > 0);
+                    mma_ss_lo(d, lo(x2) + o, hi(x2), lo(y2k) + s2 * (uint32_t)STAGE + o, hi(y2k), IDESC_T, ks > 0);
                 }
             };
             auto acc1 = [&](int j) {        // ACC1 += dS(j) Y1(j)
@@ -551,15 +554,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 const uint32_t ds = tmem + ((MODE != DKV && (j & 1)) ? 384u : 128u);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    mma_ts(tmem + 256, ds + ks * 8, y1m + s3 * STAGE + ks * (2048 >> 4), IDESC_ACC, j > 0 || ks > 0);
+                    mma_ts_lo(tmem + 256, ds + ks * 8, lo(y1m) + s3 * (uint32_t)STAGE + ks * (2048 >> 4), hi(y1m), IDESC_ACC, j > 0 || ks > 0);
             };
             auto acc2 = [&](int j, int half) {   // ACC2 += P(j) Y2(j), the K steps of one half of P
                 const int s2 = j & 1;
                 if (half == 0) BTRACE_J(1024, 8, j, 3);
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
-                    mma_ts(tmem + 384, tmem + (half * 4 + ks) * 8, y2m + s2 * STAGE + (half * 4 + ks) * (2048 >> 4), IDESC_ACC,
-                           j > 0 || half > 0 || ks > 0);
+                    mma_ts_lo(tmem + 384, tmem + (half * 4 + ks) * 8, lo(y2m) + s2 * (uint32_t)STAGE + (half * 4 + ks) * (2048 >> 4), hi(y2m),
+                              IDESC_ACC, j > 0 || half > 0 || ks > 0);
             };
             // A wait, a fence or a commit between two groups leaves the pipe idle for longer than it takes, so each
             // side waits early for the tiles it will read, fences once per hand-over from the lanes, and commits

@@ -462,23 +462,25 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 const int n_qk = max(16, (valid + 15) & ~15);
                 const uint32_t idesc_qk = idesc_bf16_f32(128, n_qk, 0, 0);
                 const uint64_t qd = q_desc0 + (g ? STAGE : 0), kd = k_desc0 + (st ? STAGE : 0);
+                const uint32_t q_lo = (uint32_t)qd, q_hi = (uint32_t)(qd >> 32), k_lo = (uint32_t)kd, k_hi = (uint32_t)(kd >> 32);
                 const uint32_t d_s = tmem + g * 128;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t o = ((ks >> 2) * SUB_BYTES + (ks & 3) * 32) >> 4;
-                    mma_ss(d_s, qd + o, kd + o, idesc_qk, ks > 0);
+                    const uint32_t o = ((ks >> 2) * SUB_BYTES + (ks & 3) * 32) >> 4;     // never carries out of the address field
+                    mma_ss_lo(d_s, q_lo + o, q_hi, k_lo + o, k_hi, idesc_qk, ks > 0);
                 }
             };
             // k-steps [ks0, ks1) of  O_g += P_g V(stage st)  (16 keys each)
             auto issue_pv = [&](int g, int st, int ks0, int ks1, bool accumulate) {
                 const uint64_t vd = v_desc0 + (st ? STAGE : 0);
+                const uint32_t v_lo = (uint32_t)vd, v_hi = (uint32_t)(vd >> 32);
                 const uint32_t d_o = tmem + 256 + g * 128, a_p = tmem + g * 128;
                 if (ks1 - ks0 == 4) {
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
-                        mma_ts(d_o, a_p + (ks0 + ks) * 8, vd + (ks0 + ks) * (2048 >> 4), IDESC_PV, accumulate || ks > 0);
+                        mma_ts_lo(d_o, a_p + (ks0 + ks) * 8, v_lo + (ks0 + ks) * (2048 >> 4), v_hi, IDESC_PV, accumulate || ks > 0);
                 } else {
-                    for (int ks = ks0; ks < ks1; ++ks) mma_ts(d_o, a_p + ks * 8, vd + ks * (2048 >> 4), IDESC_PV, accumulate || ks > ks0);
+                    for (int ks = ks0; ks < ks1; ++ks) mma_ts_lo(d_o, a_p + ks * 8, v_lo + ks * (2048 >> 4), v_hi, IDESC_PV, accumulate || ks > ks0);
                 }
             };
             // this issuer serves query tile g: S_g(0), then per key tile  O_g += P_g V(j),  S_g(j + 1)

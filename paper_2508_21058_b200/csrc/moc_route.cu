@@ -283,8 +283,8 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                         const uint32_t acc = tmem + buf * ACC_COLS;
 #pragma unroll
                         for (int ks = 0; ks < D / 16; ++ks)
-                            mma_ss(acc, qd + (((ks >> 2) * Q_SUB_BYTES + (ks & 3) * 32) >> 4),
-                                   d_term[ks >> 2] + (((ks & 3) * 32) >> 4), idesc, ks != 0);
+                            mma_ss_lo(acc, (uint32_t)qd + (((ks >> 2) * Q_SUB_BYTES + (ks & 3) * 32) >> 4), (uint32_t)(qd >> 32),
+                                      (uint32_t)d_term[ks >> 2] + (((ks & 3) * 32) >> 4), (uint32_t)(d_term[ks >> 2] >> 32), idesc, ks != 0);
                     } else
                     for (int n0 = 0; n0 < rows_sb; n0 += 128) {
                         const int n = min(128, rows_sb - n0);
@@ -295,8 +295,9 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                         for (int term = 0; term < 3; ++term) {
 #pragma unroll
                             for (int ks = 0; ks < D / 16; ++ks)
-                                mma_ss(acc, qd + (((ks >> 2) * Q_SUB_BYTES + (ks & 3) * 32) >> 4),
-                                       d_term[term * SUB + (ks >> 2)] + nofs + (((ks & 3) * 32) >> 4), idesc, (term | ks) != 0);
+                                mma_ss_lo(acc, (uint32_t)qd + (((ks >> 2) * Q_SUB_BYTES + (ks & 3) * 32) >> 4), (uint32_t)(qd >> 32),
+                                          (uint32_t)d_term[term * SUB + (ks >> 2)] + nofs + (((ks & 3) * 32) >> 4),
+                                          (uint32_t)(d_term[term * SUB + (ks >> 2)] >> 32), idesc, (term | ks) != 0);
                         }
                     }
                     tc_commit(bar(ACC_FULL + buf));
