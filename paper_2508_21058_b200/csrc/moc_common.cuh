@@ -110,15 +110,17 @@ static inline const T *ws_ptr(const void *ws, size_t off) { return reinterpret_c
 // Walks the 128-key tiles of a list of key ranges (a tile never straddles two ranges).
 struct TileIter {
     const KeyRange *rng;
-    int n, ri, t;
-    __device__ TileIter(const KeyRange *r, int n_) : rng(r), n(n_), ri(0), t(n_ > 0 ? r[0].t0 : 0) {}
+    int n, ri, t, end;      // the current range's end is kept: one load per range, not per tile
+    __device__ TileIter(const KeyRange *r, int n_) : rng(r), n(n_), ri(0), t(n_ > 0 ? r[0].t0 : 0), end(n_ > 0 ? r[0].t1 : 0) {}
     __device__ bool next(int &t0, int &valid) {
         if (ri >= n) return false;
-        const int end = rng[ri].t1;
         t0 = t;
         valid = min(128, end - t);
         t += 128;
-        if (t >= end) { ++ri; if (ri < n) t = rng[ri].t0; }
+        if (t >= end) {
+            ++ri;
+            if (ri < n) { t = rng[ri].t0; end = rng[ri].t1; }
+        }
         return true;
     }
 };
