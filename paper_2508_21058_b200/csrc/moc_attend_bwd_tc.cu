@@ -528,8 +528,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             bool ok = true;
             auto wait = [&](int b, int parity, int code) { ok = ok && mbar_wait_spin(bar(b), parity, abort_flag, p.status, code); };
             // the MMA groups, without their waits and commits
-            auto t1 = [&](int j) {          // T1(j) = X1 Y1(j)^T
-                const int s3 = j % kY1Stages;
+            // (s3 = j mod the Y1 stage count is carried along by the callers: no division on this thread)
+            auto t1 = [&](int j, int s3) {  // T1(j) = X1 Y1(j)^T
                 BTRACE_J(1024, 8, j, 0);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
@@ -548,9 +548,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     mma_ss_lo(d, lo(x2) + o, hi(x2), lo(y2k) + s2 * (uint32_t)STAGE + o, hi(y2k), IDESC_T, ks > 0);
                 }
             };
-            auto acc1 = [&](int j) {        // ACC1 += dS(j) Y1(j)
+            auto acc1 = [&](int j, int s3) {   // ACC1 += dS(j) Y1(j)
                 BTRACE_J(1024, 8, j, 2);
-                const int s3 = j % kY1Stages;
                 const uint32_t ds = tmem + ((MODE != DKV && (j & 1)) ? 384u : 128u);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
@@ -575,10 +574,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     wait(Y1_FULL, 0, BW_YFULL);
                     if (ok) {
                         tc_fence_after();
-                        t1(0);
+                        t1(0, 0);
                         tc_commit(bar(T1_FULL));
                     }
                 }
+                int s3n = 1 % kY1Stages, ph3n = 0;                       // stage and phase of tile j + 1
                 for (int j = 0; ok && j < n_tiles; ++j) {
                     const bool more = j + 1 < n_tiles;
                     if (MODE == DKV) {
@@ -587,7 +587,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                         tc_fence_after();
                         acc2(j, 0);
                     }
-                    if (more) wait(Y1_FULL + (j + 1) % kY1Stages, ((j + 1) / kY1Stages) & 1, BW_YFULL);
+                    if (more) wait(Y1_FULL + s3n, ph3n, BW_YFULL);
                     if (MODE == DKV || more) wait(P_DONE, j & 1, BW_PDONE);
                     if (!ok) break;
                     BTRACE_J(1024, 8, j, 6);
@@ -595,10 +595,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     if (MODE == DKV) acc2(j, 1);
                     BTRACE_J(1024, 8, j, 7);
                     if (more) {
-                        t1(j + 1);
+                        t1(j + 1, s3n);
                         tc_commit(bar(T1_FULL + ((j + 1) & 1)));
                         BTRACE_J(1024, 8, j + 1, 5);
                     }
+                    if (++s3n == kY1Stages) { s3n = 0; ph3n ^= 1; }
                     if (MODE == DKV) {
                         tc_commit(bar(Y2_EMPTY + (j & 1)));                 // the second of two arrivals
                         if (more) mbar_arrive(bar(T1_ISSUED));              // the other side may use the pipe again
@@ -617,6 +618,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     tc_commit(bar(T2_FULL + (j & 1)));
                     tc_commit(bar(Y2_EMPTY + (j & 1)));
                 }
+                int s3 = 0;                                               // Y1 stage of tile j
                 for (int j = 0; ok && j < n_tiles; ++j) {
                     const int jn = j + AHEAD;
                     const bool more = jn < n_tiles;
@@ -624,8 +626,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     wait(DS_DONE + (j & 1), (j >> 1) & 1, BW_DSDONE);
                     if (!ok) break;
                     tc_fence_after();
-                    acc1(j);
-                    tc_commit(bar(Y1_EMPTY + j % kY1Stages));       // at once: the next K tile waits for this stage
+                    acc1(j, s3);
+                    tc_commit(bar(Y1_EMPTY + s3));                  // at once: the next K tile waits for this stage
+                    if (++s3 == kY1Stages) s3 = 0;
                     if (more) {
                         wait(Y2_FULL + (jn & 1), (jn >> 1) & 1, BW_YFULL);
                         if (!ok) break;
