@@ -429,9 +429,14 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                             for (int c = 0; c < 8; ++c) {
                                 float cv = ((cand >> (g * 8 + c)) & 1u) ? f[c] : -INFINITY;
                                 int cj = g * 8 + c;
+                                bool placed = false;
 #pragma unroll
                                 for (int x = 0; x < KR; ++x) {
-                                    const bool up = cv > top.s[x];
+                                    // the new score takes the first slot it beats (strict '>': equal scores keep
+                                    // their arrival order, ascending chunk index); from there on every entry moves
+                                    // down one slot, equal ones included, and the last falls off
+                                    const bool up = placed || cv > top.s[x];
+                                    placed = up;
                                     const float ts = top.s[x];
                                     const int tj = top.j[x];
                                     top.s[x] = up ? cv : ts;
@@ -486,13 +491,16 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                             for (int c = 0; c < 32; ++c) eq |= (f[c] == m) ? (1u << c) : 0u;
                             const int idx = __ffs(eq) - 1;
                             if (want) {
-                                // the displaced element sinks through the sorted list (strict '>' keeps equal
-                                // scores in arrival order, which is ascending chunk index)
                                 float cv = m;
                                 int cj = j0 + idx;
+                                bool placed = false;
 #pragma unroll
                                 for (int x = 0; x < KR; ++x) {
-                                    const bool up = cv > top.s[x];
+                                    // the new score takes the first slot it beats (strict '>': equal scores keep
+                                    // their arrival order, ascending chunk index); from there on every entry moves
+                                    // down one slot, equal ones included, and the last falls off
+                                    const bool up = placed || cv > top.s[x];
+                                    placed = up;
                                     const float ts = top.s[x];
                                     const int tj = top.j[x];
                                     top.s[x] = up ? cv : ts;

@@ -92,6 +92,29 @@ def test_backward_benchmark_length_sampled():
     _backward_parity("cfg1", scalar=False, n_rows=96, heads=2)
 
 
+def test_backward_training_length_sampled():
+    """The minute-scale training layout at its full length, one head: dQ on sampled rows and dK / dV of one
+    frame in the middle of the stream (its queries are its shot window and the rows that routed to it; a caption
+    chunk is attended by all 528k queries, which the oracle cannot afford here - the single-shot test covers it)."""
+    wl = W.workload("cfg4")
+    wl.n_heads = 1
+    run = PU.GpuRun(wl, tensors=("q", "k", "v", "do")).forward().backward()
+    x = run.host_inputs()
+    orc = Oracle.from_workload(wl)
+    sel_gpu = run.sel.cpu().numpy()
+    lay = wl.layout
+    rows = W.sample_rows(wl, 64)
+    chunk = lay.n_chunks // 2 + 3
+    assert int(lay.chunk_mod[chunk]) == 0           # a video frame
+    t0, t1 = int(lay.chunk_off[chunk]), int(lay.chunk_off[chunk + 1])
+    dQ, dK, dV = orc.attend_bwd(x["q"], x["k"], x["v"], x["do"], sel_gpu, rows, 0, (t0, t1))
+    dQ_g = run.dQ.float().cpu().numpy()[rows[:, 0], rows[:, 1]]
+    dK_g, dV_g = run.dK.float().cpu().numpy()[0, t0:t1], run.dV.float().cpu().numpy()[0, t0:t1]
+    for g, r in ((dQ_g, dQ), (dK_g, dK), (dV_g, dV)):
+        assert np.max(np.abs(g - r)) <= PU.GRAD_MAX_ABS
+        assert np.sqrt(np.sum((g - r) ** 2) / np.sum(r ** 2)) < 2e-2
+
+
 def test_route_is_deterministic_and_lists_invert_selection():
     wl = W.workload("mini2")
     run = PU.GpuRun(wl).forward()
@@ -142,6 +165,33 @@ def test_all_tie_scores_pick_lowest_indices():
     assert np.max(np.abs(run.lse[0, ::37].cpu().numpy() - np.log(pairs_row))) < 1e-4
 
 
+@pytest.mark.parametrize("name", ["mini8", "mini9", "mini10", "mini11", "mini7"])
+def test_equal_descriptors_keep_index_order(name):
+    """Groups of frames with identical keys have identical descriptors, so every query scores them
+    equally: inside the sorted pick list equal scores must stay in ascending chunk order while better
+    chunks arriving later push the list down, and the one that falls off must be the highest index.
+    Covers the one-pass list, the extraction rounds with 4 / 32 / 64 entries and the passes beyond 64 picks."""
+    wl = W.workload(name)
+    lay = wl.layout
+    run = PU.GpuRun(wl)
+    video = [c for c in range(lay.n_chunks) if lay.chunk_mod[c] == 0 and lay.chunk_shot[c] == 0]
+    L0 = int(lay.chunk_off[video[0] + 1] - lay.chunk_off[video[0]])
+    same = [c for c in video if int(lay.chunk_off[c + 1] - lay.chunk_off[c]) == L0]
+    # frames 0, 3, 6, ... of the first shot share their keys; so do frames 1, 4, 7, ...
+    for grp in (same[0::3], same[1::3]):
+        src = run.x["k"][:, int(lay.chunk_off[grp[0]]):int(lay.chunk_off[grp[0]]) + L0].clone()
+        for c in grp[1:]:
+            run.x["k"][:, int(lay.chunk_off[c]):int(lay.chunk_off[c]) + L0] = src
+    run.forward()
+    x = run.host_inputs()
+    orc = Oracle.from_workload(wl)
+    desc64 = orc.chunk_pool(x["k"])
+    n, near, hard, ex, order_bad = PU.compare_routing(wl, orc, x["q"], desc64, run.sel.cpu().numpy())
+    assert hard == 0, ex
+    assert near <= max(2, int(2e-3 * n)), (near, n)
+    assert order_bad <= near + max(2, int(2e-3 * n)), order_bad
+
+
 def test_argument_errors_launch_nothing():
     wl = W.workload("mini1")
     lay = wl.layout
@@ -170,7 +220,7 @@ def test_argument_errors_launch_nothing():
     assert launch_count() == n0
 
 
-@pytest.mark.parametrize("name,rows_per_head,heads", [("cfg1", 96, None), ("cfg2", 192, 3)])
+@pytest.mark.parametrize("name,rows_per_head,heads", [("cfg1", 96, None), ("cfg2", 192, 3), ("cfg4", 192, 2), ("cfg3-m512-p8", 128, 1), ("cfg3-m256-p15", 96, 1)])
 def test_forward_benchmark_size_sampled(name, rows_per_head, heads):
     """The benchmark workload in the launch configuration bench.py times; attention
     checked on sampled rows (frame, caption and shot edges plus uniform picks), indices on
