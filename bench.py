@@ -2,7 +2,7 @@
 """Benchmark of the MoC hot path (pool -> route -> attend, + backward for the training
 workload) on seeded synthetic inputs.
 
-    python bench.py --gpus N --steps K --warmup W [--workload cfg1] [--impl reference]
+    python bench.py --gpus N --steps K --warmup W [--workload cfg2] [--impl reference]
 
 One step = one pass of the whole hot path over one batch.  The headline value is the
 selected-key attention throughput of the whole step: 4*d FLOPs per selected (query, key)
@@ -126,6 +126,15 @@ def route_bytes(wl) -> float:
     return 2.0 * (2 * L * d * H) + 4.0 * k * L * H + 2 * 4.0 * C * d * H   # K once + Q once + indices + desc write/read
 
 
+def config_of(wl, with_bwd: bool, world: int) -> dict:
+    """The workload's description, the same in both arms (what a run measured about it goes elsewhere)."""
+    H, L, d = wl.n_heads, wl.n_tokens, wl.head_dim
+    return {"workload": wl.name, "layout": wl.note, "heads": H, "head_dim": d, "tokens": L, "chunks": wl.n_chunks,
+            "top_k": wl.top_k, "window": [wl.win_back, wl.win_fwd], "backward": with_bwd,
+            "l2": "inputs larger than L2 (Q, K, V %.0f MB each); no flush" % (H * L * d * 2 / 1e6),
+            "parallelism": f"replicas x{world}"}
+
+
 def run_reference(args, wl):
     """The CPU oracle, as it stands, timed per step on a bounded sample of the workload:
     one head's descriptors and routing in full, attention on a seeded sample of its rows."""
@@ -157,8 +166,7 @@ def run_reference(args, wl):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / max(len(times), 1),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "layout": wl.note, "heads": wl.n_heads, "head_dim": wl.head_dim,
-                       "tokens": wl.n_tokens, "chunks": wl.n_chunks, "top_k": wl.top_k},
+            "config": config_of(wl, args.bwd or args.workload == "cfg4", int(os.environ.get("WORLD_SIZE", "1"))),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -195,17 +203,140 @@ def cpu_baseline(wl, budget_s: float):
             "sample": f"attention of {n} seeded rows of head 0 ({dt:.1f} s); head-0 descriptors + routing took {t_route:.1f} s"}
 
 
+def run_ours(wl, with_bwd, steps, warmup, world, local_rank, do_e2e):
+    """Times `steps` passes of the hot path on one workload; returns the measurements of this rank
+    (times already reduced to the slowest rank)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2508_21058_b200 import MocPlan, launch_count
+    from paper_2508_21058_b200 import workloads as W
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def _rec():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
+        return e
+
+    tensors = ("q", "k", "v", "do") if with_bwd else ("q", "k", "v")
+    x = W.generate(wl, "cuda", tensors)
+    plan = MocPlan.from_workload(wl)
+    ws = plan.new_workspace(with_bwd)
+    H, L, d, C, k = wl.n_heads, wl.n_tokens, wl.head_dim, wl.n_chunks, wl.top_k
+    desc = torch.empty((H, C, d), dtype=torch.float32, device="cuda")
+    sel = torch.empty((H, L, k), dtype=torch.int32, device="cuda")
+    O = torch.empty_like(x["q"])
+    lse = torch.empty((H, L), dtype=torch.float32, device="cuda")
+    grads = [torch.empty_like(x["q"]) for _ in range(3)] if with_bwd else None
+
+    def step(q, kk, v, marks=None):
+        ev = (lambda: marks.append(_rec())) if marks is not None else (lambda: None)
+        ev()
+        plan.moc_chunk_pool(kk, desc, ws)
+        ev()
+        plan.moc_route(q, desc, sel, ws)
+        ev()
+        plan.moc_attend(q, kk, v, sel, O, lse, ws)
+        ev()
+        if with_bwd:
+            plan.moc_attend_bwd(q, kk, v, O, lse, x["do"], sel, *grads, ws)
+            ev()
+
+    for _ in range(max(warmup, 3)):
+        step(x["q"], x["k"], x["v"])
+    barrier()
+    st, det = plan.moc_get_status(ws)
+    if st != 0:
+        raise SystemExit(f"device status {st} detail {det}")
+    pairs = plan.moc_selected_pairs(ws)
+    flops = step_flops(wl, pairs, with_bwd)
+
+    # ---- timed region: inputs resident in HBM, device time by CUDA events on the launching stream
+    marks_all = []
+    n0 = launch_count()
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        for _ in range(steps):
+            m = []
+            step(x["q"], x["k"], x["v"], m)
+            marks_all.append(m)
+        barrier()
+    launches = launch_count() - n0
+    total_ms = marks_all[0][0].elapsed_time(marks_all[-1][-1])
+    seg = [sum(m[i].elapsed_time(m[i + 1]) for m in marks_all) / steps for i in range(len(marks_all[0]) - 1)]
+    ms_per_step = max_over_ranks_ms(total_ms, world, "cuda") / steps
+    out = {"pairs": pairs, "flops": flops, "ms_per_step": ms_per_step, "seg": seg, "launches": int(launches),
+           "clocks": clocks.summary(), "workspace_bytes": plan.workspace_bytes(with_bwd), "e2e": None}
+
+    # ---- end to end: host buffers in, host results out, copies inside the timed region
+    if do_e2e:
+        hq, hk, hv = (x[n].cpu().pin_memory() for n in ("q", "k", "v"))
+        dq, dk, dv = (torch.empty_like(x[n]) for n in ("q", "k", "v"))
+        hO = torch.empty(O.shape, dtype=O.dtype).pin_memory()
+        hl = torch.empty(lse.shape, dtype=lse.dtype).pin_memory()
+        hg = [torch.empty(O.shape, dtype=O.dtype).pin_memory() for _ in range(3)] if with_bwd else []
+
+        def e2e_step():
+            dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
+            step(dq, dk, dv)
+            hO.copy_(O, non_blocking=True); hl.copy_(lse, non_blocking=True)
+            for a, b in zip(hg, grads or []):
+                a.copy_(b, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+
+        n_e2e = max(2, min(steps, 5))
+        e2e_step()
+        barrier()
+        e0 = _rec()
+        for _ in range(n_e2e):
+            e2e_step()
+        e1 = _rec()
+        barrier()
+        te_ms = max_over_ranks_ms(e0.elapsed_time(e1), world, "cuda")
+        h2d = 3 * hq.numel() * 2
+        d2h = hO.numel() * 2 + hl.numel() * 4 + sum(g.numel() * 2 for g in hg)
+        out["e2e"] = {"value": job_value(flops, world, te_ms / n_e2e), "unit": UNIT,
+                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e}
+    plan.close()
+    del x, ws, desc, sel, O, lse, grads
+    torch.cuda.empty_cache()
+    return out
+
+
+def rooflines(wl, r, peaks, peak_kind):
+    H, L, d = wl.n_heads, wl.n_tokens, wl.head_dim
+    t_pool, t_route, t_att = r["seg"][0], r["seg"][1], r["seg"][2]
+    att_flops = step_flops(wl, r["pairs"], False)
+    att = att_flops / (t_att * 1e-3) / 1e12
+    roofline = {"kernel": "moc_attend (tensor-core flash kernel over selected key chunks)",
+                "bound": "tensor", "achieved": att, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s", "frac": att / peaks["bf16_tflops"],
+                "frac_of_sustained": att / peaks["bf16_tflops_sustained"],
+                "traffic": measured_traffic("moc_attend", wl.name), "peak_source": f"{peak_kind} (burst bf16 matmul)", "ms": t_att}
+    rb = route_bytes(wl)
+    gbs = rb / ((t_pool + t_route) * 1e-3) / 1e9
+    routing = {"kernel": "moc_chunk_pool + moc_route", "bound": "hbm", "achieved": gbs,
+               "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+               "pool_ms": t_pool, "route_ms": t_route, "pool_gbs": (2.0 * L * d * H) / (t_pool * 1e-3) / 1e9,
+               "peak_source": peak_kind}
+    return roofline, routing
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1")
-    ap.add_argument("--scalar", action="store_true", help="use the CUDA-core attention kernels")
+    ap.add_argument("--workload", default="cfg2",
+                    help="cfg2 (the largest forward-only configuration) by default; cfg1, cfg4, cfg3-m<chunk>-p<percent>")
     ap.add_argument("--bwd", action="store_true", help="include moc_attend_bwd in the step (implied by cfg4)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="skip the short runs of the other configurations")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     ap.add_argument("--ref-rows", type=int, default=256)
     ap.add_argument("--heads", type=int, default=0, help="override the head count (profiling a smaller case)")
@@ -230,101 +361,19 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2508_21058_b200 import MocPlan, launch_count
 
     torch.cuda.set_device(local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    tensors = ("q", "k", "v", "do") if with_bwd else ("q", "k", "v")
-    x = W.generate(wl, "cuda", tensors)
-    plan = MocPlan.from_workload(wl, scalar_attend=args.scalar)
-    ws = plan.new_workspace(with_bwd)
-    H, L, d, C, k = wl.n_heads, wl.n_tokens, wl.head_dim, wl.n_chunks, wl.top_k
-    desc = torch.empty((H, C, d), dtype=torch.float32, device="cuda")
-    sel = torch.empty((H, L, k), dtype=torch.int32, device="cuda")
-    O = torch.empty_like(x["q"])
-    lse = torch.empty((H, L), dtype=torch.float32, device="cuda")
-    grads = [torch.empty_like(x["q"]) for _ in range(3)] if with_bwd else None
-
-    def step(q, kk, v, marks=None):
-        ev = (lambda: marks.append(_rec())) if marks is not None else (lambda: None)
-        ev()
-        plan.moc_chunk_pool(kk, desc, ws)
-        ev()
-        plan.moc_route(q, desc, sel, ws)
-        ev()
-        plan.moc_attend(q, kk, v, sel, O, lse, ws)
-        ev()
-        if with_bwd:
-            plan.moc_attend_bwd(q, kk, v, O, lse, x["do"], sel, *grads, ws)
-            ev()
-
-    def _rec():
-        e = torch.cuda.Event(enable_timing=True)
-        e.record()
-        return e
-
-    for _ in range(max(args.warmup, 3)):
-        step(x["q"], x["k"], x["v"])
-    barrier()
-    st, det = plan.moc_get_status(ws)
-    if st != 0:
-        raise SystemExit(f"device status {st} detail {det}")
-    pairs = plan.moc_selected_pairs(ws)
-    flops = step_flops(wl, pairs, with_bwd)
-
-    # ---- timed region: inputs resident in HBM, device time by CUDA events on the launching stream
-    marks_all = []
-    n0 = launch_count()
-    with ClockSampler(local_rank) as clocks:
-        barrier()
-        for _ in range(args.steps):
-            m = []
-            step(x["q"], x["k"], x["v"], m)
-            marks_all.append(m)
-        barrier()
-    launches = launch_count() - n0
-    total_ms = marks_all[0][0].elapsed_time(marks_all[-1][-1])
-    seg = [sum(m[i].elapsed_time(m[i + 1]) for m in marks_all) / args.steps for i in range(len(marks_all[0]) - 1)]
-    ms_per_step = max_over_ranks_ms(total_ms, world, "cuda") / args.steps
-    value = job_value(flops, world, ms_per_step)
-
-    # ---- end to end: host buffers in, host results out, copies inside the timed region
-    e2e = None
-    if not args.no_e2e:
-        hq, hk, hv = (x[n].cpu().pin_memory() for n in ("q", "k", "v"))
-        dq, dk, dv = (torch.empty_like(x[n]) for n in ("q", "k", "v"))
-        hO = torch.empty(O.shape, dtype=O.dtype).pin_memory()
-        hl = torch.empty(lse.shape, dtype=lse.dtype).pin_memory()
-        hg = [torch.empty(O.shape, dtype=O.dtype).pin_memory() for _ in range(3)] if with_bwd else []
-
-        def e2e_step():
-            dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
-            step(dq, dk, dv)
-            hO.copy_(O, non_blocking=True); hl.copy_(lse, non_blocking=True)
-            for a, b in zip(hg, grads or []):
-                a.copy_(b, non_blocking=True)
-            torch.cuda.current_stream().synchronize()
-
-        n_e2e = max(2, min(args.steps, 5))
-        e2e_step()
-        barrier()
-        e0, e1 = _rec(), None
-        for _ in range(n_e2e):
-            e2e_step()
-        e1 = _rec()
-        barrier()
-        te_ms = max_over_ranks_ms(e0.elapsed_time(e1), world, "cuda")
-        h2d = 3 * hq.numel() * 2
-        d2h = hO.numel() * 2 + hl.numel() * 4 + sum(g.numel() * 2 for g in hg)
-        e2e = {"value": job_value(flops, world, te_ms / n_e2e), "unit": UNIT,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e}
+    r = run_ours(wl, with_bwd, args.steps, args.warmup, world, local_rank, not args.no_e2e)
+    # the other configurations, a few steps each, so that one run covers the small single-shot clip, the
+    # multi-shot stream and the training step (forward + backward)
+    others = {}
+    if args.workload == "cfg2" and args.heads == 0 and not args.no_others:
+        for name, bwd in (("cfg1", False), ("cfg4", True)):
+            w2 = W.workload(name, seed=rank)
+            others[name] = (w2, bwd, run_ours(w2, bwd, 3, 3, world, local_rank, False))
 
     if rank != 0:
         if world > 1:
@@ -332,32 +381,34 @@ def main():
         return
 
     peaks, peak_kind = load_peaks()
-    t_pool, t_route, t_att = seg[0], seg[1], seg[2]
-    att_flops = step_flops(wl, pairs, False)
-    traffic = measured_traffic("moc_attend", wl.name)
-    roofline = {"kernel": "moc_attend (tensor-core flash kernel over selected key chunks)" if not args.scalar
-                else "moc_attend (CUDA-core kernels)",
-                "bound": "tensor", "achieved": att_flops / (t_att * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
-                "unit": "TFLOP/s", "frac": att_flops / (t_att * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                "frac_of_sustained": att_flops / (t_att * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
-                "traffic": traffic, "peak_source": f"{peak_kind} (burst bf16 matmul)", "ms": t_att}
-    rb = route_bytes(wl)
-    routing = {"kernel": "moc_chunk_pool + moc_route", "bound": "hbm", "achieved": rb / ((t_pool + t_route) * 1e-3) / 1e9,
-               "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rb / ((t_pool + t_route) * 1e-3) / 1e9 / peaks["hbm_gbs"],
-               "pool_ms": t_pool, "route_ms": t_route, "pool_gbs": (2.0 * L * d * H) / (t_pool * 1e-3) / 1e9,
-               "peak_source": peak_kind}
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+    H, L, d, C, k = wl.n_heads, wl.n_tokens, wl.head_dim, wl.n_chunks, wl.top_k
+    roofline, routing = rooflines(wl, r, peaks, peak_kind)
+    seg = r["seg"]
+    line = {"metric": METRIC, "value": job_value(r["flops"], world, r["ms_per_step"]), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": wl.name, "layout": wl.note, "heads": H, "head_dim": d, "tokens": L, "chunks": C,
-                       "top_k": k, "window": [wl.win_back, wl.win_fwd], "backward": with_bwd,
-                       "selected_pairs": pairs, "sparsity_vs_dense": 1.0 - pairs / (float(H) * L * L),
-                       "l2": "inputs larger than L2 (Q, K, V %.0f MB each); no flush" % (H * L * d * 2 / 1e6),
-                       "parallelism": f"replicas x{world}"},
-            "segments_ms": {"pool": t_pool, "route": t_route, "attend": t_att, **({"attend_bwd": seg[3]} if with_bwd else {})},
-            "roofline": roofline, "roofline_routing": routing, "clocks": clocks.summary(), "gpu_launches": int(launches)}
-    if e2e:
-        line["e2e"] = e2e
+            "config": config_of(wl, with_bwd, world),
+            "workload_stats": {"selected_pairs": r["pairs"], "sparsity_vs_dense": 1.0 - r["pairs"] / (float(H) * L * L),
+                               "workspace_bytes": r["workspace_bytes"]},
+            "segments_ms": {"pool": seg[0], "route": seg[1], "attend": seg[2], **({"attend_bwd": seg[3]} if with_bwd else {})},
+            "roofline": roofline, "roofline_routing": routing, "clocks": r["clocks"], "gpu_launches": r["launches"]}
+    if r["e2e"]:
+        line["e2e"] = r["e2e"]
+    if others:
+        line["other_workloads"] = {}
+        for name, (w2, bwd, r2) in others.items():
+            rf, rt = rooflines(w2, r2, peaks, peak_kind)
+            s2 = r2["seg"]
+            entry = {"steps": 3, "value": job_value(r2["flops"], world, r2["ms_per_step"]), "unit": UNIT, "backward": bwd,
+                     "ms_per_step": r2["ms_per_step"],
+                     "segments_ms": {"pool": s2[0], "route": s2[1], "attend": s2[2], **({"attend_bwd": s2[3]} if bwd else {})},
+                     "attend_tflops": rf["achieved"], "attend_frac": rf["frac"], "routing_gbs": rt["achieved"],
+                     "routing_frac": rt["frac"], "selected_pairs": r2["pairs"], "workspace_bytes": r2["workspace_bytes"],
+                     "clocks": r2["clocks"]}
+            if bwd:
+                entry["attend_bwd_tflops"] = 10.0 * w2.head_dim * r2["pairs"] / (s2[3] * 1e-3) / 1e12
+            line["other_workloads"][name] = entry
     if not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, args.cpu_budget_s)
     print(json.dumps(line))

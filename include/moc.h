@@ -21,9 +21,10 @@
  *   lse                        : DEVICE, fp32, [H][L]; natural log of the sum over the
  *                                selected keys of exp(softmax_scale * q.k).
  *   ws                         : DEVICE scratch of moc_workspace_bytes() bytes, 256-byte
- *                                aligned, owned by the caller.  moc_route writes the
- *                                chunk -> query lists into it; the same pointer, unchanged,
- *                                must be given to moc_attend / moc_attend_bwd afterwards.
+ *                                aligned, owned by the caller.  moc_route (or moc_lists_from_sel)
+ *                                writes the chunk -> query lists of the selection into it; the
+ *                                same pointer, unchanged, must be given to moc_attend /
+ *                                moc_attend_bwd afterwards.
  *   stream                     : a cudaStream_t passed as void* (NULL = default stream).
  *
  * Ownership: the caller owns every buffer.  The library allocates device memory only in
@@ -31,9 +32,12 @@
  * synchronises the stream or the device; work is enqueued on `stream` in call order.
  *
  * Errors: every function returns MOC_OK (0) or a negative moc_status.  Argument errors
- * are detected before anything is launched.  Nothing throws, aborts or traps.  Kernels
- * bound every wait; a wait that runs out sets a status word in the workspace that
- * moc_get_status() reads back (after the caller has synchronised the stream).
+ * are detected before anything is launched.  Nothing throws, aborts or traps.  What only
+ * the device can see is reported through a status word in the workspace that
+ * moc_get_status() reads back: a bounded wait that ran out (MOC_ERR_TIMEOUT; the kernel
+ * drains its copies, frees its tensor memory and returns), or a workspace that does not
+ * hold the lists of this plan (MOC_ERR_WORKSPACE; the attention kernels then return
+ * without reading or writing anything else).
  */
 #ifndef MOC_H_
 #define MOC_H_
@@ -52,21 +56,24 @@ typedef enum moc_status {
     MOC_ERR_CHUNK_TABLE = -3, /* offsets not strictly increasing from 0 to L, shots decreasing,
                                  or a modality other than 0/1                                */
     MOC_ERR_ALIGN = -4,       /* a device pointer is not aligned as required                 */
-    MOC_ERR_WORKSPACE = -5,   /* workspace missing, or routing has not been run on it        */
+    MOC_ERR_WORKSPACE = -5,   /* workspace missing; as a device status: routing (or moc_lists_from_sel)
+                                 of this plan has not been run on it                           */
     MOC_ERR_ARCH = -6,        /* the current device is not compute capability 10.x           */
     MOC_ERR_CUDA = -7,        /* a CUDA runtime call failed; see moc_last_cuda_error()       */
     MOC_ERR_TIMEOUT = -8,     /* device status: a bounded wait inside a kernel ran out       */
-    MOC_ERR_TOO_LARGE = -9    /* problem exceeds the fixed scratch of a no-allocation entry point */
+    MOC_ERR_TOO_LARGE = -9,   /* problem exceeds the fixed scratch of a no-allocation entry point, or the
+                                 workspace budget given to moc_plan_set_workspace_budget           */
+    MOC_ERR_INDEX = -10       /* device status, debug build (-DMOC_DEBUG) only: an index a kernel took
+                                 from the workspace was out of range; the access was skipped       */
 } moc_status;
 
 #define MOC_WHOLE_SHOT (-1)   /* window value: every chunk of the query's shot is an anchor  */
 #define MOC_FLAG_CAUSAL 0x1u  /* routed candidates are strictly earlier chunks (Sec. 3.2)    */
-#define MOC_FLAG_SCALAR_ATTEND 0x2u /* run attention on the plain fp32 CUDA-core kernels     */
 
 /* Problem statement (Sec. 3.1 "Dynamic Routing via Top-k Selection", Sec. 3.3).  The three
  * table pointers are HOST pointers, read during moc_plan_create only. */
 typedef struct moc_problem {
-    int32_t n_heads, n_tokens, head_dim;  /* H >= 1, L >= 1, d in {64, 128}                  */
+    int32_t n_heads, n_tokens, head_dim;  /* 1 <= H <= 65535, L >= 1, H * L < 2^31, d in {64, 128} */
     int32_t n_chunks, top_k;              /* C >= 1, 0 <= k <= 512                           */
     int32_t win_back, win_fwd;            /* intra-shot anchor window in chunks before/after
                                              the query's own chunk; MOC_WHOLE_SHOT = the
@@ -86,8 +93,18 @@ int moc_plan_create(const moc_problem *problem, moc_plan **out);
 int moc_plan_destroy(moc_plan *plan);
 
 /* Bytes of caller-owned scratch that moc_route / moc_attend (with_bwd = 0) or also
- * moc_attend_bwd (with_bwd = 1) need. */
+ * moc_attend_bwd (with_bwd = 1) need.  The largest part is the routed partial outputs (Sec. 3.3:
+ * every routed (query, chunk) pair is one attention problem; its normalised result and log-sum-exp
+ * wait in the workspace until the query's anchor pass merges them): k times the size of O for the
+ * heads in flight.  Attention runs over groups of heads so that this part stays within a budget
+ * (6 GiB by default; one head at a time is the floor). */
 int moc_workspace_bytes(const moc_plan *plan, int with_bwd, size_t *bytes);
+
+/* Chooses the heads per group so that moc_workspace_bytes(plan, 0) <= max_bytes (the with_bwd size
+ * adds 4 H L bytes).  MOC_ERR_TOO_LARGE, and the plan unchanged, if one head at a time still needs
+ * more.  Call it before asking for the size and allocating; a workspace laid out under another
+ * budget must be routed again. */
+int moc_plan_set_workspace_budget(moc_plan *plan, size_t max_bytes);
 
 /* Step 1 - chunk descriptors (Eq. 3 text: phi = mean pooling of the chunk's keys).
  * desc[h][c][:] = mean over t in chunk c of K[h][t][:], accumulated in fp32. */
@@ -107,8 +124,9 @@ int moc_chunk_pool(const moc_plan *plan, const void *K, float *desc, void *ws, v
  *   16384 (head, chunk) pairs, must use moc_chunk_pool with a workspace).
  *   K, desc: as for moc_chunk_pool; the caller still owns inputs and outputs.
  *   The call itself allocates nothing (no cudaMalloc / cudaFree, no allocating library call).
- *   The first call on each device looks up the array's device address; make that first call
- *   before starting any stream capture on that device.
+ *   The array's device address is looked up once per device, in the first moc_plan_create on that
+ *   device (which also makes the driver load the array there, so this call never has to); a plan
+ *   must exist before this call anyway.  Create the first plan before starting any stream capture.
  *   All calls share the one array, which keeps whatever the previous call left (the counters are
  *   cleared on the stream at the start of every call): two calls that may overlap on the GPU
  *   (different streams, no ordering between them) race on it - serialise them. */
@@ -120,13 +138,28 @@ int moc_chunk_pool_noalloc(const moc_plan *plan, const void *K, float *desc, voi
  * dot product: each fp32 descriptor enters as the exact sum of three bf16 terms, products are
  * exact and the accumulation is fp32); sel_idx gets the min(k, #candidates) best, ties to the
  * lower index.  Also rebuilds, in ws, the per-(head, chunk) lists of the queries that picked
- * it and the routed work items of moc_attend / moc_attend_bwd.  MOC_ERR_SHAPE if the chunk
- * count is beyond what the kernel's shared-memory tables hold (about 8000 chunks). */
+ * it and the routed work items of moc_attend / moc_attend_bwd, and marks ws as holding this
+ * plan's lists.  MOC_ERR_SHAPE if the chunk count is beyond what the kernel's shared-memory
+ * tables hold (about 8000 chunks). */
 int moc_route(const moc_plan *plan, const void *Q, const float *desc, int32_t *sel_idx, void *ws, void *stream);
+
+/* Sec. 3.3 ("head/tail indices of the selected chunks are gathered ... for the attention call"):
+ * rebuilds the chunk -> query lists and the routed work items in ws from a sel_idx that the caller
+ * has edited after moc_route (the context drop-off / drop-in of Sec. 3.1 is such an edit), so that
+ * moc_attend / moc_attend_bwd attend over exactly that selection.  An entry is kept if it names a
+ * chunk that may be routed to from its row (0 <= j < C, not an anchor of the row's chunk, strictly
+ * earlier when the plan is causal) and does not repeat an earlier slot of the row; every other entry
+ * is an empty slot and is overwritten with -1, so that afterwards sel_idx states the selection in force.
+ * Slots need not be sorted or packed to the front. */
+int moc_lists_from_sel(const moc_plan *plan, int32_t *sel_idx, void *ws, void *stream);
 
 /* Step 6 - sparse attention (Eq. 2): O_i = softmax(scale q_i K_Omega^T) V_Omega over the
  * tokens of the chunks in Omega(i) = anchors(c(i)) U sel_idx[i]; lse as defined above.
- * bf16 products, fp32 accumulation and softmax. */
+ * bf16 products, fp32 accumulation and softmax.
+ * The kernels walk the selection through the lists that moc_route or moc_lists_from_sel left in
+ * ws, not through sel_idx: sel_idx must be the array the last of those calls on ws wrote or
+ * checked, unchanged since (after editing it, call moc_lists_from_sel).  A ws that does not hold
+ * this plan's lists makes every block return at once with device status MOC_ERR_WORKSPACE. */
 int moc_attend(const moc_plan *plan, const void *Q, const void *K, const void *V, const int32_t *sel_idx,
                void *O, float *lse, void *ws, void *stream);
 
@@ -134,18 +167,21 @@ int moc_attend(const moc_plan *plan, const void *Q, const void *K, const void *V
  * differentiated, gradients reach Q, K, V only through the attention over selected
  * chunks; none flows through the descriptors or scores).  bf16 products (P and dS are rounded
  * to bf16 before their contractions), fp32 accumulation.  Needs with_bwd workspace, written by
- * moc_route and moc_attend for the same inputs; overwrites the forward's routed partials. */
+ * moc_route (or moc_lists_from_sel) and moc_attend for the same inputs; overwrites the forward's
+ * routed partials.  sel_idx: as for moc_attend. */
 int moc_attend_bwd(const moc_plan *plan, const void *Q, const void *K, const void *V, const void *O,
                    const float *lse, const void *dO, const int32_t *sel_idx, void *dQ, void *dK, void *dV,
                    void *ws, void *stream);
 
-/* Number of selected (query, key-token) pairs summed over all heads and queries, from the
- * plan's anchor tables and a HOST copy of the per-(head, chunk) pick counts is not needed:
- * this reads the counts that moc_route left in ws (synchronises `stream`). */
+/* Number of selected (query, key-token) pairs summed over all heads and queries (the unit of
+ * the FLOP count of Sec. 3.3: 4 d per pair forward): the anchor pairs follow from the plan's
+ * tables, the routed pairs from the per-(head, chunk) pick counts that moc_route or
+ * moc_lists_from_sel left in ws.  Copies those counts to the host: synchronises `stream`. */
 int moc_selected_pairs(const moc_plan *plan, const void *ws, void *stream, int64_t *pairs);
 
-/* Reads the device status word of ws (synchronous copy on `stream`): MOC_OK or
- * MOC_ERR_TIMEOUT, with `detail` (optional) receiving a kernel-specific code. */
+/* Reads the device status word of ws (synchronous copy on `stream`): MOC_OK, MOC_ERR_TIMEOUT
+ * or MOC_ERR_WORKSPACE, with `detail` (optional) receiving a kernel-specific code (for a
+ * timeout, which wait gave up). */
 int moc_get_status(const moc_plan *plan, const void *ws, void *stream, int *device_status, int *detail);
 
 /* How many kernel launches the library has enqueued since it was loaded. */

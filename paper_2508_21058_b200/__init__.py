@@ -3,8 +3,8 @@
 The binding only marshals arguments; every step of the path runs in the library's CUDA
 kernels.  Loading fails loudly if ``libmoc.so`` is missing: there is no CPU fallback.
 """
-from .binding import (MocError, MocPlan, FLAG_CAUSAL, FLAG_SCALAR_ATTEND, WHOLE_SHOT, lib_path, load_library,
+from .binding import (MocError, MocPlan, FLAG_CAUSAL, WHOLE_SHOT, lib_path, load_library,
                       launch_count)
 
-__all__ = ["MocError", "MocPlan", "FLAG_CAUSAL", "FLAG_SCALAR_ATTEND", "WHOLE_SHOT", "lib_path", "load_library",
+__all__ = ["MocError", "MocPlan", "FLAG_CAUSAL", "WHOLE_SHOT", "lib_path", "load_library",
            "launch_count"]

@@ -10,7 +10,6 @@ import torch
 
 _DIR = os.path.dirname(os.path.abspath(__file__))
 FLAG_CAUSAL = 0x1
-FLAG_SCALAR_ATTEND = 0x2
 WHOLE_SHOT = -1
 
 
@@ -31,7 +30,9 @@ _lib = None
 
 
 def lib_path() -> str:
-    return os.path.join(_DIR, "libmoc.so")
+    """The library this process loads: libmoc.so beside this file, or (MOC_LIBRARY=debug) the build with
+    index checks, libmoc_debug.so."""
+    return os.path.join(_DIR, "libmoc_debug.so" if os.environ.get("MOC_LIBRARY") == "debug" else "libmoc.so")
 
 
 def load_library():
@@ -50,7 +51,13 @@ def load_library():
     lib.moc_workspace_bytes.argtypes = [vp, i32, C.POINTER(sz)]
     lib.moc_chunk_pool.argtypes = [vp, vp, vp, vp, vp]
     lib.moc_chunk_pool_noalloc.argtypes = [vp, vp, vp, vp]
+    lib.moc_plan_set_workspace_budget.argtypes = [vp, sz]
     lib.moc_route.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.moc_lists_from_sel.argtypes = [vp, vp, vp, vp]
+    # test hooks (exported, not in the public header)
+    lib.moc_debug_use_cuda_core_attention.argtypes = [vp, i32]
+    lib.moc_debug_set_wait_limit_us.argtypes = [vp, C.c_uint]
+    lib.moc_debug_wait_probe.argtypes = [vp, vp, i32, vp]
     lib.moc_attend.argtypes = [vp] * 9
     lib.moc_attend_bwd.argtypes = [vp] * 13
     lib.moc_selected_pairs.argtypes = [vp, vp, vp, C.POINTER(C.c_int64)]
@@ -94,13 +101,15 @@ class MocPlan:
         off = np.ascontiguousarray(chunk_off, np.int32)
         shot = np.ascontiguousarray(chunk_shot, np.int32)
         mod = np.ascontiguousarray(chunk_mod, np.uint8)
-        flags = (FLAG_CAUSAL if causal else 0) | (FLAG_SCALAR_ATTEND if scalar_attend else 0)
+        flags = FLAG_CAUSAL if causal else 0
         pr = _Problem(int(n_heads), int(n_tokens), int(head_dim), len(shot), int(top_k), int(win_back), int(win_fwd),
                       flags, float(softmax_scale), off.ctypes.data, shot.ctypes.data, mod.ctypes.data)
         if len(off) != len(shot) + 1 or len(mod) != len(shot):
             raise MocError(-3, "moc error -3: chunk tables have inconsistent lengths")
         _check(self._lib.moc_plan_create(C.byref(pr), C.byref(self._h)))
         self.H, self.L, self.d, self.C, self.k = int(n_heads), int(n_tokens), int(head_dim), len(shot), int(top_k)
+        if scalar_attend:       # test hook: the in-library CUDA-core cross-check of the attention kernels
+            _check(self._lib.moc_debug_use_cuda_core_attention(self._h, 1))
 
     @classmethod
     def from_workload(cls, wl, n_heads=None, **kw):
@@ -124,6 +133,9 @@ class MocPlan:
         _check(self._lib.moc_workspace_bytes(self._h, int(with_bwd), C.byref(n)))
         return int(n.value)
 
+    def moc_plan_set_workspace_budget(self, max_bytes: int):
+        _check(self._lib.moc_plan_set_workspace_budget(self._h, C.c_size_t(int(max_bytes))))
+
     def new_workspace(self, with_bwd=False, device="cuda") -> torch.Tensor:
         return torch.empty(self.workspace_bytes(with_bwd), dtype=torch.uint8, device=device)
 
@@ -137,6 +149,9 @@ class MocPlan:
 
     def moc_route(self, Q, desc, sel_idx, ws):
         _check(self._lib.moc_route(self._h, _ptr(Q), _ptr(desc), _ptr(sel_idx), _ptr(ws), _stream()))
+
+    def moc_lists_from_sel(self, sel_idx, ws):
+        _check(self._lib.moc_lists_from_sel(self._h, _ptr(sel_idx), _ptr(ws), _stream()))
 
     def moc_attend(self, Q, K, V, sel_idx, O, lse, ws):
         _check(self._lib.moc_attend(self._h, _ptr(Q), _ptr(K), _ptr(V), _ptr(sel_idx), _ptr(O), _ptr(lse), _ptr(ws),
@@ -155,6 +170,13 @@ class MocPlan:
         st, det = C.c_int(0), C.c_int(0)
         _check(self._lib.moc_get_status(self._h, _ptr(ws), _stream(), C.byref(st), C.byref(det)))
         return int(st.value), int(det.value)
+
+    # test hooks
+    def debug_set_wait_limit_us(self, us: int):
+        _check(self._lib.moc_debug_set_wait_limit_us(self._h, int(us)))
+
+    def debug_wait_probe(self, ws, code: int):
+        _check(self._lib.moc_debug_wait_probe(self._h, _ptr(ws), int(code), _stream()))
 
     # convenience: allocate outputs and run the forward path
     def forward(self, Q, K, V, ws=None):

@@ -41,12 +41,14 @@ enum BwdWait { BW_XFULL = 64, BW_YFULL, BW_YEMPTY, BW_T1FULL, BW_T2FULL, BW_PDON
 struct BwdParams {
     const __nv_bfloat16 *Q, *K, *V, *dO;
     const float *lse, *delta;
-    const int32_t *sel;
     __nv_bfloat16 *dQ, *dK, *dV;
-    __nv_bfloat16 *part;          // [H][L][k][d] routed dQ partials
+    __nv_bfloat16 *part;          // [Hg][L][k][d] routed dQ partials of the group of heads in flight
+    const float *part_lse;        // [H][L][k] the forward's routed log-sum-exps: -inf marks an empty slot
     const KeyRange *rng;          // dQ modes: key ranges the items index
     const WorkItem *items;
-    const int *n_items_dev;       // routed mode: item count on the device
+    const int *item_lo_dev, *item_hi_dev;   // routed mode: the group's item range [*lo, *hi) on the device
+    int h0;                       // first head of the group in flight
+    uint32_t cookie;              // what the workspace's status area must hold
     const KTile *ktiles;          // dK/dV mode
     const int32_t *off, *ranc_off, *ranc, *cap_off;
     const int *cnt;
@@ -58,21 +60,6 @@ struct BwdParams {
 };
 
 constexpr int kY1Stages = 3, kY2Stages = 2;   // stages of the streamed tiles Y1 (read twice per tile) and Y2
-// Optional cycle-stamp tracing of one CTA per mode (build with -DMOC_TRACE): each hook stores clock64()
-// into a slot of g_trace_bwd, read back with moc_trace_read_bwd().  Compiled out otherwise.
-// slot map: 0 start, 1 TMEM ready, 2 X staged, 3 epilogue begins, 4 epilogue done; lanes, tile j: 16 + 8 j +
-// {0 T1 ready, 1 P done, 2 T2 ready, 3 dS done}; issuer, tile j: 1024 + 8 j + {0 T1, 1 T2, 2 ACC1, 3 ACC2}
-// (stamped after the step's wait); producer, tile j: 1536 + 4 j + {0 stages free, 1 copies done or issued}.
-#ifdef MOC_TRACE
-__device__ long long g_trace_bwd[3][2048];
-#define BTRACE_CTA (MODE == DQ_ROUTED ? blockIdx.x == 5000 : MODE == DQ_ANCHOR ? (blockIdx.x == 70 && blockIdx.y == 3) : (blockIdx.x == 100 && blockIdx.y == 3))
-#define BTRACE(slot) do { if (BTRACE_CTA) g_trace_bwd[MODE][(slot)] = clock64(); } while (0)
-#define BTRACE_J(base, stride, j, k) do { if ((j) < 60) BTRACE((base) + (stride) * (j) + (k)); } while (0)
-#else
-#define BTRACE(slot) ((void)0)
-#define BTRACE_J(base, stride, j, k) ((void)0)
-#endif
-
 constexpr int kBwdThreads = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -104,10 +91,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
     constexpr int X_FULL = 0, Y1_FULL = 1, Y1_EMPTY = 4, Y2_FULL = 7, Y2_EMPTY = 9, T1_FULL = 11, T2_FULL = 13,
                   P_HALF = 15, P_DONE = 16, DS_DONE = 17, ACC_FULL = 19, T1_ISSUED = 20, RD1 = 21, RD2 = 22;
 
-    if (threadIdx.x == 0) BTRACE(0);
     if (threadIdx.x == 0) {
         s_abort = 0;
         int valid = (*(volatile int *)p.status == 0);
+        if (valid && (uint32_t)((volatile int *)p.status)[ST_COOKIE] != p.cookie) {
+            atomicCAS(p.status, 0, MOC_ERR_WORKSPACE);      // not this plan's lists: report, touch nothing else
+            valid = 0;
+        }
         uint32_t dyn_bytes;
         asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_bytes));
         if (valid && (sbase - smem_u32(smem_raw)) + (uint32_t)N_TILES_SMEM * TILE_BYTES > dyn_bytes) {
@@ -116,11 +106,21 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             valid = 0;
         }
         if (MODE != DKV) {
-            const int item = blockIdx.x >> 1, half = blockIdx.x & 1;
-            if (MODE == DQ_ROUTED && valid && item >= *p.n_items_dev) valid = 0;
+            int item = blockIdx.x >> 1;
+            const int half = blockIdx.x & 1;
+            if (MODE == DQ_ROUTED && valid) {
+                item += *p.item_lo_dev;
+                if (item >= *p.item_hi_dev) valid = 0;
+            }
+            WorkItem w = {};
             if (valid) {
-                const WorkItem w = p.items[item];
-                w_h = MODE == DQ_ROUTED ? w.h : (int)blockIdx.y;
+                w = p.items[item];
+                if (MODE == DQ_ROUTED && !index_ok((unsigned)w.h < (unsigned)p.H && w.rows > 0 && w.rows <= kQTileRows && w.first >= 0 &&
+                                                   (size_t)w.first + w.rows <= p.cap_total && w.nrng == 1, p.status, IX_BWD_ITEM_FIELDS))
+                    valid = 0;
+            }
+            if (valid) {
+                w_h = MODE == DQ_ROUTED ? w.h : p.h0 + (int)blockIdx.y;
                 w_first = w.first + half * 128;
                 w_rows = min(128, w.rows - half * 128);
                 w_rng = p.rng + w.rng_off;
@@ -179,7 +179,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
     // TMEM columns: T1 [0,128)  T2 [128,256)  ACC1 [256,384)  ACC2 [384,512); the dQ modes have no ACC2
     // and use its columns as a second T2, for the odd tiles
     const uint32_t tmem = tmem_slot;
-    if (threadIdx.x == 0) BTRACE(1);
     const int h = w_h, rows = w_rows, n_tiles = w_ntiles;
     volatile int *abort_flag = &s_abort;
 
@@ -192,7 +191,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
         const int r = threadIdx.x & 127;              // row of the stationary tile = TMEM lane
         const int half = warp >> 2;
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-        int qi = -1, slot = 0, n_sel = 0;             // n_sel: routed picks of the query (anchor mode)
+        int qi = -1, slot = 0;
         float lse2 = INFINITY, dlt = 0.f;             // dQ modes: this lane's query
         if (MODE != DKV) {
             if (r < rows) {
@@ -200,14 +199,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     const int e = p.qlist[(size_t)h * p.cap_total + w_first + r];
                     qi = e / p.k;
                     slot = e - qi * p.k;
+                    (void)index_ok(e >= 0 && qi < p.L, p.status, IX_BWD_LIST_ENTRY);
+                    if ((unsigned)qi >= (unsigned)p.L) qi = -1;      // never follow an entry that is not a row of this head
                 } else {
                     qi = w_first + r;
                 }
-                lse2 = p.lse[(size_t)h * p.L + qi] * kLog2e;
-                dlt = p.delta[(size_t)h * p.L + qi];
-                if (MODE == DQ_ANCHOR) {               // picks come first, -1 padding after them
-                    const int32_t *sel = p.sel + ((size_t)h * p.L + qi) * p.k;
-                    for (int s = 0; s < p.k; ++s) n_sel += sel[s] >= 0;
+                if (qi >= 0) {
+                    lse2 = p.lse[(size_t)h * p.L + qi] * kLog2e;
+                    dlt = p.delta[(size_t)h * p.L + qi];
                 }
             }
             // stage the item's rows, one half Q and the other dO: consecutive threads take consecutive 16-byte pieces
@@ -231,7 +230,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             }
             fence_proxy_async_smem();
             mbar_arrive(bar(X_FULL));
-            if (threadIdx.x == 0) BTRACE(2);
         }
         const float c = p.scale_log2;
         TileIter it(w_rng, MODE == DKV ? 0 : w_nrng);
@@ -246,7 +244,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            if (threadIdx.x == 0) BTRACE_J(16, 8, jt, 0);
             // ---- P = exp2(scale log2(e) S - lse log2(e)) from T1
             const uint32_t t2c = (MODE != DKV && st) ? 384u : 128u;       // T2 (then dS) of this tile
             float pv[64];
@@ -295,13 +292,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 tc_fence_before();
                 mbar_arrive(bar(P_DONE));
             }
-            if (threadIdx.x == 0) BTRACE_J(16, 8, jt, 1);
             // ---- dS = P (dP - delta) from T2, written over T2 columns that have been read
             ok = mbar_wait_spin(bar(T2_FULL + st), (jt >> 1) & 1, abort_flag, p.status, BW_T2FULL);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            if (threadIdx.x == 0) BTRACE_J(16, 8, jt, 2);
 #pragma unroll
             for (int rd = 0; rd < 2; ++rd) {
                 const int ch = rd * 2 + half;
@@ -329,7 +324,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(DS_DONE + st));
-            if (threadIdx.x == 0) BTRACE_J(16, 8, jt, 3);
             if (++s3 == kY1Stages) { s3 = 0; ph3 ^= 1; }
         }
         // ---- epilogue
@@ -339,7 +333,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
         }
         if (ok) {
             tc_fence_after();
-            if (threadIdx.x == 0) BTRACE(3);
 #pragma unroll 1
             for (int ch = half; ch < D / 32; ch += 2) {
                 uint32_t v[32];
@@ -361,18 +354,22 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     }
                 };
                 if (MODE == DQ_ROUTED) {
-                    if (qi >= 0) store_row(p.part + (((size_t)h * p.L + qi) * p.k + slot) * D + ch * 32);
+                    if (qi >= 0) store_row(p.part + (((size_t)(h - p.h0) * p.L + qi) * p.k + slot) * D + ch * 32);
                 } else if (MODE == DQ_ANCHOR) {
                     if (qi >= 0) {
-                        // the routed partials of this query, four slots requested together
-                        const uint4 *src = reinterpret_cast<const uint4 *>(p.part + ((size_t)h * p.L + qi) * p.k * D + ch * 32);
-                        for (int s0 = 0; s0 < n_sel; s0 += 4) {
+                        // the routed partials of this query, four slots requested together; a slot is in use
+                        // if the forward left a finite log-sum-exp for it
+                        const uint4 *src = reinterpret_cast<const uint4 *>(p.part + ((size_t)(h - p.h0) * p.L + qi) * p.k * D + ch * 32);
+                        const float *pl = p.part_lse + ((size_t)h * p.L + qi) * p.k;
+                        for (int s0 = 0; s0 < p.k; s0 += 4) {
                             uint4 raw[4][4];
 #pragma unroll
-                            for (int u = 0; u < 4; ++u)
+                            for (int u = 0; u < 4; ++u) {
+                                const bool used = s0 + u < p.k && pl[s0 + u] != -INFINITY;
 #pragma unroll
                                 for (int q4 = 0; q4 < 4; ++q4)
-                                    raw[u][q4] = s0 + u < n_sel ? __ldcg(src + (size_t)(s0 + u) * (D / 8) + q4) : make_uint4(0, 0, 0, 0);
+                                    raw[u][q4] = used ? __ldcg(src + (size_t)(s0 + u) * (D / 8) + q4) : make_uint4(0, 0, 0, 0);
+                            }
 #pragma unroll
                             for (int u = 0; u < 4; ++u)
 #pragma unroll
@@ -400,7 +397,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 }
             }
         }
-        if (threadIdx.x == 0) BTRACE(4);
     } else if (warp < 12) {
         // ------------------------------------------------------------ producers
         asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
@@ -413,7 +409,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 while (it.next(t0, valid)) {
                     const int s2 = jt & 1;
                     if (!mbar_wait(bar(Y1_EMPTY + s3), ph3 ^ 1, abort_flag, p.status, BW_YEMPTY)) break;
-                    BTRACE_J(1536, 4, jt, 0);
                     mbar_expect_tx(bar(Y1_FULL + s3), TILE_BYTES);
 #pragma unroll
                     for (int sub = 0; sub < SUB; ++sub)
@@ -424,7 +419,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
 #pragma unroll
                     for (int sub = 0; sub < SUB; ++sub)
                         tma_load_2d(sY2 + s2 * TILE_BYTES + sub * SUB_BYTES, &tmV, sub * 64, h * p.L + t0, bar(Y2_FULL + s2));
-                    BTRACE_J(1536, 4, jt, 1);
                     ++jt;
                     if (++s3 == kY1Stages) { s3 = 0; ph3 ^= 1; }
                 }
@@ -470,7 +464,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 }
                 q = -1;
                 if (r0 < r1) { if (r0 + i < r1) q = r0 + i; }
-                else if (e0 + i < n_list) q = list[e0 + i] / p.k;
+                else if (e0 + i < n_list && index_ok((size_t)p.cap_off[chunk] + e0 + i < p.cap_total, p.status, IX_BWD_LIST_POSITION)) {
+                    q = list[e0 + i] / p.k;
+                    if (!index_ok((unsigned)q < (unsigned)p.L, p.status, IX_BWD_LIST_ENTRY)) q = -1;
+                }
                 if (r0 < r1) r0 += 128; else e0 += 128;
                 // a column without a query gets lse = +inf: its P and dS come out as exact zeros
                 q_lse = q >= 0 ? p.lse[(size_t)h * p.L + q] * kLog2e : INFINITY;
@@ -485,7 +482,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 if (jt >= 2) ok = ok && mbar_wait(bar(DS_DONE + s2), ((jt - 2) >> 1) & 1, abort_flag, p.status, BW_DSDONE);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (warp == 8 && lane == 0) BTRACE_J(1536, 4, jt, 0);
                 s_ld[s2][0][i] = q_lse;
                 s_ld[s2][1][i] = q_del;
                 constexpr int RP = 32 / CH;                    // rows per instruction
@@ -504,7 +500,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 fence_proxy_async_smem();
                 mbar_arrive(bar(Y1_FULL + s3));
                 mbar_arrive(bar(Y2_FULL + s2));
-                if (warp == 8 && lane == 0) BTRACE_J(1536, 4, jt, 1);
                 if (++s3 == kY1Stages) { s3 = 0; ph3 ^= 1; }
             }
         }
@@ -530,17 +525,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             // the MMA groups, without their waits and commits
             // (s3 = j mod the Y1 stage count is carried along by the callers: no division on this thread)
             auto t1 = [&](int j, int s3) {  // T1(j) = X1 Y1(j)^T
-                BTRACE_J(1024, 8, j, 0);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t o = ((ks >> 2) * SUB_BYTES + (ks & 3) * 32) >> 4;
                     mma_ss_lo(tmem, lo(x1) + o, hi(x1), lo(y1k) + s3 * (uint32_t)STAGE + o, hi(y1k), IDESC_T, ks > 0);
                 }
-                BTRACE_J(1024, 8, j, 4);
             };
             auto t2 = [&](int j) {          // T2(j) = X2 Y2(j)^T
                 const int s2 = j & 1;
-                BTRACE_J(1024, 8, j, 1);
                 const uint32_t d = tmem + ((MODE != DKV && s2) ? 384u : 128u);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
@@ -549,7 +541,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 }
             };
             auto acc1 = [&](int j, int s3) {   // ACC1 += dS(j) Y1(j)
-                BTRACE_J(1024, 8, j, 2);
                 const uint32_t ds = tmem + ((MODE != DKV && (j & 1)) ? 384u : 128u);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
@@ -557,7 +548,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
             };
             auto acc2 = [&](int j, int half) {   // ACC2 += P(j) Y2(j), the K steps of one half of P
                 const int s2 = j & 1;
-                if (half == 0) BTRACE_J(1024, 8, j, 3);
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
                     mma_ts_lo(tmem + 384, tmem + (half * 4 + ks) * 8, lo(y2m) + s2 * (uint32_t)STAGE + (half * 4 + ks) * (2048 >> 4), hi(y2m),
@@ -590,14 +580,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                     if (more) wait(Y1_FULL + s3n, ph3n, BW_YFULL);
                     if (MODE == DKV || more) wait(P_DONE, j & 1, BW_PDONE);
                     if (!ok) break;
-                    BTRACE_J(1024, 8, j, 6);
                     tc_fence_after();
                     if (MODE == DKV) acc2(j, 1);
-                    BTRACE_J(1024, 8, j, 7);
                     if (more) {
                         t1(j + 1, s3n);
                         tc_commit(bar(T1_FULL + ((j + 1) & 1)));
-                        BTRACE_J(1024, 8, j + 1, 5);
                     }
                     if (++s3n == kY1Stages) { s3n = 0; ph3n ^= 1; }
                     if (MODE == DKV) {
@@ -656,7 +643,9 @@ static int attend_bwd_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv
     if (int r = make_tmap_2d_bf16(&tmK, K, (uint64_t)p->H * p->L, D, 128)) return r;
     if (int r = make_tmap_2d_bf16(&tmV, V, (uint64_t)p->H * p->L, D, 128)) return r;
     BwdParams a;
-    a.Q = Q; a.K = K; a.V = V; a.dO = dO; a.lse = lse; a.delta = delta; a.sel = sel;
+    a.Q = Q; a.K = K; a.V = V; a.dO = dO; a.lse = lse; a.delta = delta;
+    a.part_lse = ws_ptr<float>(ws, p->ws.part_lse);
+    a.cookie = p->cookie; a.h0 = 0; a.item_lo_dev = a.item_hi_dev = nullptr;
     a.dQ = dQ; a.dK = dK; a.dV = dV;
     a.part = ws_ptr<__nv_bfloat16>(ws, p->ws.part_o);      // the forward's partial outputs are no longer needed
     a.ktiles = p->d_ktiles; a.off = p->d_off; a.ranc_off = p->d_ranc_off; a.ranc = p->d_ranc; a.cap_off = p->d_cap_off;
@@ -669,47 +658,45 @@ static int attend_bwd_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv
     // seven tiles (X1 X2, three Y1 stages, two Y2 stages) and the slack that aligns them to 1024 bytes; at
     // d = 128 that is all an SM has, so the request is what the kernel's static variables leave of the limit
     const size_t tiles = (size_t)(2 + kY1Stages + kY2Stages) * 128 * D * 2;
-    static size_t smem_mode[2][3] = {{0, 0, 0}, {0, 0, 0}};
-    if (!smem_mode[D == 128][0]) {
-        int dev = 0, optin = 0;
-        MOC_CUDA_TRY(cudaGetDevice(&dev));
-        MOC_CUDA_TRY(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    size_t smem[3];
+    {
+        int optin = 0;
+        MOC_CUDA_TRY(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, p->device));
         const void *fn[3] = {(const void *)attend_bwd_tc_kernel<D, DQ_ROUTED>, (const void *)attend_bwd_tc_kernel<D, DQ_ANCHOR>,
                              (const void *)attend_bwd_tc_kernel<D, DKV>};
-        size_t got[3];
         for (int m = 0; m < 3; ++m) {
             cudaFuncAttributes fa;
             MOC_CUDA_TRY(cudaFuncGetAttributes(&fa, fn[m]));
-            got[m] = std::min(tiles + 1024, (size_t)optin - fa.sharedSizeBytes);
-            if (got[m] < tiles) return MOC_ERR_SHAPE;
-            MOC_CUDA_TRY(cudaFuncSetAttribute(fn[m], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)got[m]));
+            smem[m] = std::min(tiles + 1024, (size_t)optin - fa.sharedSizeBytes);
+            if (smem[m] < tiles) return MOC_ERR_SHAPE;
+            MOC_CUDA_TRY(cudaFuncSetAttribute(fn[m], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem[m]));
         }
-        for (int m = 2; m >= 0; --m) smem_mode[D == 128][m] = got[m];
     }
-    const size_t *smem = smem_mode[D == 128];
-    if (p->k > 0) {
-        a.rng = p->d_chunk_rng;
-        a.items = ws_ptr<WorkItem>(ws, p->ws.rtiles);
-        a.n_items_dev = ws_ptr<int>(ws, p->ws.tile_off) + (size_t)p->H * p->C;
-        const long long bound = (long long)p->H * (((long long)p->L * p->k + kQTileRows - 1) / kQTileRows + p->C);
-        attend_bwd_tc_kernel<D, DQ_ROUTED><<<(unsigned)(2 * bound), kBwdThreads, smem[DQ_ROUTED], s>>>(tmK, tmV, a);
+    // dQ group by group of heads (the routed mode leaves the group's partials in the workspace, the
+    // anchor mode adds them up), then dK / dV of every key tile
+    const int *tile_off = ws_ptr<int>(ws, p->ws.tile_off);
+    for (int h0 = 0; h0 < p->H; h0 += p->heads_per_group) {
+        const int hg = std::min(p->heads_per_group, p->H - h0);
+        a.h0 = h0;
+        if (p->k > 0) {
+            a.rng = p->d_chunk_rng;
+            a.items = ws_ptr<WorkItem>(ws, p->ws.rtiles);
+            a.item_lo_dev = tile_off + (size_t)h0 * p->C;
+            a.item_hi_dev = tile_off + (size_t)(h0 + hg) * p->C;
+            const long long bound = (long long)hg * (((long long)p->L * p->k + kQTileRows - 1) / kQTileRows + p->C);
+            attend_bwd_tc_kernel<D, DQ_ROUTED><<<(unsigned)(2 * bound), kBwdThreads, smem[DQ_ROUTED], s>>>(tmK, tmV, a);
+            MOC_LAUNCH_CHECK();
+        }
+        a.rng = p->d_anc_rng;
+        a.items = p->d_qitems;
+        a.item_lo_dev = a.item_hi_dev = nullptr;
+        attend_bwd_tc_kernel<D, DQ_ANCHOR><<<dim3((unsigned)(2 * p->qitems.size()), (unsigned)hg), kBwdThreads, smem[DQ_ANCHOR], s>>>(tmK, tmV, a);
         MOC_LAUNCH_CHECK();
     }
-    a.rng = p->d_anc_rng;
-    a.items = p->d_qitems;
-    a.n_items_dev = nullptr;
-    attend_bwd_tc_kernel<D, DQ_ANCHOR><<<dim3((unsigned)(2 * p->qitems.size()), (unsigned)p->H), kBwdThreads, smem[DQ_ANCHOR], s>>>(tmK, tmV, a);
-    MOC_LAUNCH_CHECK();
     attend_bwd_tc_kernel<D, DKV><<<dim3((unsigned)p->ktiles.size(), (unsigned)p->H), kBwdThreads, smem[DKV], s>>>(tmK, tmV, a);
     MOC_LAUNCH_CHECK();
     return MOC_OK;
 }
-
-#ifdef MOC_TRACE
-extern "C" int moc_trace_read_bwd(long long *host, int n) {
-    return (int)cudaMemcpyFromSymbol(host, g_trace_bwd, sizeof(long long) * (size_t)n);
-}
-#endif
 
 int launch_attend_bwd_tc(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
                          const __nv_bfloat16 *O, const float *lse, const __nv_bfloat16 *dO, const int32_t *sel,

@@ -27,30 +27,14 @@
 //   warp 11    idle (fills the third warpgroup).
 // Every mbarrier wait is bounded; a wait that runs out flags the workspace status word
 // and the CTA drains and leaves.
+#include <algorithm>
+
 #include "moc_common.cuh"
 #include "moc_tc.cuh"
 
 namespace moc {
 
 using namespace tc;
-
-// Optional cycle-stamp tracing of one CTA per pass (build with -DMOC_TRACE): each hook stores
-// clock64() into a slot of g_trace, read back with moc_trace_read().  Compiled out otherwise.
-#ifdef MOC_TRACE
-__device__ long long g_trace[8192];
-// -DMOC_TRACE_PASS=1 stamps the routed pass only, =0 the anchor pass only; by default both write (the anchor pass last)
-#ifndef MOC_TRACE_PASS
-#define MOC_TRACE_PASS 2
-#endif
-#define TRACE_CTA (blockIdx.x == (ROUTED ? 5000 : 70) && (ROUTED || blockIdx.y == 3) && (MOC_TRACE_PASS == 2 || (int)ROUTED == MOC_TRACE_PASS))
-#define TRACE(slot) do { if (TRACE_CTA) g_trace[(slot)] = clock64(); } while (0)
-#else
-#define TRACE(slot) ((void)0)
-#endif
-// slot map: 0 start, 1 TMEM ready, 10+g Q staged, 12+g epilogue begins, 14+g epilogue done;
-// softmax of tile g, key tile j: 100 + 1000 g + 8 j + {0 S ready, 1 S loaded, 2 max known,
-// 3 first half of P stored, 4 exponentials done, 5 P stored};  MMA issuer g: 2100 + 1000 g + 8 j +
-// {0 loop top, 1 K/V ready, 2 first half of P seen, 3 all of P seen, 4 P V issued, 5 next S issued}
 
 struct AttendParams {
     const __nv_bfloat16 *Q;
@@ -59,8 +43,10 @@ struct AttendParams {
     __nv_bfloat16 *part_o;
     float *part_lse;
     const KeyRange *rng;        // key ranges the items index: merged anchor ranges, or the chunks
-    const WorkItem *items;      // anchor pass: one head's items (blockIdx.y = head); routed pass: every item
-    const int *n_items_dev;     // routed pass: the item count lives on the device
+    const WorkItem *items;      // anchor pass: one head's items (blockIdx.y = head - h0); routed pass: every item
+    const int *item_lo_dev, *item_hi_dev;   // routed pass: the group's item range [*lo, *hi) lives on the device
+    int h0;                     // first head of the group in flight (its partials are part_o[h - h0])
+    uint32_t cookie;            // what the workspace's status area must hold
     const int32_t *qlist;       // [H][cap_total]
     size_t cap_total;
     int *status;
@@ -101,14 +87,28 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     // barrier indices
     constexpr int Q_FULL = 0, K_FULL = 2, K_EMPTY = 4, V_FULL = 6, V_EMPTY = 8, S_FULL = 10, P_FULL = 12, O_FULL = 14, TURN = 16, P_HALF = 18;
 
-    if (threadIdx.x == 0) TRACE(0);
     if (threadIdx.x == 0) {
         s_abort = 0;
         int valid = (*(volatile int *)p.status == 0);
-        if (ROUTED && valid && (int)blockIdx.x >= *p.n_items_dev) valid = 0;
+        if (valid && (uint32_t)((volatile int *)p.status)[ST_COOKIE] != p.cookie) {
+            // the workspace does not hold this plan's lists: report, touch nothing else
+            atomicCAS(p.status, 0, MOC_ERR_WORKSPACE);
+            valid = 0;
+        }
+        int item = blockIdx.x;
+        if (ROUTED && valid) {
+            item += *p.item_lo_dev;
+            if (item >= *p.item_hi_dev) valid = 0;
+        }
+        WorkItem w = {};
         if (valid) {
-            const WorkItem w = p.items[blockIdx.x];
-            w_h = ROUTED ? w.h : (int)blockIdx.y;
+            w = p.items[item];
+            if (ROUTED && !index_ok((unsigned)w.h < (unsigned)p.H && w.rows > 0 && w.rows <= kQTileRows && w.first >= 0 &&
+                                    (size_t)w.first + w.rows <= p.cap_total && w.nrng == 1, p.status, IX_ITEM_FIELDS))
+                valid = 0;
+        }
+        if (valid) {
+            w_h = ROUTED ? w.h : p.h0 + (int)blockIdx.y;
             w_first = w.first;
             w_rows = w.rows;
             w_rng = p.rng + w.rng_off;
@@ -140,7 +140,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     __syncthreads();
     tc_fence_after();
 
-    if (threadIdx.x == 0) TRACE(1);
     const uint32_t tmem = tmem_slot;
     const int h = w_h, rows = w_rows, first = w_first, n_tiles = w_ntiles;
     const bool two = rows > 128;            // is query tile 1 populated?
@@ -163,6 +162,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                     const int e = p.qlist[(size_t)h * p.cap_total + first + rt];
                     qi = e / p.k;
                     slot = e - qi * p.k;
+                    (void)index_ok(e >= 0 && qi < p.L, p.status, IX_LIST_ENTRY);
+                    if ((unsigned)qi >= (unsigned)p.L) qi = -1;      // never follow an entry that is not a row of this head
                 } else {
                     qi = first + rt;
                 }
@@ -190,11 +191,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             mbar_arrive(bar(Q_FULL + g));
             if (!ROUTED && qi >= 0) {
                 // the epilogue will merge this row's routed partials: start them on their way into L2 now
-                const char *po = reinterpret_cast<const char *>(p.part_o + ((size_t)h * p.L + qi) * p.k * D);
+                const char *po = reinterpret_cast<const char *>(p.part_o + ((size_t)(h - p.h0) * p.L + qi) * p.k * D);
                 for (int b = 0; b < p.k * D * 2; b += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(po + b));
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(p.part_lse + ((size_t)h * p.L + qi) * p.k));
             }
-            if (r == 0) TRACE(10 + g);
 
             float m_run = -INFINITY, l_run = 0.f;
             const float c = p.scale_log2;
@@ -205,13 +205,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 ok = mbar_wait(bar(S_FULL + g), jt & 1, abort_flag, p.status, W_SFULL);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (r == 0) TRACE(100 + g * 1000 + jt * 8 + 0);
                 tc_fence_after();
                 uint32_t v[4][32];
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) tmem_ld32(tS + ch * 32, v[ch]);
                 tmem_wait_ld();
-                if (r == 0) TRACE(100 + g * 1000 + jt * 8 + 1);
                 if (valid < kBN) {
 #pragma unroll
                     for (int ch = 0; ch < 4; ++ch)
@@ -227,7 +225,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                     for (int x = 0; x < 32; x += 2) m4[ch] = max3(m4[ch], __uint_as_float(v[ch][x]), __uint_as_float(v[ch][x + 1]));
                 }
                 const float m_new = fmaxf(m_run, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * c);
-                if (r == 0) TRACE(100 + g * 1000 + jt * 8 + 2);
                 float alpha = 1.f;
                 if (jt == 0) {
                     m_run = m_new;
@@ -279,22 +276,18 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                         tmem_wait_st();
                         tc_fence_before();
                         mbar_arrive(bar(P_HALF + g));
-                        if (r == 0) TRACE(100 + g * 1000 + jt * 8 + 3);
                     }
                 }
-                if (r == 0) TRACE(100 + g * 1000 + jt * 8 + 4);
                 if (two) mbar_arrive(bar(TURN + g));
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(P_FULL + g));
-                if (r == 0) TRACE(100 + g * 1000 + jt * 8 + 5);
                 float s0, s1;
                 unpack2(add2(sum_a, sum_b), s0, s1);
                 l_run = l_run * alpha + (s0 + s1);
                 ++jt;
             }
             // ---- epilogue
-            if (r == 0) TRACE(12 + g);
             // The merge weights of the routed partials depend only on log-sum-exps: have them ready before
             // the last P V lands.  wslot[s] = exp(lse_s - lse_total), w_own likewise for this pass's own part.
             const float inv_l = 1.f / l_run;
@@ -308,7 +301,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             const __nv_bfloat16 *po = nullptr;
             if (!ROUTED && ok && qi >= 0 && p.k > 0) {
                 pl = p.part_lse + ((size_t)h * p.L + qi) * p.k;
-                po = p.part_o + ((size_t)h * p.L + qi) * p.k * D;
+                po = p.part_o + ((size_t)(h - p.h0) * p.L + qi) * p.k * D;
                 if (p.k <= KW) {
                     float plv[KW];
 #pragma unroll
@@ -390,7 +383,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                         }
                     }
                     if (qi < 0) continue;
-                    __nv_bfloat16 *dst = ROUTED ? p.part_o + (((size_t)h * p.L + qi) * p.k + slot) * D + ch * 32
+                    __nv_bfloat16 *dst = ROUTED ? p.part_o + (((size_t)(h - p.h0) * p.L + qi) * p.k + slot) * D + ch * 32
                                                 : p.O + ((size_t)h * p.L + qi) * D + ch * 32;
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4) {
@@ -499,20 +492,15 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 const int st = jt & 1, sn = (jt + 1) & 1;
                 const uint32_t ph = (jt >> 1) & 1, phn = ((jt + 1) >> 1) & 1;
                 const bool more = it.next(t0, valid_next);
-                TRACE(2100 + g * 1000 + jt * 8 + 0);
                 if (!mbar_wait(bar(V_FULL + st), ph, abort_flag, p.status, W_VFULL)) break;
                 if (more && !mbar_wait(bar(K_FULL + sn), phn, abort_flag, p.status, W_KFULL)) break;
-                TRACE(2100 + g * 1000 + jt * 8 + 1);
                 const int steps = (valid + 15) >> 4, half = min(steps, 4);
                 if (!mbar_wait(bar(P_HALF + g), jt & 1, abort_flag, p.status, W_PHALF)) break;
-                TRACE(2100 + g * 1000 + jt * 8 + 2);
                 tc_fence_after();
                 issue_pv(g, st, 0, half, jt > 0);
                 if (!mbar_wait(bar(P_FULL + g), jt & 1, abort_flag, p.status, W_PFULL)) break;
-                TRACE(2100 + g * 1000 + jt * 8 + 3);
                 tc_fence_after();
                 if (steps > half) issue_pv(g, st, half, steps, true);
-                TRACE(2100 + g * 1000 + jt * 8 + 4);
                 // a commit between two groups of MMAs leaves the pipe idle: the next S goes out first, then all commits
                 if (more) {
                     issue_qk(g, sn, valid_next);
@@ -523,12 +511,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                     tc_commit(bar(V_EMPTY + st));
                     tc_commit(bar(O_FULL + g));
                 }
-                TRACE(2100 + g * 1000 + jt * 8 + 5);
                 valid = valid_next;
             }
         }
     }
-    if (warp < 8 && (threadIdx.x & 127) == 0) TRACE(14 + (warp >> 2));
     tc_fence_before();
     __syncthreads();
     if (warp == 8) tmem_dealloc(tmem, kTmemCols);
@@ -574,39 +560,38 @@ static int attend_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfl
     a.status = ws_ptr<int>(ws, p->ws.status);
     a.H = p->H; a.L = p->L; a.k = p->k;
     a.scale_log2 = p->scale * 1.4426950408889634f;
+    a.cookie = p->cookie;
     // always the d = 128 footprint: more than half an SM's shared memory, so CTAs (which each
     // take all 512 TMEM columns) never share an SM
     const size_t smem = 6 * (size_t)128 * 128 * 2 + 1024;
-    static bool attr_done[2] = {false, false};
-    if (!attr_done[D == 128]) {
-        MOC_CUDA_TRY(cudaFuncSetAttribute(attend_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        MOC_CUDA_TRY(cudaFuncSetAttribute(attend_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_done[D == 128] = true;
-    }
-    if (p->k > 0) {
-        // routed pass: the items and their count were left in the workspace by moc_route; the grid covers
-        // the most there can be
-        a.rng = p->d_chunk_rng;
-        a.items = ws_ptr<WorkItem>(ws, p->ws.rtiles);
-        a.n_items_dev = ws_ptr<int>(ws, p->ws.tile_off) + (size_t)p->H * p->C;
-        const long long bound = (long long)p->H * (((long long)p->L * p->k + kQTileRows - 1) / kQTileRows + p->C);
-        attend_tc_kernel<D, true><<<(unsigned)bound, kThreads, smem, s>>>(tmK, tmV, a);
+    MOC_CUDA_TRY(cudaFuncSetAttribute(attend_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    MOC_CUDA_TRY(cudaFuncSetAttribute(attend_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    // group by group of heads: the routed pass leaves the group's partials in the workspace, the anchor
+    // pass merges them
+    const int *tile_off = ws_ptr<int>(ws, p->ws.tile_off);
+    for (int h0 = 0; h0 < p->H; h0 += p->heads_per_group) {
+        const int hg = std::min(p->heads_per_group, p->H - h0);
+        a.h0 = h0;
+        if (p->k > 0) {
+            // routed pass: the items and their count were left in the workspace with the lists; the grid
+            // covers the most the group can have
+            a.rng = p->d_chunk_rng;
+            a.items = ws_ptr<WorkItem>(ws, p->ws.rtiles);
+            a.item_lo_dev = tile_off + (size_t)h0 * p->C;
+            a.item_hi_dev = tile_off + (size_t)(h0 + hg) * p->C;
+            const long long bound = (long long)hg * (((long long)p->L * p->k + kQTileRows - 1) / kQTileRows + p->C);
+            attend_tc_kernel<D, true><<<(unsigned)bound, kThreads, smem, s>>>(tmK, tmV, a);
+            MOC_LAUNCH_CHECK();
+        }
+        a.rng = p->d_anc_rng;
+        a.items = p->d_qitems;
+        a.item_lo_dev = a.item_hi_dev = nullptr;
+        dim3 grid((unsigned)p->qitems.size(), (unsigned)hg);
+        attend_tc_kernel<D, false><<<grid, kThreads, smem, s>>>(tmK, tmV, a);
         MOC_LAUNCH_CHECK();
     }
-    a.rng = p->d_anc_rng;
-    a.items = p->d_qitems;
-    a.n_items_dev = nullptr;
-    dim3 grid((unsigned)p->qitems.size(), (unsigned)p->H);
-    attend_tc_kernel<D, false><<<grid, kThreads, smem, s>>>(tmK, tmV, a);
-    MOC_LAUNCH_CHECK();
     return MOC_OK;
 }
-
-#ifdef MOC_TRACE
-extern "C" int moc_trace_read(long long *host, int n) {
-    return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * (size_t)n);
-}
-#endif
 
 int launch_attend_tc(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
                      const int32_t *, __nv_bfloat16 *O, float *lse, void *ws, cudaStream_t s) {

@@ -12,7 +12,11 @@ namespace moc {
 
 constexpr int kQTileRows = 256;     // query rows per attention work item (two 128-row MMA tiles)
 constexpr int kPoolSlice = 256;     // tokens per chunk-pool work unit
-constexpr int kStatusWords = 16;    // status area at the head of the workspace (int32 each)
+constexpr int kStatusWords = 16;    // status area at the head of the workspace (int32 each):
+// [0] device status (a moc_status), [1] detail code, [2] cookie of the plan whose lists the workspace holds,
+// [3] limit of every bounded wait in microseconds (0 = the default of one second)
+enum StatusWord { ST_STATUS = 0, ST_DETAIL = 1, ST_COOKIE = 2, ST_WAIT_US = 3 };
+constexpr unsigned kPrivFlagCudaCoreAttend = 0x80000000u;   // plan flag outside the public header: test hook
 
 // One contiguous range of key tokens [t0, t1).
 struct KeyRange { int32_t t0, t1; };
@@ -27,19 +31,18 @@ struct WorkItem { int32_t h, first, rows, ntiles, rng_off, nrng, t0, t1; };
 struct KTile { int32_t chunk, t0, valid, pad; };
 
 struct WsLayout {
-    size_t status;      // int32[kStatusWords]: [0] device status, [1] detail, [2] routed-flag
+    size_t status;      // int32[kStatusWords], see StatusWord
     size_t cnt;         // int32[H][C]     routed picks per (head, chunk); doubles as the list cursor while routing
     size_t tile_off;    // int32[H*C+1]    running count of routed attention tiles over (head, chunk) pairs
     size_t rtiles;      // WorkItem[H * (ceil(L k / 256) + C)]  routed work items, written after routing
     size_t qlist;       // int32[H][cap_total]  per (head, chunk) list at cap_off[c]: entries i*k+s of the picks of c
     size_t desc3;       // bf16 [H][3][Cpad][d]  descriptors split into three bf16 terms (hi + mid + lo)
     size_t pool_part;   // float[H][n_pool_units][d] partial key sums
-    size_t pool_done;   // int32[H][C] arrival counters (self-resetting)
-    size_t part_o;      // bf16 [H][L][k][d] routed partial outputs (normalised)
+    size_t pool_done;   // int32[H][C] arrival counters (cleared at the start of every pooling call)
+    size_t part_o;      // bf16 [Hg][L][k][d] routed partial outputs (normalised) of one group of Hg heads at a time
     size_t part_lse;    // float[H][L][k]    routed partial log-sum-exp (-inf = unused slot)
     size_t fwd_end;
     size_t delta;       // float[H][L]       rowsum(dO * O)
-    size_t dq_acc;      // float[H][L][d]    fp32 dQ accumulator
     size_t bwd_end;
 };
 
@@ -65,6 +68,10 @@ struct moc_plan {
     std::vector<int32_t> cap_off;            // [C+1] start of chunk c's query list inside a head's list area
     int c_pad;                               // C rounded up to a multiple of 16 (MMA N granularity)
     int n_pool_units;
+    int heads_per_group;                     // Hg: heads whose routed partials are held at once (attention runs group by group)
+    size_t partials_budget;                  // bytes the routed partials may take; sets Hg
+    uint32_t cookie;                         // hash of the problem, written into a workspace this plan has routed on
+    uint32_t wait_us;                        // limit of the kernels' bounded waits (0 = default); tests shorten it
     // device tables (one allocation)
     void *d_blob;
     int32_t *d_off, *d_shot, *d_tok_chunk, *d_anc_off, *d_ranc_off, *d_ranc, *d_pool_unit_off, *d_pool_unit_chunk, *d_cap_off;
@@ -107,6 +114,20 @@ template <typename T>
 static inline const T *ws_ptr(const void *ws, size_t off) { return reinterpret_cast<const T *>(static_cast<const char *>(ws) + off); }
 
 #ifdef __CUDACC__
+// Debug build (-DMOC_DEBUG): every index a kernel takes from the workspace (list entries, list positions,
+// work-item fields) is checked before it is used as an address; a bad one records MOC_ERR_INDEX with `code`
+// in the status area and the access is skipped.  In the release build the checks cost nothing.
+enum IndexCheck { IX_ITEM_FIELDS = 200, IX_LIST_POSITION, IX_LIST_ENTRY, IX_APPEND_POSITION, IX_BWD_ITEM_FIELDS,
+                  IX_BWD_LIST_POSITION, IX_BWD_LIST_ENTRY };
+#ifdef MOC_DEBUG
+__device__ __forceinline__ bool index_ok(bool cond, int *status, int code) {
+    if (!cond && atomicCAS(status, 0, MOC_ERR_INDEX) == 0) status[ST_DETAIL] = code;
+    return cond;
+}
+#else
+__device__ __forceinline__ bool index_ok(bool, int *, int) { return true; }
+#endif
+
 // Walks the 128-key tiles of a list of key ranges (a tile never straddles two ranges).
 struct TileIter {
     const KeyRange *rng;
@@ -126,11 +147,15 @@ struct TileIter {
 };
 #endif
 
+void layout_workspace(moc_plan *p);
+
 static inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 // kernels' host launchers (each returns a moc_status)
 int launch_chunk_pool(const moc_plan *p, const __nv_bfloat16 *K, float *desc, void *ws, cudaStream_t s);
 int launch_route(const moc_plan *p, const __nv_bfloat16 *Q, const float *desc, int32_t *sel, void *ws, cudaStream_t s);
+int launch_lists_from_sel(const moc_plan *p, int32_t *sel, void *ws, cudaStream_t s);
+int pool_scratch_prepare(int device);     // looks up (once per device) the fixed scratch array of moc_chunk_pool_noalloc
 int launch_attend_scalar(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
                          const int32_t *sel, __nv_bfloat16 *O, float *lse, void *ws, cudaStream_t s);
 int launch_attend_bwd_scalar(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
@@ -144,3 +169,15 @@ int launch_attend_tc(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloa
                      const int32_t *sel, __nv_bfloat16 *O, float *lse, void *ws, cudaStream_t s);
 
 }  // namespace moc
+
+// Test hooks: exported, but not part of the public header (tests declare them themselves).
+extern "C" {
+// attention and its backward on the plain fp32 CUDA-core kernels (an in-library cross-check that reads
+// the selection straight from sel_idx)
+int moc_debug_use_cuda_core_attention(moc_plan *plan, int on);
+// limit of every bounded device-side wait, in microseconds, for workspaces routed from now on (0 = default)
+int moc_debug_set_wait_limit_us(moc_plan *plan, unsigned us);
+// one block whose only wait is on a barrier that nothing ever arrives on: it must give up after the limit,
+// record MOC_ERR_TIMEOUT with detail `code` in ws, and return
+int moc_debug_wait_probe(const moc_plan *plan, void *ws, int code, void *stream);
+}

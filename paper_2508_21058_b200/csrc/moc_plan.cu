@@ -33,9 +33,17 @@ static bool is_anchor(const moc_plan *p, int c, int j) {
     return true;
 }
 
-static void layout_workspace(moc_plan *p) {
+// Workspace layout.  The routed partial outputs ([heads][L][k][d] bf16, k times the size of O) are held for
+// one group of Hg heads at a time; attention and its backward run group by group.  Hg is the largest
+// even split of the heads whose partials stay within the plan's budget (at least one head).
+void layout_workspace(moc_plan *p) {
     WsLayout &w = p->ws;
     const size_t H = p->H, L = p->L, d = p->d, C = p->C, k = p->k;
+    const size_t per_head = sizeof(__nv_bfloat16) * L * k * d;
+    size_t hg = per_head ? std::max<size_t>(1, p->partials_budget / per_head) : H;
+    hg = std::min(hg, H);
+    const size_t groups = (H + hg - 1) / hg;
+    p->heads_per_group = (int)((H + groups - 1) / groups);
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
     w.status = take(sizeof(int32_t) * kStatusWords);
@@ -46,12 +54,26 @@ static void layout_workspace(moc_plan *p) {
     w.desc3 = take(sizeof(__nv_bfloat16) * H * 3 * (size_t)p->c_pad * d);
     w.pool_part = take(sizeof(float) * H * (size_t)p->n_pool_units * d);
     w.pool_done = take(sizeof(int32_t) * H * C);
-    w.part_o = take(sizeof(__nv_bfloat16) * H * L * k * d);
+    w.part_o = take(per_head * (size_t)p->heads_per_group);
     w.part_lse = take(sizeof(float) * H * L * (k ? k : 1));
     w.fwd_end = o;
     w.delta = take(sizeof(float) * H * L);
-    w.dq_acc = take(sizeof(float) * H * L * d);
     w.bwd_end = o;
+}
+
+// FNV-1a over the problem: a workspace routed by one plan is not accepted by a plan of another problem
+static uint32_t plan_cookie(const moc_plan *p) {
+    uint32_t hsh = 2166136261u;
+    auto mix = [&](const void *data, size_t n) {
+        const unsigned char *b = static_cast<const unsigned char *>(data);
+        for (size_t i = 0; i < n; ++i) { hsh ^= b[i]; hsh *= 16777619u; }
+    };
+    const int32_t hdr[] = {p->H, p->L, p->d, p->C, p->k, p->win_back, p->win_fwd, (int32_t)(p->flags & MOC_FLAG_CAUSAL)};
+    mix(hdr, sizeof hdr);
+    mix(p->off.data(), p->off.size() * 4);
+    mix(p->shot.data(), p->shot.size() * 4);
+    mix(p->mod.data(), p->mod.size());
+    return hsh ? hsh : 1u;
 }
 
 }  // namespace moc
@@ -63,12 +85,14 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
     *out = nullptr;
     if (!pr->chunk_off || !pr->chunk_shot || !pr->chunk_mod) return MOC_ERR_NULL;
     if (pr->n_heads < 1 || pr->n_tokens < 1 || pr->n_chunks < 1 || pr->n_chunks > pr->n_tokens) return MOC_ERR_SHAPE;
+    // heads index grid.y; head * L + token is a 32-bit row coordinate of the tensor maps
+    if (pr->n_heads > 65535 || (double)pr->n_heads * pr->n_tokens >= 2147483647.0) return MOC_ERR_SHAPE;
     if (pr->head_dim != 64 && pr->head_dim != 128) return MOC_ERR_SHAPE;
     if (pr->top_k < 0 || pr->top_k > 512) return MOC_ERR_SHAPE;
     if (pr->win_back < MOC_WHOLE_SHOT || pr->win_fwd < MOC_WHOLE_SHOT) return MOC_ERR_SHAPE;
     if ((double)pr->n_tokens * (pr->top_k ? pr->top_k : 1) >= 2147483647.0) return MOC_ERR_SHAPE;
     if ((double)pr->n_heads * pr->n_chunks >= 1e8) return MOC_ERR_SHAPE;
-    if (pr->flags & ~(MOC_FLAG_CAUSAL | MOC_FLAG_SCALAR_ATTEND)) return MOC_ERR_SHAPE;
+    if (pr->flags & ~MOC_FLAG_CAUSAL) return MOC_ERR_SHAPE;
     if (!(pr->softmax_scale >= 0.f) || isinf(pr->softmax_scale)) return MOC_ERR_SHAPE;
     const int C = pr->n_chunks, L = pr->n_tokens;
     if (pr->chunk_off[0] != 0 || pr->chunk_off[C] != L) return MOC_ERR_CHUNK_TABLE;
@@ -147,7 +171,12 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
         p->cap_off[c + 1] = (int32_t)next;
     }
     p->c_pad = (C + 15) / 16 * 16;
+    p->partials_budget = (size_t)6 << 30;
+    p->wait_us = 0;
+    p->cookie = plan_cookie(p);
     layout_workspace(p);
+    // the fixed scratch of moc_chunk_pool_noalloc: its address is looked up here, where allocating is allowed
+    if (int r = pool_scratch_prepare(dev)) { delete p; return r; }
 
     // one device blob
     size_t o = 0;
@@ -191,6 +220,23 @@ extern "C" int moc_plan_destroy(moc_plan *p) {
     return MOC_OK;
 }
 
+extern "C" int moc_plan_set_workspace_budget(moc_plan *p, size_t max_bytes) {
+    if (!p) return MOC_ERR_NULL;
+    const size_t per_head = sizeof(__nv_bfloat16) * (size_t)p->L * p->k * p->d;
+    const size_t old = p->partials_budget;
+    p->partials_budget = per_head;                       // one head at a time: the smallest workspace there is
+    layout_workspace(p);
+    const size_t rest = p->ws.fwd_end - per_head;
+    if (p->ws.fwd_end > max_bytes) {
+        p->partials_budget = old;
+        layout_workspace(p);
+        return MOC_ERR_TOO_LARGE;
+    }
+    p->partials_budget = std::max(per_head, max_bytes - rest - 4096);
+    layout_workspace(p);
+    return MOC_OK;
+}
+
 extern "C" int moc_workspace_bytes(const moc_plan *p, int with_bwd, size_t *bytes) {
     if (!p || !bytes) return MOC_ERR_NULL;
     *bytes = with_bwd ? p->ws.bwd_end : p->ws.fwd_end;
@@ -230,6 +276,14 @@ extern "C" int moc_route(const moc_plan *p, const void *Q, const float *desc, in
     return launch_route(p, (const __nv_bfloat16 *)Q, desc, sel_idx, ws, (cudaStream_t)stream);
 }
 
+extern "C" int moc_lists_from_sel(const moc_plan *p, int32_t *sel_idx, void *ws, void *stream) {
+    if (int r = enter(p)) return r;
+    if (p->k > 0) { if (int r = check_dev_ptrs({sel_idx}, 4)) return r; }
+    if (!ws) return MOC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return MOC_ERR_ALIGN;
+    return launch_lists_from_sel(p, sel_idx, ws, (cudaStream_t)stream);
+}
+
 extern "C" int moc_attend(const moc_plan *p, const void *Q, const void *K, const void *V, const int32_t *sel_idx,
                           void *O, float *lse, void *ws, void *stream) {
     if (int r = enter(p)) return r;
@@ -239,7 +293,7 @@ extern "C" int moc_attend(const moc_plan *p, const void *Q, const void *K, const
     if (!ws) return MOC_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return MOC_ERR_ALIGN;
     auto q = (const __nv_bfloat16 *)Q, k = (const __nv_bfloat16 *)K, v = (const __nv_bfloat16 *)V;
-    if (p->flags & MOC_FLAG_SCALAR_ATTEND)
+    if (p->flags & kPrivFlagCudaCoreAttend)
         return launch_attend_scalar(p, q, k, v, sel_idx, (__nv_bfloat16 *)O, lse, ws, (cudaStream_t)stream);
     return launch_attend_tc(p, q, k, v, sel_idx, (__nv_bfloat16 *)O, lse, ws, (cudaStream_t)stream);
 }
@@ -253,7 +307,7 @@ extern "C" int moc_attend_bwd(const moc_plan *p, const void *Q, const void *K, c
     if (p->k > 0) { if (int r = check_dev_ptrs({sel_idx}, 4)) return r; }
     if (!ws) return MOC_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return MOC_ERR_ALIGN;
-    auto bwd = (p->flags & MOC_FLAG_SCALAR_ATTEND) ? launch_attend_bwd_scalar : launch_attend_bwd_tc;
+    auto bwd = (p->flags & kPrivFlagCudaCoreAttend) ? launch_attend_bwd_scalar : launch_attend_bwd_tc;
     return bwd(p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, (const __nv_bfloat16 *)O, lse,
                (const __nv_bfloat16 *)dO, sel_idx, (__nv_bfloat16 *)dQ, (__nv_bfloat16 *)dK, (__nv_bfloat16 *)dV, ws,
                (cudaStream_t)stream);
@@ -288,6 +342,18 @@ extern "C" int moc_get_status(const moc_plan *p, const void *ws, void *stream, i
     return MOC_OK;
 }
 
+extern "C" int moc_debug_use_cuda_core_attention(moc_plan *p, int on) {
+    if (!p) return MOC_ERR_NULL;
+    p->flags = on ? (p->flags | kPrivFlagCudaCoreAttend) : (p->flags & ~kPrivFlagCudaCoreAttend);
+    return MOC_OK;
+}
+
+extern "C" int moc_debug_set_wait_limit_us(moc_plan *p, unsigned us) {
+    if (!p) return MOC_ERR_NULL;
+    p->wait_us = us;
+    return MOC_OK;
+}
+
 extern "C" int64_t moc_launch_count(void) { return (int64_t)g_launches.load(); }
 
 extern "C" const char *moc_strerror(int s) {
@@ -297,11 +363,12 @@ extern "C" const char *moc_strerror(int s) {
         case MOC_ERR_SHAPE: return "unsupported shape or parameter";
         case MOC_ERR_CHUNK_TABLE: return "invalid chunk table";
         case MOC_ERR_ALIGN: return "misaligned device pointer";
-        case MOC_ERR_WORKSPACE: return "workspace missing or not routed";
+        case MOC_ERR_WORKSPACE: return "workspace missing, or it does not hold this plan's routing";
         case MOC_ERR_ARCH: return "device is not sm_100 or differs from the plan's device";
         case MOC_ERR_CUDA: return "CUDA runtime error";
         case MOC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
-        case MOC_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the no-allocation entry point";
+        case MOC_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the no-allocation entry point, or the workspace budget";
+        case MOC_ERR_INDEX: return "debug build: an index taken from the workspace was out of range";
         default: return "unknown status";
     }
 }

@@ -132,18 +132,31 @@ constexpr int kMaxDevices = 64;
 static std::mutex g_scratch_mu;
 static unsigned char *g_scratch_addr[kMaxDevices] = {};
 
-// Device address of the scratch array on the current device.  In host code the array's
-// name is only a handle; the address a kernel can use comes from cudaGetSymbolAddress,
-// once per device, with that device current.
-static int pool_scratch_address(int device, unsigned char **out) {
+// Device address of the scratch array on `device`, which must be current.  In host code the array's
+// name is only a handle; the address a kernel can use comes from cudaGetSymbolAddress, once per device.
+// Called from moc_plan_create: the lookup is also what makes the driver load this module (and with it
+// place the array) on the device, so it happens where allocating is allowed and never inside
+// moc_chunk_pool_noalloc; the kernels' attributes are queried for the same reason (their code is loaded).
+int pool_scratch_prepare(int device) {
     if (device < 0 || device >= kMaxDevices) return MOC_ERR_ARCH;
     std::lock_guard<std::mutex> g(g_scratch_mu);
     if (!g_scratch_addr[device]) {
         void *ptr = nullptr;
         MOC_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_pool_scratch));
         if (!ptr) return MOC_ERR_CUDA;
+        cudaFuncAttributes fa;
+        MOC_CUDA_TRY(cudaFuncGetAttributes(&fa, chunk_pool_kernel<128>));
+        MOC_CUDA_TRY(cudaFuncGetAttributes(&fa, chunk_pool_kernel<64>));
+        MOC_CUDA_TRY(cudaFuncGetAttributes(&fa, zero_i32_kernel));
         g_scratch_addr[device] = static_cast<unsigned char *>(ptr);
     }
+    return MOC_OK;
+}
+
+static int pool_scratch_address(int device, unsigned char **out) {
+    if (device < 0 || device >= kMaxDevices) return MOC_ERR_ARCH;
+    std::lock_guard<std::mutex> g(g_scratch_mu);
+    if (!g_scratch_addr[device]) return MOC_ERR_CUDA;      // no plan was ever created on this device
     *out = g_scratch_addr[device];
     return MOC_OK;
 }

@@ -44,18 +44,6 @@ __host__ __device__ constexpr int rt_threads(int ng) { return 64 + 128 * ng + 64
 constexpr int kRtResident = 192;      // up to this many (padded) chunks the whole block stays resident
 constexpr int kRtBlock = 128;         // otherwise chunks are streamed in blocks of this many
 
-// Optional cycle stamps of one CTA (build with -DMOC_TRACE), read back with moc_trace_read_route().
-// slot 0 start; selection group sg, n-th unit of the group: 100 + 1000 sg + 16 n + {0 unit begins,
-// 1 scores ready, 2 selection done, 3 previous unit's lists written, 4 ranks taken, 5 ranges reserved,
-// 6 scores loaded, 8 + r selection round r done};
-// issuer: 3000 + 4 n + {0 inputs ready, 1 accumulator free, 2 MMAs issued, 3 unit begins}
-#ifdef MOC_TRACE
-__device__ long long g_trace_route[8192];
-#define RTRACE(slot) do { if (blockIdx.x == 70 && (slot) < 8192) g_trace_route[(slot)] = clock64(); } while (0)
-#else
-#define RTRACE(slot) ((void)0)
-#endif
-
 enum RouteWait { RW_QFULL = 32, RW_QEMPTY, RW_DFULL, RW_DEMPTY, RW_ACCFULL, RW_ACCEMPTY, RW_GROUP };
 
 template <int KMAX>
@@ -69,13 +57,14 @@ struct TopK {
 };
 
 // desc3[h][t][c][:] for t = 0, 1, 2: bf16 terms of desc[h][c][:] (rows c >= C are zero);
-// also clears the pick counters and the status words.
+// also clears the pick counters and the status words (the workspace holds no plan's lists until they
+// are complete) and states the limit of the bounded waits.  With desc == nullptr only the clearing is done.
 __global__ void route_prep_kernel(const float *__restrict__ desc, __nv_bfloat16 *__restrict__ desc3, int *__restrict__ cnt,
-                                  int *__restrict__ status, int H, int C, int c_pad, int d) {
-    const size_t n = (size_t)H * c_pad * d;
+                                  int *__restrict__ status, int H, int C, int c_pad, int d, unsigned wait_us) {
+    const size_t n = desc ? (size_t)H * c_pad * d : 0;
     const size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
     if (i < (size_t)H * C) cnt[i] = 0;
-    if (i < kStatusWords) status[i] = 0;
+    if (i < kStatusWords) status[i] = i == ST_WAIT_US ? (int)wait_us : 0;
     if (i >= n) return;
     const int x = (int)(i % d);
     const int c = (int)((i / d) % c_pad);
@@ -108,6 +97,7 @@ struct RouteParams {
     int d_rows;             // descriptor rows per term held in shared memory: c_pad (resident) or sb_rows (streamed)
     int q_stages;
     int n_pass;             // selection passes over a tile's scores: 64 picks each (the scores are recomputed per pass)
+    int surv_cap;           // threshold selection: survivor slots per query row in shared memory (0 = not used)
     size_t cap_total;
 };
 
@@ -145,6 +135,8 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     const int hist_ints = (KMAX <= 8 && p.C <= 256 ? 4 : 1) * p.C;
     int *s_cap = hist_base + NG * hist_ints;                             // copy of cap_off[0 .. C)
     uint16_t *s_reach = reinterpret_cast<uint16_t *>(s_cap + p.C);      // chunks in reach of each of this CTA's units
+    // threshold selection: per group, surv_cap slots of (score, column) per query row; slot e of row r at [e][r]
+    float *surv_base = reinterpret_cast<float *>(reinterpret_cast<uintptr_t>(s_reach + p.tiles_per_head / p.ctas_per_head + 16) + 15 & ~(uintptr_t)15);
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     constexpr int Q_FULL = 0, Q_EMPTY = kMaxStages, D_FULL = 2 * kMaxStages, D_EMPTY = D_FULL + 1, ACC_FULL = D_FULL + 2,
                   ACC_EMPTY = ACC_FULL + NG, GROUP = ACC_EMPTY + NG;
@@ -171,7 +163,6 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
     volatile int *abort_flag = &s_abort;
-    if (threadIdx.x == 0) RTRACE(0);
 
     // this CTA's units: 128-query tiles of ONE head (u counts tiles of that head), so its descriptor block
     // never changes while it fits in shared memory
@@ -256,7 +247,6 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 const int reach = s_reach[n], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
                 const int buf = n % NG;
                 const int qn = n, st = qn % p.q_stages;
-                RTRACE(3000 + n * 4 + 3);
                 for (int rep = 0; ok && rep < n_pass; ++rep)
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
                     if (sb == 0 && rep == 0) {
@@ -269,12 +259,10 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                         ++dn;
                         res_sb = sb;
                     }
-                    RTRACE(3000 + n * 4 + 0);
                     const int uses = nacc_total[buf];
                     ok = mbar_wait(bar(ACC_EMPTY + buf), (uses & 1) ^ 1, abort_flag, p.status, RW_ACCEMPTY);
                     if (!ok) break;
                     tc_fence_after();
-                    RTRACE(3000 + n * 4 + 1);
                     const int rows_sb = max(16, min(min(p.sb_rows, p.c_pad - sb * p.sb_rows), (reach - sb * p.sb_rows + 15) & ~15));
                     const uint64_t qd = q_desc0 + (uint64_t)(st * (Q_TILE_BYTES >> 4));
                     if (FEW) {
@@ -286,8 +274,8 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                             mma_ss_lo(acc, (uint32_t)qd + (((ks >> 2) * Q_SUB_BYTES + (ks & 3) * 32) >> 4), (uint32_t)(qd >> 32),
                                       (uint32_t)d_term[ks >> 2] + (((ks & 3) * 32) >> 4), (uint32_t)(d_term[ks >> 2] >> 32), idesc, ks != 0);
                     } else
-                    for (int n0 = 0; n0 < rows_sb; n0 += 128) {
-                        const int n = min(128, rows_sb - n0);
+                    for (int n0 = 0; n0 < rows_sb; n0 += 256) {       // one instruction spans up to 256 chunks
+                        const int n = min(256, rows_sb - n0);
                         const uint32_t idesc = idesc_bf16_f32(128, n, 0, 0);
                         const uint32_t acc = tmem + buf * ACC_COLS + n0;
                         const uint32_t nofs = (uint32_t)(((resident ? sb * p.sb_rows : 0) + n0) * 128) >> 4;
@@ -301,7 +289,6 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                         }
                     }
                     tc_commit(bar(ACC_FULL + buf));
-                    RTRACE(3000 + n * 4 + 2);
                     ++nacc_total[buf];
                     // streamed blocks: the next step, if it needs another block, may overwrite this one once
                     // these MMAs are done
@@ -356,7 +343,10 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 int32_t *list = p.qlist + (size_t)pend.h * p.cap_total;
 #pragma unroll
                 for (int x = 0; x < KR; ++x)           // j holds (chunk << 8 | rank) here: a tile has 128 rows
-                    if (x < p.k && pend.j[x] >= 0) list[s_cap[pend.j[x] >> 8] + baseb[pend.j[x] >> 8] + (pend.j[x] & 255)] = pend.i * p.k + x;
+                    if (x < p.k && pend.j[x] >= 0) {
+                        const size_t at = (size_t)s_cap[pend.j[x] >> 8] + baseb[pend.j[x] >> 8] + (pend.j[x] & 255);
+                        if (index_ok(at < p.cap_total, p.status, IX_APPEND_POSITION)) list[at] = pend.i * p.k + x;
+                    }
             }
         };
         if (deferred) {
@@ -380,8 +370,6 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             const int i2 = unit_of(n + NG) * kRtRows + r;
             const bool live2 = n + NG < nu && i2 < p.L;
             if (live2) nx_ci = p.tok_chunk[i2];       // the next unit's chunk, loaded a unit ahead (its anchor word follows below)
-            [[maybe_unused]] const int tn = 100 + sg * 1000 + (n / NG) * 16;
-            if (gt == 0) RTRACE(tn + 0);
             // More than 64 picks are taken 64 at a time: every pass sees the tile's scores again (the issuer
             // recomputes them) and considers only the chunks that come after the previous pass's last pick in
             // the order of the result (score descending, then chunk index ascending).
@@ -397,7 +385,6 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ++nacc;
-                if (gt == 0) RTRACE(tn + 1);
                 tc_fence_after();
                 const int rows_sb = max(16, min(min(p.sb_rows, p.c_pad - sb * p.sb_rows), (reach - sb * p.sb_rows + 15) & ~15));
                 if (FEW) {
@@ -447,20 +434,46 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                             }
                         }
                     }
-                    if (gt == 0) RTRACE(tn + 8);
-                } else
+                } else {
+                // candidate bits of the 32 chunks from j0 on: a real chunk, not an anchor, strictly earlier if causal
+                auto cand_bits = [&](int j0) {
+                    const uint32_t aw = j0 == 0 ? aw_next : (live ? p.anc_bits[(size_t)ci * p.words + (j0 >> 5)] : 0u);
+                    uint32_t cand = ~aw;
+                    const int lim = min(p.C, p.causal ? ci : p.C) - j0;     // chunks j0 .. j0 + lim - 1 may be picked
+                    cand = lim <= 0 ? 0u : (lim >= 32 ? cand : (cand & ((1u << lim) - 1u)));
+                    return live ? cand : 0u;
+                };
+                // one candidate into the sorted list: it takes the first slot it beats (strict '>': equal scores keep
+                // their arrival order, ascending chunk index); from there on every entry moves down one slot, equal
+                // ones included, and the last falls off
+                auto insert = [&](float cv, int cj) {
+                    bool placed = false;
+#pragma unroll
+                    for (int x = 0; x < KR; ++x) {
+                        const bool up = placed || cv > top.s[x];
+                        placed = up;
+                        const float ts = top.s[x];
+                        const int tj = top.j[x];
+                        top.s[x] = up ? cv : ts;
+                        top.j[x] = up ? cj : tj;
+                        cv = up ? ts : cv;
+                        cj = up ? tj : cj;
+                    }
+                };
+                auto update_kth = [&]() {
+                    kth = top.s[0];
+#pragma unroll
+                    for (int x = 1; x < KR; ++x) kth = (x < kp) ? top.s[x] : kth;
+                };
+                // Best-first extraction: up to k members of a 32-chunk block can enter the list; they are taken one
+                // per round, the block's best first, while any row of the warp still has one above its k-th score.
+                auto extract_blocks = [&]() {
                 for (int cc = 0; cc < rows_sb; cc += 32) {
                     uint32_t v[32];
                     tmem_ld32(acc + cc, v);
                     const int j0 = sb * p.sb_rows + cc;
-                    const uint32_t aw = (sb == 0 && cc == 0) ? aw_next : (live ? p.anc_bits[(size_t)ci * p.words + (j0 >> 5)] : 0u);
-                    // candidate bits of this block: a real chunk, not an anchor, strictly earlier if causal
-                    uint32_t cand = ~aw;
-                    const int lim = min(p.C, p.causal ? ci : p.C) - j0;     // chunks j0 .. j0 + lim - 1 may be picked
-                    cand = lim <= 0 ? 0u : (lim >= 32 ? cand : (cand & ((1u << lim) - 1u)));
-                    if (!live) cand = 0u;
+                    const uint32_t cand = cand_bits(j0);
                     tmem_wait_ld();
-                    if (gt == 0) RTRACE(tn + 6);
                     {
                         float f[32];
 #pragma unroll
@@ -472,7 +485,6 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                                 f[c] = after ? f[c] : -INFINITY;
                             }
                         }
-                        // up to k members of the block can enter the list: take them best first
 #pragma unroll 1
                         for (int round = 0; round < kp; ++round) {
                             float m8[4];
@@ -483,48 +495,114 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                                 m8[q] = max3(a, b, fmaxf(f[q * 8 + 6], f[q * 8 + 7]));
                             }
                             const float m = fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3]));
-                            const float thr = kth;                                              // the list's k-th score
-                            const bool want = m > thr;
+                            const bool want = m > kth;                                          // above the list's k-th score
                             if (!__any_sync(0xffffffffu, want)) break;
                             uint32_t eq = 0u;                                                   // lowest index among equals
 #pragma unroll
                             for (int c = 0; c < 32; ++c) eq |= (f[c] == m) ? (1u << c) : 0u;
                             const int idx = __ffs(eq) - 1;
                             if (want) {
-                                float cv = m;
-                                int cj = j0 + idx;
-                                bool placed = false;
-#pragma unroll
-                                for (int x = 0; x < KR; ++x) {
-                                    // the new score takes the first slot it beats (strict '>': equal scores keep
-                                    // their arrival order, ascending chunk index); from there on every entry moves
-                                    // down one slot, equal ones included, and the last falls off
-                                    const bool up = placed || cv > top.s[x];
-                                    placed = up;
-                                    const float ts = top.s[x];
-                                    const int tj = top.j[x];
-                                    top.s[x] = up ? cv : ts;
-                                    top.j[x] = up ? cj : tj;
-                                    cv = up ? ts : cv;
-                                    cj = up ? tj : cj;
-                                }
-                                kth = top.s[0];
-#pragma unroll
-                                for (int x = 1; x < KR; ++x) kth = (x < kp) ? top.s[x] : kth;
+                                insert(m, j0 + idx);
+                                update_kth();
                             }
                             const uint32_t clr = want ? (1u << idx) : 0u;
 #pragma unroll
                             for (int c = 0; c < 32; ++c) f[c] = ((clr >> c) & 1u) ? -INFINITY : f[c];
-                            if (gt == 0) RTRACE(tn + 8 + round);
                         }
                     }
+                }
+                };
+                // Threshold selection (lists of at most 16 picks).  A lower bound `thr` of the row's final k-th score
+                // is known before any candidate is inserted: in the tile's first scoring step it is the k-th largest
+                // of G group maxima (group = chunks with equal index mod G: k groups whose maximum is at least thr
+                // hold k different candidates at least thr), later the list's own k-th score.  Only the candidates at
+                // least thr - a few more than k per row - go through the sorted insertion, which is where the work
+                // is: each row's survivors are queued in shared memory (score and column, in chunk order) and the
+                // warp inserts every row's e-th survivor together, so the insertion runs max-over-rows(survivors)
+                // times per warp instead of once per chunk.  A row with more survivors than slots (many equal scores)
+                // sends its warp through the best-first extraction instead, which needs no queue.
+                bool fast = KMAX <= 16 && p.surv_cap > 0;
+                if (fast) {
+                    constexpr int G = KMAX <= 8 ? 16 : 32;
+                    float thr = kth;
+                    if (sb == 0) {
+                        float gm[G];
+#pragma unroll
+                        for (int x = 0; x < G; ++x) gm[x] = -INFINITY;
+#pragma unroll 1
+                        for (int cc = 0; cc < rows_sb; cc += 32) {
+                            uint32_t v[32];
+                            tmem_ld32(acc + cc, v);
+                            const uint32_t cand = cand_bits(sb * p.sb_rows + cc);
+                            tmem_wait_ld();
+                            if (__all_sync(0xffffffffu, cand == 0xffffffffu)) {
+#pragma unroll
+                                for (int x = 0; x < G; ++x)
+                                    gm[x] = G == 16 ? max3(gm[x], __uint_as_float(v[x]), __uint_as_float(v[x + 16])) : fmaxf(gm[x], __uint_as_float(v[x]));
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < 32; ++c) {
+                                    const float f = ((cand >> c) & 1u) ? __uint_as_float(v[c]) : -INFINITY;
+                                    gm[c % G] = fmaxf(gm[c % G], f);
+                                }
+                            }
+                        }
+                        float t[KR];           // the KR largest group maxima, descending
+#pragma unroll
+                        for (int y = 0; y < KR; ++y) t[y] = -INFINITY;
+#pragma unroll
+                        for (int x = 0; x < G; ++x) {
+                            float cv = gm[x];
+#pragma unroll
+                            for (int y = 0; y < KR; ++y) {
+                                const float hi = fmaxf(t[y], cv);
+                                cv = fminf(t[y], cv);
+                                t[y] = hi;
+                            }
+                        }
+                        thr = t[0];
+#pragma unroll
+                        for (int y = 1; y < KR; ++y) thr = (y < kp) ? t[y] : thr;
+                    }
+                    thr = fmaxf(thr, -FLT_MAX);          // a chunk that is not a candidate (-inf) never survives
+                    float *sv = surv_base + (size_t)sg * p.surv_cap * 160 + gt;          // 128 floats + 128 bytes per slot
+                    uint8_t *sj = reinterpret_cast<uint8_t *>(surv_base + (size_t)sg * p.surv_cap * 160 + (size_t)p.surv_cap * 128) + gt;
+                    int cnt = 0;
+#pragma unroll 1
+                    for (int cc = 0; cc < rows_sb; cc += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(acc + cc, v);
+                        const uint32_t cand = cand_bits(sb * p.sb_rows + cc);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            const float f = ((cand >> c) & 1u) ? __uint_as_float(v[c]) : -INFINITY;
+                            const bool keep = f >= thr;
+                            if (keep && cnt < p.surv_cap) {
+                                sv[cnt * 128] = f;
+                                sj[cnt * 128] = (uint8_t)(cc + c);
+                            }
+                            cnt += keep ? 1 : 0;
+                        }
+                    }
+                    fast = !__any_sync(0xffffffffu, cnt > p.surv_cap);
+                    if (fast) {
+                        const int nmax = __reduce_max_sync(0xffffffffu, cnt);
+                        const int jb = sb * p.sb_rows;
+#pragma unroll 1
+                        for (int e = 0; e < nmax; ++e) {
+                            if (e < cnt) insert(sv[e * 128], jb + (int)sj[e * 128]);
+                        }
+                        update_kth();
+                    }
+                }
+                if (!fast) extract_blocks();
                 }
                 tc_fence_before();
                 mbar_arrive(bar(ACC_EMPTY + sg));
             }
             if (!ok) break;
             nx_aw = live2 ? p.anc_bits[(size_t)nx_ci * p.words] : 0u;
-            if (gt == 0) RTRACE(tn + 2);
             // sel_idx and the empty slots' partial log-sum-exp
             int32_t *out = p.sel + ((size_t)h * p.L + i) * p.k + pass * 64;
             float *pl = p.part_lse + ((size_t)h * p.L + i) * p.k + pass * 64;
@@ -552,7 +630,6 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 }
                 ok = group_sync();
                 if (!ok) break;
-                if (gt == 0) RTRACE(tn + 3);
                 if (pend.open) write_entries();
                 pend.base0 = 0; pend.base1 = 0;
                 if (gt < p.C) {
@@ -567,10 +644,8 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 for (int x = 0; x < KR; ++x) pend.j[x] = njr[x];
                 pend.h = h; pend.i = i; pend.live = live; pend.open = true;
                 ++ndef;
-                if (gt == 0) RTRACE(tn + 5);
                 continue;
             }
-            if (gt == 0) RTRACE(tn + 3);
             // tile-local rank of every pick (shared-memory histogram), then one global atomic per picked
             // chunk reserves this tile's range in that chunk's list
             for (int x = gt; x < p.C; x += 128) hist[x] = 0;
@@ -589,7 +664,6 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             }
             ok = group_sync();
             if (!ok) break;
-            if (gt == 0) RTRACE(tn + 4);
             {
                 for (int x = gt; x < p.C; x += 128) {
                     const int n = hist[x];
@@ -601,12 +675,14 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                     int32_t *list = p.qlist + (size_t)h * p.cap_total;
 #pragma unroll
                     for (int x = 0; x < KR; ++x)
-                        if (pend.j[x] >= 0) list[s_cap[pend.j[x]] + hist[pend.j[x]] + pend.rank[x]] = i * p.k + pass * 64 + x;
+                        if (pend.j[x] >= 0) {
+                            const size_t at = (size_t)s_cap[pend.j[x]] + hist[pend.j[x]] + pend.rank[x];
+                            if (index_ok(at < p.cap_total, p.status, IX_APPEND_POSITION)) list[at] = i * p.k + pass * 64 + x;
+                        }
                 }
                 ok = group_sync();
                 if (!ok) break;
             }
-            if (gt == 0) RTRACE(tn + 5);
             }   // pass
         }
         if (ok && pend.open) {                 // the last unit's entries
@@ -620,9 +696,9 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
 }
 
 // gtile[i] = attention tiles (of kQTileRows picks) before (head, chunk) pair i, with a final total;
-// flags the workspace as routed.
+// marks the workspace as holding the lists of the plan with this cookie.
 __global__ void __launch_bounds__(1024) route_tiles_kernel(const int *__restrict__ cnt, int *__restrict__ gtile,
-                                                           int *__restrict__ status, int HC) {
+                                                           int *__restrict__ status, int HC, uint32_t cookie) {
     __shared__ int st[1024];
     const int t = threadIdx.x;
     const int per = (HC + 1023) / 1024;
@@ -643,7 +719,7 @@ __global__ void __launch_bounds__(1024) route_tiles_kernel(const int *__restrict
         gtile[i] = eb;
         eb += (cnt[i] + kQTileRows - 1) / kQTileRows;
     }
-    if (t == 1023) { gtile[HC] = st[1023]; status[2] = 1; }
+    if (t == 1023) { gtile[HC] = st[1023]; status[ST_COOKIE] = (int)cookie; }
 }
 
 // The routed work items of (head, chunk) pair i: one per kQTileRows entries of its query list.
@@ -658,11 +734,87 @@ __global__ void route_items_kernel(const int *__restrict__ cnt, const int *__res
         items[at + x] = WorkItem{h, cap_off[c] + x * kQTileRows, min(kQTileRows, n - x * kQTileRows), key_tiles, c, 1, off[c], off[c + 1]};
 }
 
-#ifdef MOC_TRACE
-extern "C" int moc_trace_read_route(long long *host, int n) {
-    return (int)cudaMemcpyFromSymbol(host, g_trace_route, sizeof(long long) * (size_t)n);
+
+// Tile counts, routed work items and the cookie, from the per-(head, chunk) pick counts and lists.
+static int finish_lists(const moc_plan *p, void *ws, cudaStream_t s) {
+    int *cnt = ws_ptr<int>(ws, p->ws.cnt);
+    route_tiles_kernel<<<1, 1024, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off), ws_ptr<int>(ws, p->ws.status), p->H * p->C, p->cookie);
+    MOC_LAUNCH_CHECK();
+    if (p->k > 0) {
+        route_items_kernel<<<(unsigned)((p->H * p->C + 3) / 4), 128, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off),
+                                                                               ws_ptr<WorkItem>(ws, p->ws.rtiles), p->d_off,
+                                                                               p->d_cap_off, p->H, p->C);
+        MOC_LAUNCH_CHECK();
+    }
+    return MOC_OK;
 }
-#endif
+
+// Inverse index of a given sel_idx: 256 consecutive rows of one head per block.  Pass 1 checks every entry
+// (a chunk that may be routed to from the row, not a repeat of an earlier slot), blanks the others, marks the
+// empty slots' partial log-sum-exp and counts the block's picks per chunk in shared memory; then one global
+// atomic per picked chunk reserves the block's range in that chunk's list, and pass 2 writes the entries.
+__global__ void __launch_bounds__(256) lists_from_sel_kernel(int32_t *__restrict__ sel, float *__restrict__ part_lse,
+                                                             int *__restrict__ cnt, int32_t *__restrict__ qlist,
+                                                             const int32_t *__restrict__ tok_chunk, const uint32_t *__restrict__ anc_bits,
+                                                             const int32_t *__restrict__ cap_off, int *__restrict__ status,
+                                                             int L, int C, int k, int words, int causal, size_t cap_total) {
+    extern __shared__ int sh[];
+    int *hist = sh, *base = sh + C;
+    const int h = blockIdx.y, i = blockIdx.x * 256 + threadIdx.x;
+    for (int x = threadIdx.x; x < C; x += 256) hist[x] = 0;
+    __syncthreads();
+    int32_t *row = sel + ((size_t)h * L + i) * k;
+    if (i < L) {
+        const int ci = tok_chunk[i];
+        float *pl = part_lse + ((size_t)h * L + i) * k;
+        for (int s = 0; s < k; ++s) {
+            const int j = row[s];
+            bool ok = j >= 0 && j < C && (!causal || j < ci);
+            if (ok) ok = !((anc_bits[(size_t)ci * words + (j >> 5)] >> (j & 31)) & 1u);
+            for (int e = 0; ok && e < s; ++e) ok = row[e] != j;        // earlier slots are already checked
+            if (ok) atomicAdd(&hist[j], 1);
+            else {
+                if (j != -1) row[s] = -1;
+                pl[s] = -INFINITY;
+            }
+        }
+    }
+    __syncthreads();
+    for (int x = threadIdx.x; x < C; x += 256) {
+        const int n = hist[x];
+        base[x] = n ? atomicAdd(&cnt[h * C + x], n) : 0;
+        hist[x] = 0;
+    }
+    __syncthreads();
+    if (i < L) {
+        int32_t *list = qlist + (size_t)h * cap_total;
+        for (int s = 0; s < k; ++s) {
+            const int j = row[s];
+            if (j >= 0) {
+                const int at = cap_off[j] + base[j] + atomicAdd(&hist[j], 1);
+                if (index_ok(at < cap_off[j + 1], status, IX_APPEND_POSITION)) list[at] = i * k + s;
+            }
+        }
+    }
+}
+
+int launch_lists_from_sel(const moc_plan *p, int32_t *sel, void *ws, cudaStream_t s) {
+    int *cnt = ws_ptr<int>(ws, p->ws.cnt);
+    int *status = ws_ptr<int>(ws, p->ws.status);
+    const size_t n = std::max((size_t)p->H * p->C, (size_t)kStatusWords);
+    route_prep_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(nullptr, nullptr, cnt, status, p->H, p->C, p->c_pad, p->d, p->wait_us);
+    MOC_LAUNCH_CHECK();
+    if (p->k > 0) {
+        const size_t smem = 2 * sizeof(int) * (size_t)p->C;
+        if (smem > 200 * 1024) return MOC_ERR_SHAPE;
+        MOC_CUDA_TRY(cudaFuncSetAttribute(lists_from_sel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        lists_from_sel_kernel<<<dim3((unsigned)((p->L + 255) / 256), (unsigned)p->H), 256, smem, s>>>(
+            sel, ws_ptr<float>(ws, p->ws.part_lse), cnt, ws_ptr<int32_t>(ws, p->ws.qlist), p->d_tok_chunk, p->d_anc_bits,
+            p->d_cap_off, status, p->L, p->C, p->k, p->words, (p->flags & MOC_FLAG_CAUSAL) ? 1 : 0, (size_t)p->cap_off[p->C]);
+        MOC_LAUNCH_CHECK();
+    }
+    return finish_lists(p, ws, s);
+}
 
 template <int D>
 static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float *desc, int32_t *sel, void *ws,
@@ -672,7 +824,7 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
     __nv_bfloat16 *desc3 = ws_ptr<__nv_bfloat16>(ws, p->ws.desc3);
     {
         const size_t n = std::max((size_t)p->H * p->c_pad * D, (size_t)kStatusWords);   // covers H * C too
-        route_prep_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(desc, desc3, cnt, status, p->H, p->C, p->c_pad, D);
+        route_prep_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(desc, desc3, cnt, status, p->H, p->C, p->c_pad, D, p->wait_us);
         MOC_LAUNCH_CHECK();
     }
     if (p->k > 0) {
@@ -684,20 +836,33 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         a.causal = (p->flags & MOC_FLAG_CAUSAL) ? 1 : 0;
         a.tiles_per_head = (p->L + kRtRows - 1) / kRtRows;
         a.d_rows = p->c_pad <= kRtResident ? p->c_pad : kRtBlock;
-        a.sb_rows = std::min(a.d_rows, kRtBlock);     // steps of at most 128 chunks: an accumulator is a quarter of TMEM
+        // a scoring step fills one accumulator: a quarter of TMEM (128 chunks) with four selection groups, half of it
+        // (256 chunks) with two, which is every case but the few-chunk one; streamed blocks are 128 chunks
+        a.sb_rows = std::min(a.d_rows, p->c_pad <= 32 ? kRtBlock : 2 * kRtBlock);
         a.cap_total = (size_t)p->cap_off[p->C];
         const size_t q_tile = (size_t)kRtRows * D * 2, d_block = ((size_t)3 * a.d_rows * D * 2 + 1023) & ~(size_t)1023;
         a.ctas_per_head = std::max(1, std::min(p->n_sm / p->H, a.tiles_per_head));
         const unsigned grid = (unsigned)(p->H * a.ctas_per_head);
-        // Four selection groups (more warps to hide the selection's latencies) when an accumulator fits
-        // a quarter of TMEM and k <= 8; one when the 64-entry list takes nearly all of a thread's registers; two otherwise.
-        const int ng = (a.sb_rows <= 128 && p->k <= 8) ? 4 : p->k > 32 ? 1 : 2;
+        // Four selection groups with few chunks (more warps to hide the selection's latencies); one when the
+        // 64-entry list takes nearly all of a thread's registers; two otherwise.
+        const bool few = p->c_pad <= 32 && p->k <= 8;
+        const int ng = few ? 4 : p->k > 32 ? 1 : 2;
         a.n_pass = p->k > 64 ? (p->k + 63) / 64 : 1;
         // one histogram per group, the list offsets, and one byte per unit of a CTA
         const size_t hist = (ng * (p->k <= 8 && p->C <= 256 ? 4 : 1) + 1) * sizeof(int) * (size_t)p->C + 2 * (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
         if (d_block + q_tile + hist > budget) return MOC_ERR_SHAPE;
-        a.q_stages = (int)std::min<size_t>(4, (budget - d_block - hist) / q_tile);
-        const size_t smem = 1024 + d_block + a.q_stages * q_tile + hist;
+        // threshold selection (lists of at most 16 picks, not the few-chunk case): survivor slots per row, as many
+        // as fit beside two Q stages, at least k + 4 (else the best-first extraction alone is used)
+        a.surv_cap = 0;
+        size_t surv = 0;
+        if (!few && p->k <= 16 && budget > d_block + hist + 2 * q_tile + 16) {
+            const size_t room = budget - d_block - hist - 2 * q_tile - 16, per_slot = (size_t)ng * 160 * sizeof(float);
+            const int want = std::max(12, 2 * p->k + 4), have = (int)std::min<size_t>(room / per_slot, 255);
+            if (have >= p->k + 4) a.surv_cap = std::min(want, have);
+            surv = 16 + a.surv_cap * per_slot;
+        }
+        a.q_stages = (int)std::min<size_t>(4, (budget - d_block - hist - surv) / q_tile);
+        const size_t smem = 1024 + d_block + a.q_stages * q_tile + hist + surv;
         CUtensorMap tmQ, tmD;
         if (int r = make_tmap_2d_bf16(&tmQ, Q, (uint64_t)p->H * p->L, D, kRtRows)) return r;
         if (int r = make_tmap_2d_bf16(&tmD, desc3, (uint64_t)p->H * 3 * p->c_pad, D, (uint32_t)a.d_rows)) return r;
@@ -706,24 +871,15 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         MOC_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel<D, KM, NG, FW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
         route_tc_kernel<D, KM, NG, FW><<<grid, rt_threads(NG), smem, s>>>(tmQ, tmD, a);                                     \
     } while (0)
-        const bool few = p->c_pad <= 32 && p->k <= 8;       // then ng == 4 as well
-        if (p->k <= 4) { if (few) MOC_ROUTE_CASE(4, 4, true); else if (ng == 4) MOC_ROUTE_CASE(4, 4, false); else MOC_ROUTE_CASE(4, 2, false); }
-        else if (p->k <= 8) { if (few) MOC_ROUTE_CASE(8, 4, true); else if (ng == 4) MOC_ROUTE_CASE(8, 4, false); else MOC_ROUTE_CASE(8, 2, false); }
+        if (p->k <= 4) { if (few) MOC_ROUTE_CASE(4, 4, true); else MOC_ROUTE_CASE(4, 2, false); }
+        else if (p->k <= 8) { if (few) MOC_ROUTE_CASE(8, 4, true); else MOC_ROUTE_CASE(8, 2, false); }
         else if (p->k <= 16) MOC_ROUTE_CASE(16, 2, false);
         else if (p->k <= 32) MOC_ROUTE_CASE(32, 2, false);
         else MOC_ROUTE_CASE(64, 1, false);                 // beyond 64 picks: several passes of 64
 #undef MOC_ROUTE_CASE
         MOC_LAUNCH_CHECK();
     }
-    route_tiles_kernel<<<1, 1024, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off), status, p->H * p->C);
-    MOC_LAUNCH_CHECK();
-    if (p->k > 0) {
-        route_items_kernel<<<(unsigned)((p->H * p->C + 3) / 4), 128, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off),
-                                                                               ws_ptr<WorkItem>(ws, p->ws.rtiles), p->d_off,
-                                                                               p->d_cap_off, p->H, p->C);
-        MOC_LAUNCH_CHECK();
-    }
-    return MOC_OK;
+    return finish_lists(p, ws, s);
 }
 
 int launch_route(const moc_plan *p, const __nv_bfloat16 *Q, const float *desc, int32_t *sel, void *ws, cudaStream_t s) {

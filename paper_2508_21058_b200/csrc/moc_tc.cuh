@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "moc_common.cuh"
+
 namespace moc {
 namespace tc {
 
@@ -41,7 +43,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-constexpr uint64_t kWaitLimitNs = 1000000000ull;   // every wait gives up after about one second
+constexpr uint64_t kWaitLimitNs = 1000000000ull;   // every wait gives up after about one second ...
+// ... unless the workspace's status area states another limit (microseconds; tests shorten it).  Read only
+// on the slow path of a wait, every few hundred polls.
+__device__ __forceinline__ uint64_t wait_limit_ns(const int *status) {
+    const unsigned us = (unsigned)__ldcg(status + ST_WAIT_US);
+    return (us && us < 1000000u) ? (uint64_t)us * 1000ull : kWaitLimitNs;     // never longer than the default
+}
 
 // Bounded wait.  Returns false when the CTA is aborting (this or another wait ran out);
 // the first wait to run out records `code` in the status words.
@@ -52,7 +60,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 0xff) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (global_timer_ns() - t0 > wait_limit_ns(status)) {
                 *abort_flag = 1;
                 if (atomicCAS(status, 0, MOC_ERR_TIMEOUT) == 0) status[1] = code;
                 return false;
@@ -81,7 +89,7 @@ __device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, vo
         if (mbar_test_wait(bar, parity)) return true;
         if ((it & 0xfff) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (global_timer_ns() - t0 > wait_limit_ns(status)) {
                 *abort_flag = 1;
                 if (atomicCAS(status, 0, MOC_ERR_TIMEOUT) == 0) status[1] = code;
                 return false;

@@ -306,17 +306,20 @@ def as_u16(t: torch.Tensor) -> np.ndarray:
 
 
 def sample_rows(wl: Workload, per_head: int, seed: int = 0) -> np.ndarray:
-    """int32 [n, 2] (head, token) pairs: first and last token of every chunk (frame,
-    caption and shot edges, which include rows with fewer than k candidates) for
-    every head, topped up with seeded uniform picks to ``per_head`` rows."""
+    """int32 [n, 2] (head, token) pairs, about ``per_head`` per head: at most half of them
+    are first and last tokens of chunks (frame, caption and shot edges, which include rows
+    with fewer than k candidates; a seeded subset when there are more edges than that), the
+    rest are seeded uniform picks over the whole stream, so rows in the interior of every
+    kind of chunk are always present whatever the number of edges."""
     lay = wl.layout
     edges = np.unique(np.concatenate([lay.chunk_off[:-1], lay.chunk_off[1:] - 1]))
     rng = np.random.RandomState(7919 + seed)
     out = []
     for h in range(wl.n_heads):
         toks = edges
-        if len(toks) > per_head:
-            toks = np.sort(rng.choice(toks, per_head, replace=False))
+        n_edge = max(1, per_head // 2)
+        if len(toks) > n_edge:
+            toks = np.sort(rng.choice(toks, n_edge, replace=False))
         extra = per_head - len(toks)
         if extra > 0:
             toks = np.unique(np.concatenate([toks, rng.randint(0, lay.n_tokens, extra)]))

@@ -20,16 +20,16 @@ def _forward_parity(name, scalar, rows_per_head=None):
     run = PU.GpuRun(wl, scalar_attend=scalar).forward()
     x = run.host_inputs()
     orc = Oracle.from_workload(wl)
+    rec = None if scalar else name
     # step 1: descriptors
     desc64 = orc.chunk_pool(x["k"])
     desc_gpu = run.desc.cpu().numpy()
     assert np.max(np.abs(desc_gpu - desc64)) <= PU.DESC_ATOL
+    if rec:
+        PU.report(rec, "descriptors", {"max_abs": float(np.max(np.abs(desc_gpu - desc64)))})
     # steps 2-5: indices (oracle routed from its own fp64 descriptors)
     sel_gpu = run.sel.cpu().numpy()
-    n, near, hard, ex, order_bad = PU.compare_routing(wl, orc, x["q"], desc64, sel_gpu)
-    assert hard == 0, ex
-    assert near <= max(2, int(2e-3 * n)), (near, n)
-    assert order_bad <= near + max(2, int(2e-3 * n))
+    n, near = PU.assert_routing(wl, orc, x["q"], desc64, sel_gpu, rec)
     # step 6: attention over the GPU's own selection (equal to the oracle's up to the near ties above)
     rows = None if rows_per_head is None else W.sample_rows(wl, rows_per_head)
     O_ref, lse_ref = orc.attend(x["q"], x["k"], x["v"], sel_gpu, rows)
@@ -39,7 +39,7 @@ def _forward_parity(name, scalar, rows_per_head=None):
     else:
         O_g, l_g = O_gpu[rows[:, 0], rows[:, 1]], lse_gpu[rows[:, 0], rows[:, 1]]
     err = PU.attention_errors(O_g, l_g, O_ref, lse_ref)
-    PU.assert_attention_close(err)
+    PU.assert_attention_close(err, rec)
     return run, err, near, n
 
 
@@ -53,7 +53,7 @@ def test_forward_small(name):
     _forward_parity(name, scalar=False, rows_per_head=None if name != "midi2" else 400)
 
 
-def _backward_parity(name, scalar, n_rows=64, heads=None):
+def _backward_parity(name, scalar, n_rows=64, heads=None, record=None):
     wl = W.workload(name)
     if heads is not None:
         wl.n_heads = heads
@@ -65,15 +65,13 @@ def _backward_parity(name, scalar, n_rows=64, heads=None):
     rows = W.sample_rows(wl, n_rows)
     dQ_g = run.dQ.float().cpu().numpy()
     dK_g, dV_g = run.dK.float().cpu().numpy(), run.dV.float().cpu().numpy()
-    for key_head, chunk in ((0, 0), (wl.n_heads - 1, lay.n_chunks // 2), (0, lay.n_chunks - 2)):
+    for n, (key_head, chunk) in enumerate(((0, 0), (wl.n_heads - 1, lay.n_chunks // 2), (0, lay.n_chunks - 2))):
         t0, t1 = int(lay.chunk_off[chunk]), int(lay.chunk_off[chunk + 1])
         dQ, dK, dV = orc.attend_bwd(x["q"], x["k"], x["v"], x["do"], sel_gpu, rows, key_head, (t0, t1))
-        assert np.max(np.abs(dQ_g[rows[:, 0], rows[:, 1]] - dQ)) <= PU.GRAD_MAX_ABS
-        assert np.max(np.abs(dK_g[key_head, t0:t1] - dK)) <= PU.GRAD_MAX_ABS
-        assert np.max(np.abs(dV_g[key_head, t0:t1] - dV)) <= PU.GRAD_MAX_ABS
-        # not vacuous: relative L2 as well
-        for g, r in ((dQ_g[rows[:, 0], rows[:, 1]], dQ), (dK_g[key_head, t0:t1], dK), (dV_g[key_head, t0:t1], dV)):
-            assert np.sqrt(np.sum((g - r) ** 2) / np.sum(r ** 2)) < 2e-2
+        rec = record if n == 0 else None
+        PU.assert_grad_close(dQ_g[rows[:, 0], rows[:, 1]], dQ, rec, "dQ")
+        PU.assert_grad_close(dK_g[key_head, t0:t1], dK, rec, "dK_first_chunk")
+        PU.assert_grad_close(dV_g[key_head, t0:t1], dV, rec, "dV_first_chunk")
 
 
 @pytest.mark.parametrize("name", ["cfg0", "mini2", "mini4", "mini3"])
@@ -89,30 +87,42 @@ def test_backward_small(name):
 def test_backward_benchmark_length_sampled():
     """The single-shot clip at its full length (two heads: heads are independent): dQ on sampled rows, dK / dV
     of the caption chunk (selected by every query), of a middle frame and of the last-but-one frame."""
-    _backward_parity("cfg1", scalar=False, n_rows=96, heads=2)
+    _backward_parity("cfg1", scalar=False, n_rows=96, heads=2, record="cfg1")
 
 
-def test_backward_training_length_sampled():
-    """The minute-scale training layout at its full length, one head: dQ on sampled rows and dK / dV of one
-    frame in the middle of the stream (its queries are its shot window and the rows that routed to it; a caption
-    chunk is attended by all 528k queries, which the oracle cannot afford here - the single-shot test covers it)."""
-    wl = W.workload("cfg4")
+def _backward_full_length(name, chunk, n_rows, record, what):
+    """One head of a multi-shot layout at its full length: dQ on sampled rows (edges and interior), dK / dV of
+    one key chunk (the oracle recomputes the forward of every query that attends to it)."""
+    wl = W.workload(name)
     wl.n_heads = 1
     run = PU.GpuRun(wl, tensors=("q", "k", "v", "do")).forward().backward()
     x = run.host_inputs()
     orc = Oracle.from_workload(wl)
     sel_gpu = run.sel.cpu().numpy()
     lay = wl.layout
-    rows = W.sample_rows(wl, 64)
-    chunk = lay.n_chunks // 2 + 3
-    assert int(lay.chunk_mod[chunk]) == 0           # a video frame
+    rows = W.sample_rows(wl, n_rows)
     t0, t1 = int(lay.chunk_off[chunk]), int(lay.chunk_off[chunk + 1])
     dQ, dK, dV = orc.attend_bwd(x["q"], x["k"], x["v"], x["do"], sel_gpu, rows, 0, (t0, t1))
-    dQ_g = run.dQ.float().cpu().numpy()[rows[:, 0], rows[:, 1]]
-    dK_g, dV_g = run.dK.float().cpu().numpy()[0, t0:t1], run.dV.float().cpu().numpy()[0, t0:t1]
-    for g, r in ((dQ_g, dQ), (dK_g, dK), (dV_g, dV)):
-        assert np.max(np.abs(g - r)) <= PU.GRAD_MAX_ABS
-        assert np.sqrt(np.sum((g - r) ** 2) / np.sum(r ** 2)) < 2e-2
+    PU.assert_grad_close(run.dQ.float().cpu().numpy()[rows[:, 0], rows[:, 1]], dQ, record, "dQ")
+    PU.assert_grad_close(run.dK.float().cpu().numpy()[0, t0:t1], dK, record, "dK_" + what)
+    PU.assert_grad_close(run.dV.float().cpu().numpy()[0, t0:t1], dV, record, "dV_" + what)
+
+
+def test_backward_training_length_sampled():
+    """The minute-scale training layout at its full length, one head: dQ on sampled rows and dK / dV of one
+    frame in the middle of the stream (its queries are its shot window and the rows that routed to it)."""
+    wl = W.workload("cfg4")
+    chunk = wl.layout.n_chunks // 2 + 3
+    assert int(wl.layout.chunk_mod[chunk]) == 0           # a video frame
+    _backward_full_length("cfg4", chunk, 512, "cfg4", "mid_frame")
+
+
+def test_backward_caption_chunk_at_multi_shot_length():
+    """dK / dV of a caption chunk of the 8-shot stream at its full length (one head): every one of the 264k
+    queries attends to it, so its key tiles see the longest query stream the backward has."""
+    wl = W.workload("cfg2")
+    chunk = int(np.nonzero(wl.layout.chunk_mod == 1)[0][3])          # the caption of the fourth shot
+    _backward_full_length("cfg2", chunk, 512, "cfg2", "caption")
 
 
 def test_route_is_deterministic_and_lists_invert_selection():
@@ -186,10 +196,7 @@ def test_equal_descriptors_keep_index_order(name):
     x = run.host_inputs()
     orc = Oracle.from_workload(wl)
     desc64 = orc.chunk_pool(x["k"])
-    n, near, hard, ex, order_bad = PU.compare_routing(wl, orc, x["q"], desc64, run.sel.cpu().numpy())
-    assert hard == 0, ex
-    assert near <= max(2, int(2e-3 * n)), (near, n)
-    assert order_bad <= near + max(2, int(2e-3 * n)), order_bad
+    PU.assert_routing(wl, orc, x["q"], desc64, run.sel.cpu().numpy())
 
 
 def test_argument_errors_launch_nothing():
@@ -220,27 +227,35 @@ def test_argument_errors_launch_nothing():
     assert launch_count() == n0
 
 
-@pytest.mark.parametrize("name,rows_per_head,heads", [("cfg1", 96, None), ("cfg2", 192, 3), ("cfg4", 192, 2), ("cfg3-m512-p8", 128, 1), ("cfg3-m256-p15", 96, 1)])
+SWEEP = [f"cfg3-m{m}-p{p}" for m in (1560, 1024, 512, 256) for p in (8, 15, 25)]
+
+
+@pytest.mark.parametrize("name,rows_per_head,heads",
+                         [("cfg1", 2048, None), ("cfg2", 2048, None), ("cfg4", 2048, 6)] + [(n, 2048, 1) for n in SWEEP])
 def test_forward_benchmark_size_sampled(name, rows_per_head, heads):
-    """The benchmark workload in the launch configuration bench.py times; attention
-    checked on sampled rows (frame, caption and shot edges plus uniform picks), indices on
-    every row of a sample of heads."""
+    """The benchmark workloads at their full length, in the launch configuration bench.py times (cfg1 and the
+    multi-shot stream with all 24 heads, the training layout on 6 heads, every chunk-size / sparsity point of
+    the sweep on one head: heads are independent).  Indices are compared on EVERY row; attention on 2048 rows
+    per head, half of them chunk edges and half uniform picks over the stream."""
     wl = W.workload(name)
-    if heads is not None:       # the multi-shot stream at its full length, on a few heads (each head is independent)
+    if heads is not None:
         wl.n_heads = heads
     run = PU.GpuRun(wl).forward()
     x = run.host_inputs()
     orc = Oracle.from_workload(wl)
     desc64 = orc.chunk_pool(x["k"])
-    assert np.max(np.abs(run.desc.cpu().numpy() - desc64)) <= PU.DESC_ATOL
+    derr = float(np.max(np.abs(run.desc.cpu().numpy() - desc64)))
+    PU.report(name, "descriptors", {"max_abs": derr})
+    assert derr <= PU.DESC_ATOL
     sel_gpu = run.sel.cpu().numpy()
-    n, near, hard, ex, _ = PU.compare_routing(wl, orc, x["q"], desc64, sel_gpu)
-    assert hard == 0, ex
-    assert near <= int(2e-3 * n), (near, n)
+    PU.assert_routing(wl, orc, x["q"], desc64, sel_gpu, name)
     rows = W.sample_rows(wl, rows_per_head)
     O_ref, lse_ref = orc.attend(x["q"], x["k"], x["v"], sel_gpu, rows)
     hh, ii = (torch.from_numpy(rows[:, a].astype(np.int64)).cuda() for a in (0, 1))
     O_g = run.O[hh, ii].float().cpu().numpy()
     l_g = run.lse[hh, ii].cpu().numpy()
-    PU.assert_attention_close(PU.attention_errors(O_g, l_g, O_ref, lse_ref))
-    assert run.plan.moc_selected_pairs(run.ws) > 0
+    PU.assert_attention_close(PU.attention_errors(O_g, l_g, O_ref, lse_ref), name)
+    pairs = run.plan.moc_selected_pairs(run.ws)
+    PU.report(name, "workload", {"heads": wl.n_heads, "tokens": wl.n_tokens, "chunks": wl.n_chunks, "top_k": wl.top_k,
+                                 "selected_pairs": int(pairs), "workspace_bytes": run.plan.workspace_bytes(False)})
+    assert pairs > 0

@@ -184,6 +184,41 @@ def test_topk_equals_best_k_subset_and_library_topk(name):
         assert np.all(sel[h, i, min(wl.top_k, len(cands)):] == -1)
 
 
+def test_score_table_equals_library_contraction_on_listed_rows():
+    """The oracle's score table (Eq. 3, the raw dot product of a query with every chunk descriptor) is what
+    decides whether a difference between two selections is a near tie, so it gets its own pin: an fp64
+    library contraction of the widened queries with descriptors that are NOT the oracle's (random, so a
+    wrong descriptor stride shows), on (head, token) rows listed out of order and from distinct heads (so a
+    swapped index, a row taken from the wrong head or an output written in sorted order shows), with an
+    unmasked table (anchors and future chunks included)."""
+    wl = W.workload("mini2")
+    wl.n_heads = 3
+    x = make(wl)
+    orc = Oracle.from_workload(wl)
+    rng = np.random.RandomState(11)
+    desc = rng.standard_normal((wl.n_heads, wl.n_chunks, wl.head_dim))
+    L = wl.n_tokens
+    rows = np.array([[2, L - 1], [0, 5], [1, 700], [2, 0], [0, L - 2], [1, 5], [1, 4], [0, 700], [2, 333]], np.int32)
+    got = orc.scores(x["q"], desc, rows)
+    assert got.shape == (len(rows), wl.n_chunks)
+    Qf = bits_f64(x["q"])
+    ref = np.einsum("nd,ncd->nc", Qf[rows[:, 0], rows[:, 1]], desc[rows[:, 0]])
+    assert np.max(np.abs(got - ref)) < 1e-12
+    # the rows really differ between heads and tokens, so the comparison above can tell them apart
+    assert np.min(np.abs(ref[1] - ref[5])) > 1e-6 and np.min(np.abs(ref[5] - ref[6])) > 1e-6
+    # and the scores the selection reports for its picks are entries of this table
+    desc_o = orc.chunk_pool(x["k"])
+    sel, sel_score, nxt = orc.route(x["q"], desc_o, with_scores=True)
+    tab = orc.scores(x["q"], desc_o, rows)
+    for r, (h, i) in enumerate(rows):
+        for s in range(wl.top_k):
+            if sel[h, i, s] >= 0:
+                assert sel_score[h, i, s] == tab[r, sel[h, i, s]]
+        picked = sel_score[h, i][sel[h, i] >= 0]
+        if len(picked) == wl.top_k and np.isfinite(nxt[h, i]):
+            assert nxt[h, i] <= picked.min()          # the best chunk left out never beats a pick
+
+
 def test_noncausal_variant_routes_to_future_chunks_too():
     wl = W.workload("mini5")
     wl.n_heads = 1
