@@ -50,6 +50,15 @@ def _p(a):
     return C.c_void_p(a.ctypes.data) if a is not None else C.c_void_p(0)
 
 
+def philox4x32(ctr, key):
+    """Philox4x32-10 of one counter block (4 x uint32) under a key (2 x uint32)."""
+    c = np.ascontiguousarray(ctr, np.uint32)
+    k = np.ascontiguousarray(key, np.uint32)
+    out = np.zeros(4, np.uint32)
+    _load().moc_oracle_philox4x32(_p(c), _p(k), _p(out))
+    return out
+
+
 def num_threads() -> int:
     return int(_load().moc_oracle_num_threads())
 
@@ -134,6 +143,16 @@ class Oracle:
         self.lib.moc_oracle_attend_rows(C.byref(self.cfg), _p(Q), _p(K), _p(V), _p(sel_idx), C.c_double(scale),
                                         C.c_int(len(rows)), _p(rows), _p(O), _p(lse))
         return O, lse
+
+    def context_drop(self, sel_idx, p_max, lam, seed):
+        """Context drop-off / drop-in (Sec. 3.1) applied to a copy of sel_idx.  Returns
+        (edited sel_idx, n_dropped, n_drawn, n_added), the last three [H, L] int32."""
+        out = np.ascontiguousarray(sel_idx, np.int32).copy()
+        assert out.shape == (self.H, self.L, self.k)
+        nd, nm, na = (np.zeros((self.H, self.L), np.int32) for _ in range(3))
+        self.lib.moc_oracle_context_drop(C.byref(self.cfg), _p(out), C.c_float(p_max), C.c_float(lam),
+                                         C.c_uint64(int(seed)), _p(nd), _p(nm), _p(na))
+        return out, nd, nm, na
 
     def attend_bwd(self, Q, K, V, dO, sel_idx, rows=None, key_head=0, key_range=None, scale=0.0):
         """dQ [n, d] of the listed rows and (dK, dV) [t1-t0, d] of tokens ``key_range`` of

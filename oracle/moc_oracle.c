@@ -15,7 +15,10 @@
  * case Q = 0 (first candidates win, LSE = log |selected tokens|); fp64 library
  * softmax attention with an explicit mask and its autograd for forward and
  * backward; finite differences; the paper's printed sparsity column for the pair
- * count.  No function here is unpinned.
+ * count; the published known-answer vectors for the counter-based generator and closed-form
+ * expectations, set relations and the identity case for the drop-off / drop-in regulariser;
+ * einsum and an independent numpy restatement for the shot-level (outer-loop) routing.
+ * No function here is unpinned.
  */
 #include <math.h>
 #include <stdint.h>
@@ -307,6 +310,122 @@ void moc_oracle_attend_bwd(const moc_oracle_cfg *p, const uint16_t *Q, const uin
         }
         free(mask); free(z); free(prob); free(o); free(aK); free(aV);
     }
+}
+
+
+/* ---- Counter-based random numbers: Philox4x32-10 as defined by Salmon, Moraes, Dror and Shaw,
+ * "Parallel random numbers: as easy as 1, 2, 3" (SC'11): ten rounds of
+ *   (c0, c1, c2, c3) <- (hi(M1 c2) ^ c1 ^ k0,  lo(M1 c2),  hi(M0 c0) ^ c3 ^ k1,  lo(M0 c0))
+ * with M0 = 0xD2511F53, M1 = 0xCD9E8D57, the key bumped by (0x9E3779B9, 0xBB67AE85) between rounds.
+ * The regulariser below draws from it; the CUDA library has its own implementation of the same
+ * definition.  Pinned by the known-answer vectors published with the generator. ---- */
+void moc_oracle_philox4x32(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1, n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* d-th uniform draw of row (h, i): word d % 4 of the block with counter (i, h, d / 4, 0) and key = seed;
+ * its top 24 bits scaled to [0, 1), which is exact in single precision. */
+static float row_uniform(uint64_t seed, int h, int i, int d) {
+    uint32_t ctr[4] = {(uint32_t)i, (uint32_t)h, (uint32_t)(d / 4), 0u}, key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)}, out[4];
+    moc_oracle_philox4x32(ctr, key, out);
+    return (float)(out[d % 4] >> 8) * (1.0f / 16777216.0f);
+}
+
+/* ---- Sec. 3.1 "Context drop-off" and "Context drop-in": training-time edits of a routed selection.
+ * For every query (h, i), on its k slots (the paper's top-k; -1 = empty slot):
+ *   drop-off: p_drop = U * p_max with U ~ Uniform[0, 1); floor(p_drop * k) of the row's picks (never more
+ *             than it has) are removed, each chosen uniformly among the picks still there;
+ *   drop-in:  m ~ Poisson(lambda) chunks are added, each chosen uniformly among the chunks that may be
+ *             routed to from the row (not an anchor, strictly earlier if causal) and that are neither in the
+ *             routed selection nor added already; they go into the free slots (empty or just dropped),
+ *             lowest slot first, for as long as there is a free slot and a chunk left to add.
+ * Where a draw decides an integer the arithmetic is single precision, as in the CUDA kernel:
+ *   draw 0: U;  draw 1: the Poisson variate by inversion (smallest m with u < cdf[m], cdf accumulated in
+ *   double from exp(-lambda) by term_j = term_{j-1} lambda / j and rounded to single; at most 31);
+ *   draw 2 + r: the r-th removal takes the floor(u * n_left)-th pick still there, in slot order;
+ *   draw 2 + k + t: the t-th addition takes the floor(u * n_left)-th eligible chunk, in chunk order.
+ * n_dropped / n_drawn / n_added ([H][L], optional) report what happened per row. ---- */
+void moc_oracle_context_drop(const moc_oracle_cfg *p, int32_t *sel_idx, float p_max, float lambda, uint64_t seed,
+                             int32_t *n_dropped, int32_t *n_drawn, int32_t *n_added) {
+    float cdf[32];
+    {
+        double term = exp(-(double)lambda), acc = term;
+        cdf[0] = (float)acc;
+        for (int j = 1; j < 32; ++j) {
+            term = term * (double)lambda / (double)j;
+            acc += term;
+            cdf[j] = (float)acc;
+        }
+    }
+    int k = p->k;
+#pragma omp parallel for collapse(2) schedule(dynamic, 64)
+    for (int h = 0; h < p->H; ++h)
+        for (int i = 0; i < p->L; ++i) {
+            int32_t *row = sel_idx + ((size_t)h * p->L + i) * k;
+            int c = chunk_of(p, i);
+            int32_t *orig = (int32_t *)malloc(sizeof(int32_t) * (size_t)(k > 0 ? k : 1));
+            char *gone = (char *)calloc((size_t)(k > 0 ? k : 1), 1);       /* 1: this slot's pick was dropped */
+            memcpy(orig, row, sizeof(int32_t) * (size_t)k);
+            int n_sel = 0;
+            for (int s = 0; s < k; ++s) n_sel += orig[s] >= 0;
+            /* drop-off */
+            float p_drop = row_uniform(seed, h, i, 0) * p_max;
+            int n_drop = (int)(p_drop * (float)k);
+            if (n_drop > n_sel) n_drop = n_sel;
+            for (int r = 0; r < n_drop; ++r) {
+                int n_left = n_sel - r;
+                int pos = (int)(row_uniform(seed, h, i, 2 + r) * (float)n_left);
+                if (pos > n_left - 1) pos = n_left - 1;
+                for (int s = 0; s < k; ++s) {
+                    if (orig[s] < 0 || gone[s]) continue;
+                    if (pos-- == 0) { gone[s] = 1; row[s] = -1; break; }
+                }
+            }
+            /* drop-in */
+            float u = row_uniform(seed, h, i, 1);
+            int m = 0;
+            while (m < 31 && !(u < cdf[m])) ++m;
+            int added = 0;
+            for (int t = 0; t < m; ++t) {
+                int slot = -1;
+                for (int s = 0; s < k && slot < 0; ++s)
+                    if (row[s] < 0) slot = s;
+                if (slot < 0) break;
+                /* eligible: a candidate of the row that is neither a routed pick (kept or dropped) nor added already */
+                int n_left = 0;
+                for (int j = 0; j < p->C; ++j) {
+                    if (!is_candidate(p, c, j)) continue;
+                    int used = 0;
+                    for (int s = 0; s < k && !used; ++s) used = (orig[s] == j) || (row[s] == j);
+                    n_left += !used;
+                }
+                if (n_left == 0) break;
+                int pos = (int)(row_uniform(seed, h, i, 2 + k + t) * (float)n_left);
+                if (pos > n_left - 1) pos = n_left - 1;
+                for (int j = 0; j < p->C; ++j) {
+                    if (!is_candidate(p, c, j)) continue;
+                    int used = 0;
+                    for (int s = 0; s < k && !used; ++s) used = (orig[s] == j) || (row[s] == j);
+                    if (used) continue;
+                    if (pos-- == 0) { row[slot] = j; break; }
+                }
+                ++added;
+            }
+            size_t r_ = (size_t)h * p->L + i;
+            if (n_dropped) n_dropped[r_] = n_drop;
+            if (n_drawn) n_drawn[r_] = m;
+            if (n_added) n_added[r_] = added;
+            free(orig);
+            free(gone);
+        }
 }
 
 int moc_oracle_num_threads(void) {

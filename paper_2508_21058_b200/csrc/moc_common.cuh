@@ -66,7 +66,12 @@ struct moc_plan {
     std::vector<int32_t> pool_unit_off;      // [C+1] prefix of pool units per chunk
     int words;                               // uint32 words per anchor bitmap row
     std::vector<int32_t> cap_off;            // [C+1] start of chunk c's query list inside a head's list area
-    int c_pad;                               // C rounded up to a multiple of 16 (MMA N granularity)
+    // Routing scores only the chunks that can ever be picked: text chunks are anchors of every query, so the score
+    // matrix has one column per non-text chunk ("column" = index among those, in chunk order).
+    int ncol;                                // number of columns
+    int cwords;                              // uint32 words per candidate bitmap row (over columns)
+    int prefix_mode;                         // 1: every query chunk's candidates are exactly the columns [0, lim[c])
+    int c_pad;                               // columns rounded up to a multiple of 16 (MMA N granularity)
     int n_pool_units;
     int heads_per_group;                     // Hg: heads whose routed partials are held at once (attention runs group by group)
     size_t partials_budget;                  // bytes the routed partials may take; sets Hg
@@ -77,6 +82,8 @@ struct moc_plan {
     int32_t *d_off, *d_shot, *d_tok_chunk, *d_anc_off, *d_ranc_off, *d_ranc, *d_pool_unit_off, *d_pool_unit_chunk, *d_cap_off;
     uint8_t *d_mod;
     uint32_t *d_anc_bits;
+    uint32_t *d_cand_c;                      // [C][cwords] candidate columns of a query in chunk c (causality included)
+    int32_t *d_lim, *d_reach, *d_col_chunk;  // [C] prefix length (-1: not a prefix); [C] columns any query up to chunk c can reach; [ncol] chunk of a column
     moc::KeyRange *d_anc_rng;
     moc::WorkItem *d_qitems;
     moc::KeyRange *d_chunk_rng;              // [C] token range of every chunk

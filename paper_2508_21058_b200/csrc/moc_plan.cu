@@ -170,7 +170,31 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
         if (next >= 2147483647LL) { delete p; return MOC_ERR_SHAPE; }
         p->cap_off[c + 1] = (int32_t)next;
     }
-    p->c_pad = (C + 15) / 16 * 16;
+    // score columns: the chunks that are not text; per query chunk its candidate columns (not an anchor, strictly
+    // earlier if causal), whether they form a prefix of the columns (they do under the causal rule: everything
+    // before the own shot's window), and how far any query up to that chunk can reach
+    std::vector<int32_t> col_chunk, col_of(C, -1);
+    for (int j = 0; j < C; ++j)
+        if (p->mod[j] != 1) { col_of[j] = (int32_t)col_chunk.size(); col_chunk.push_back(j); }
+    p->ncol = (int)col_chunk.size();
+    p->cwords = std::max(1, (p->ncol + 31) / 32);
+    p->c_pad = std::max(16, (p->ncol + 15) / 16 * 16);
+    std::vector<uint32_t> cand_c((size_t)C * p->cwords, 0u);
+    std::vector<int32_t> lim(C, 0), reach(C, 0);
+    p->prefix_mode = 1;
+    for (int c = 0; c < C; ++c) {
+        int n_cand = 0, top = 0;
+        for (int j = 0; j < C; ++j) {
+            if (is_anchor(p, c, j) || ((p->flags & MOC_FLAG_CAUSAL) && j >= c)) continue;
+            const int col = col_of[j];          // a non-anchor is never text
+            cand_c[(size_t)c * p->cwords + col / 32] |= 1u << (col % 32);
+            ++n_cand;
+            top = col + 1;
+        }
+        lim[c] = top == n_cand ? n_cand : -1;
+        if (lim[c] < 0) p->prefix_mode = 0;
+        reach[c] = std::max(top, c ? reach[c - 1] : 0);
+    }
     p->partials_budget = (size_t)6 << 30;
     p->wait_us = 0;
     p->cookie = plan_cookie(p);
@@ -185,6 +209,7 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
     size_t o_bits = take(4 * bits.size()), o_aoff = take(4 * (C + 1)), o_arng = take(sizeof(KeyRange) * p->anc_rng.size());
     size_t o_roff = take(4 * (C + 1)), o_ranc = take(4 * p->ranc.size()), o_qt = take(sizeof(WorkItem) * p->qitems.size());
     size_t o_puo = take(4 * (C + 1)), o_puc = take(4 * unit_chunk.size()), o_cap = take(4 * (C + 1)), o_crng = take(sizeof(KeyRange) * C), o_kt = take(sizeof(KTile) * p->ktiles.size());
+    size_t o_candc = take(4 * cand_c.size()), o_lim = take(4 * C), o_reach = take(4 * C), o_colc = take(4 * std::max<size_t>(col_chunk.size(), 1));
     cudaError_t e = cudaMalloc(&p->d_blob, o);
     if (e != cudaSuccess) { set_cuda_error(e, "cudaMalloc(plan tables)"); delete p; return MOC_ERR_CUDA; }
     char *b = static_cast<char *>(p->d_blob);
@@ -198,7 +223,9 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
                         up(o_qt, p->qitems.data(), sizeof(WorkItem) * p->qitems.size()),
                         up(o_puo, p->pool_unit_off.data(), 4 * (C + 1)), up(o_puc, unit_chunk.data(), 4 * unit_chunk.size()),
                         up(o_cap, p->cap_off.data(), 4 * (C + 1)), up(o_crng, chunk_rng.data(), sizeof(KeyRange) * C),
-                        up(o_kt, p->ktiles.data(), sizeof(KTile) * p->ktiles.size())};
+                        up(o_kt, p->ktiles.data(), sizeof(KTile) * p->ktiles.size()),
+                        up(o_candc, cand_c.data(), 4 * cand_c.size()), up(o_lim, lim.data(), 4 * C), up(o_reach, reach.data(), 4 * C),
+                        up(o_colc, col_chunk.data(), 4 * col_chunk.size())};
     for (cudaError_t x : es)
         if (x != cudaSuccess) { set_cuda_error(x, "cudaMemcpy(plan tables)"); cudaFree(p->d_blob); delete p; return MOC_ERR_CUDA; }
     p->d_off = (int32_t *)(b + o_off); p->d_shot = (int32_t *)(b + o_shot); p->d_mod = (uint8_t *)(b + o_mod);
@@ -209,6 +236,8 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
     p->d_cap_off = (int32_t *)(b + o_cap);
     p->d_chunk_rng = (KeyRange *)(b + o_crng);
     p->d_ktiles = (KTile *)(b + o_kt);
+    p->d_cand_c = (uint32_t *)(b + o_candc); p->d_lim = (int32_t *)(b + o_lim); p->d_reach = (int32_t *)(b + o_reach);
+    p->d_col_chunk = (int32_t *)(b + o_colc);
     *out = p;
     return MOC_OK;
 }

@@ -43,6 +43,7 @@ constexpr int kRtRows = 128;          // queries per tile
 __host__ __device__ constexpr int rt_threads(int ng) { return 64 + 128 * ng + 64; }   // producer, issuer | NG selection groups | second issuer, idle
 constexpr int kRtResident = 192;      // up to this many (padded) chunks the whole block stays resident
 constexpr int kRtBlock = 128;         // otherwise chunks are streamed in blocks of this many
+constexpr int kRtDeferredChunks = 512; // up to this many chunks (and 8 picks) a unit's list append is finished behind the next unit's selection
 
 enum RouteWait { RW_QFULL = 32, RW_QEMPTY, RW_DFULL, RW_DEMPTY, RW_ACCFULL, RW_ACCEMPTY, RW_GROUP };
 
@@ -56,11 +57,12 @@ struct TopK {
     }
 };
 
-// desc3[h][t][c][:] for t = 0, 1, 2: bf16 terms of desc[h][c][:] (rows c >= C are zero);
-// also clears the pick counters and the status words (the workspace holds no plan's lists until they
+// desc3[h][t][col][:] for t = 0, 1, 2: bf16 terms of the descriptor of score column col (the col-th non-text
+// chunk; rows beyond the last column are zero); also clears the pick counters and the status words (the workspace holds no plan's lists until they
 // are complete) and states the limit of the bounded waits.  With desc == nullptr only the clearing is done.
 __global__ void route_prep_kernel(const float *__restrict__ desc, __nv_bfloat16 *__restrict__ desc3, int *__restrict__ cnt,
-                                  int *__restrict__ status, int H, int C, int c_pad, int d, unsigned wait_us) {
+                                  int *__restrict__ status, const int32_t *__restrict__ col_chunk, int H, int C, int ncol,
+                                  int c_pad, int d, unsigned wait_us) {
     const size_t n = desc ? (size_t)H * c_pad * d : 0;
     const size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
     if (i < (size_t)H * C) cnt[i] = 0;
@@ -69,7 +71,7 @@ __global__ void route_prep_kernel(const float *__restrict__ desc, __nv_bfloat16 
     const int x = (int)(i % d);
     const int c = (int)((i / d) % c_pad);
     const int h = (int)(i / ((size_t)d * c_pad));
-    float v = c < C ? desc[((size_t)h * C + c) * d + x] : 0.f;
+    float v = c < ncol ? desc[((size_t)h * C + col_chunk[c]) * d + x] : 0.f;
     const __nv_bfloat16 hi = __float2bfloat16_rn(v);
     v -= __bfloat162float(hi);
     const __nv_bfloat16 mid = __float2bfloat16_rn(v);
@@ -87,10 +89,13 @@ struct RouteParams {
     int *cnt;
     int32_t *qlist;
     const int32_t *tok_chunk;
-    const uint32_t *anc_bits;
+    const uint32_t *cand_c;     // [C][cwords] candidate columns per query chunk
+    const int32_t *lim;         // [C] prefix mode: the candidates of a query in chunk c are the columns [0, lim[c])
+    const int32_t *reach;       // [C] columns any query up to chunk c can pick from
+    const int32_t *col_chunk;   // [ncol] chunk of a score column
     const int32_t *cap_off;
     int *status;
-    int H, L, C, c_pad, k, words, causal;
+    int H, L, C, ncol, c_pad, k, cwords, prefix;
     int tiles_per_head;     // ceil(L / 128)
     int ctas_per_head;      // the grid is H * ctas_per_head
     int sb_rows;            // chunks per scoring step (one accumulator's worth)
@@ -101,9 +106,9 @@ struct RouteParams {
     size_t cap_total;
 };
 
-// chunks a tile can pick from: those before the chunk of its last row (causal), else all
+// score columns a tile can pick from: what the chunk of its last row can reach
 __device__ __forceinline__ int chunks_in_reach(const RouteParams &p, int t) {
-    return p.causal ? p.tok_chunk[min(p.L, (t + 1) * kRtRows) - 1] : p.C;
+    return p.reach[p.tok_chunk[min(p.L, (t + 1) * kRtRows) - 1]];
 }
 
 // FEW (at most 32 padded chunks, k <= 8): the three descriptor terms form one B operand of 3 c_pad rows, so a
@@ -132,9 +137,10 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     int *hist_base = reinterpret_cast<int *>(gbase + (sQ - sbase) + p.q_stages * Q_TILE_BYTES);
     // per selection group: one histogram of C counters, or (deferred list append) two alternating histograms and
     // two alternating tables of list bases
-    const int hist_ints = (KMAX <= 8 && p.C <= 256 ? 4 : 1) * p.C;
+    const int hist_ints = (KMAX <= 8 && p.C <= kRtDeferredChunks ? 4 : 1) * p.C;
     int *s_cap = hist_base + NG * hist_ints;                             // copy of cap_off[0 .. C)
-    uint16_t *s_reach = reinterpret_cast<uint16_t *>(s_cap + p.C);      // chunks in reach of each of this CTA's units
+    int *s_col = s_cap + p.C;                                            // copy of col_chunk[0 .. ncol)
+    uint16_t *s_reach = reinterpret_cast<uint16_t *>(s_col + p.ncol);   // columns in reach of each of this CTA's units
     // threshold selection: per group, surv_cap slots of (score, column) per query row; slot e of row r at [e][r]
     float *surv_base = reinterpret_cast<float *>(reinterpret_cast<uintptr_t>(s_reach + p.tiles_per_head / p.ctas_per_head + 16) + 15 & ~(uintptr_t)15);
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
@@ -172,6 +178,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     const int nu = (p.tiles_per_head - part + p.ctas_per_head - 1) / p.ctas_per_head;      // units of this CTA
     auto unit_of = [&](int n) { return part + n * p.ctas_per_head; };
     for (int x = threadIdx.x; x < p.C; x += kRtThreads) s_cap[x] = p.cap_off[x];
+    for (int x = threadIdx.x; x < p.ncol; x += kRtThreads) s_col[x] = p.col_chunk[x];
     for (int x = threadIdx.x; x < nu; x += kRtThreads) s_reach[x] = (uint16_t)chunks_in_reach(p, unit_of(x));
     __syncthreads();
     constexpr int ACC_COLS = 512 / NG;   // TMEM columns per accumulator (NG = 4 only with sb_rows <= 128)
@@ -185,21 +192,26 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             prefetch_tensormap(&tmD);
             int res_sb = -1, qn = 0, dn = 0;
             bool ok = true;
-            for (int n = 0; ok && n < nu; ++n) {
-                const int u = unit_of(n);
-                const int reach = s_reach[n], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
+            // Streamed descriptor blocks are shared by a round of NG consecutive units (one per selection group):
+            // the round's Q tiles are loaded first, then every block is loaded once and scored against all of
+            // them.  With a resident block a round is one unit.
+            const int grp = resident ? 1 : NG;
+            for (int n0 = 0; ok && n0 < nu; n0 += grp) {
+                const int n1 = min(n0 + grp, nu);
+                int n_sb = 1;
+                for (int n = n0; n < n1; ++n) n_sb = max(n_sb, (s_reach[n] + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a column in reach
+                for (int n = n0; ok && n < n1; ++n) {
+                    const int st = qn % p.q_stages;
+                    ok = mbar_wait(bar(Q_EMPTY + st), ((qn / p.q_stages) & 1) ^ 1, abort_flag, p.status, RW_QEMPTY);
+                    if (!ok) break;
+                    mbar_expect_tx(bar(Q_FULL + st), Q_TILE_BYTES);
+#pragma unroll
+                    for (int sub = 0; sub < SUB; ++sub)
+                        tma_load_2d(sQ + st * Q_TILE_BYTES + sub * Q_SUB_BYTES, &tmQ, sub * 64, h * p.L + unit_of(n) * kRtRows, bar(Q_FULL + st));
+                    ++qn;
+                }
                 for (int rep = 0; ok && rep < n_pass; ++rep)
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
-                    if (sb == 0 && rep == 0) {
-                        const int st = qn % p.q_stages;
-                        ok = mbar_wait(bar(Q_EMPTY + st), ((qn / p.q_stages) & 1) ^ 1, abort_flag, p.status, RW_QEMPTY);
-                        if (!ok) break;
-                        mbar_expect_tx(bar(Q_FULL + st), Q_TILE_BYTES);
-#pragma unroll
-                        for (int sub = 0; sub < SUB; ++sub)
-                            tma_load_2d(sQ + st * Q_TILE_BYTES + sub * Q_SUB_BYTES, &tmQ, sub * 64, h * p.L + u * kRtRows, bar(Q_FULL + st));
-                        ++qn;
-                    }
                     if (resident ? dn == 0 : sb != res_sb) {
                         ok = mbar_wait(bar(D_EMPTY), (dn & 1) ^ 1, abort_flag, p.status, RW_DEMPTY);
                         if (!ok) break;
@@ -243,63 +255,68 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
 #pragma unroll
             for (int x = 0; x < NG; ++x) nacc_total[x] = 0;
             bool ok = true;
-            for (int n = first; ok && n < nu; n += stride) {
-                const int reach = s_reach[n], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
-                const int buf = n % NG;
-                const int qn = n, st = qn % p.q_stages;
+            // a round: one unit (resident block; the two issuers take alternate units), or NG consecutive units that
+            // share every streamed block
+            const int grp = resident ? 1 : NG;
+            for (int n0 = first; ok && n0 < nu; n0 += resident ? stride : grp) {
+                const int n1 = min(n0 + grp, nu);
+                int n_sb = 1;
+                for (int n = n0; n < n1; ++n) n_sb = max(n_sb, (s_reach[n] + p.sb_rows - 1) / p.sb_rows);
+                for (int n = n0; ok && n < n1; ++n)
+                    ok = mbar_wait(bar(Q_FULL + n % p.q_stages), (n / p.q_stages) & 1, abort_flag, p.status, RW_QFULL);
                 for (int rep = 0; ok && rep < n_pass; ++rep)
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
-                    if (sb == 0 && rep == 0) {
-                        ok = mbar_wait(bar(Q_FULL + st), (qn / p.q_stages) & 1, abort_flag, p.status, RW_QFULL);
-                        if (!ok) break;
-                    }
                     if (resident ? dn == 0 : sb != res_sb) {
                         ok = mbar_wait(bar(D_FULL), dn & 1, abort_flag, p.status, RW_DFULL);
                         if (!ok) break;
                         ++dn;
                         res_sb = sb;
                     }
-                    const int uses = nacc_total[buf];
-                    ok = mbar_wait(bar(ACC_EMPTY + buf), (uses & 1) ^ 1, abort_flag, p.status, RW_ACCEMPTY);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const int rows_sb = max(16, min(min(p.sb_rows, p.c_pad - sb * p.sb_rows), (reach - sb * p.sb_rows + 15) & ~15));
-                    const uint64_t qd = q_desc0 + (uint64_t)(st * (Q_TILE_BYTES >> 4));
-                    if (FEW) {
-                        // one chain: B = the 3 c_pad rows (hi, mid, lo terms) of the block, three column groups out
-                        const uint32_t idesc = idesc_bf16_f32(128, 3 * p.c_pad, 0, 0);
-                        const uint32_t acc = tmem + buf * ACC_COLS;
-#pragma unroll
-                        for (int ks = 0; ks < D / 16; ++ks)
-                            mma_ss_lo(acc, (uint32_t)qd + (((ks >> 2) * Q_SUB_BYTES + (ks & 3) * 32) >> 4), (uint32_t)(qd >> 32),
-                                      (uint32_t)d_term[ks >> 2] + (((ks & 3) * 32) >> 4), (uint32_t)(d_term[ks >> 2] >> 32), idesc, ks != 0);
-                    } else
-                    for (int n0 = 0; n0 < rows_sb; n0 += 256) {       // one instruction spans up to 256 chunks
-                        const int n = min(256, rows_sb - n0);
-                        const uint32_t idesc = idesc_bf16_f32(128, n, 0, 0);
-                        const uint32_t acc = tmem + buf * ACC_COLS + n0;
-                        const uint32_t nofs = (uint32_t)(((resident ? sb * p.sb_rows : 0) + n0) * 128) >> 4;
-#pragma unroll
-                        for (int term = 0; term < 3; ++term) {
+                    for (int n = n0; ok && n < n1; ++n) {
+                        const int reach = s_reach[n];
+                        if (sb >= max(1, (reach + p.sb_rows - 1) / p.sb_rows)) continue;       // this unit needs no such block
+                        const int buf = n % NG, st = n % p.q_stages;
+                        const int uses = nacc_total[buf];
+                        ok = mbar_wait(bar(ACC_EMPTY + buf), (uses & 1) ^ 1, abort_flag, p.status, RW_ACCEMPTY);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const int rows_sb = max(16, min(min(p.sb_rows, p.c_pad - sb * p.sb_rows), (reach - sb * p.sb_rows + 15) & ~15));
+                        const uint64_t qd = q_desc0 + (uint64_t)(st * (Q_TILE_BYTES >> 4));
+                        if (FEW) {
+                            // one chain: B = the 3 c_pad rows (hi, mid, lo terms) of the block, three column groups out
+                            const uint32_t idesc = idesc_bf16_f32(128, 3 * p.c_pad, 0, 0);
+                            const uint32_t acc = tmem + buf * ACC_COLS;
 #pragma unroll
                             for (int ks = 0; ks < D / 16; ++ks)
                                 mma_ss_lo(acc, (uint32_t)qd + (((ks >> 2) * Q_SUB_BYTES + (ks & 3) * 32) >> 4), (uint32_t)(qd >> 32),
-                                          (uint32_t)d_term[term * SUB + (ks >> 2)] + nofs + (((ks & 3) * 32) >> 4),
-                                          (uint32_t)(d_term[term * SUB + (ks >> 2)] >> 32), idesc, (term | ks) != 0);
+                                          (uint32_t)d_term[ks >> 2] + (((ks & 3) * 32) >> 4), (uint32_t)(d_term[ks >> 2] >> 32), idesc, ks != 0);
+                        } else {
+                            // one instruction spans the step's columns (at most 256)
+                            const uint32_t idesc = idesc_bf16_f32(128, rows_sb, 0, 0);
+                            const uint32_t acc = tmem + buf * ACC_COLS;
+                            const uint32_t nofs = (uint32_t)((resident ? sb * p.sb_rows : 0) * 128) >> 4;
+#pragma unroll
+                            for (int term = 0; term < 3; ++term) {
+#pragma unroll
+                                for (int ks = 0; ks < D / 16; ++ks)
+                                    mma_ss_lo(acc, (uint32_t)qd + (((ks >> 2) * Q_SUB_BYTES + (ks & 3) * 32) >> 4), (uint32_t)(qd >> 32),
+                                              (uint32_t)d_term[term * SUB + (ks >> 2)] + nofs + (((ks & 3) * 32) >> 4),
+                                              (uint32_t)(d_term[term * SUB + (ks >> 2)] >> 32), idesc, (term | ks) != 0);
+                            }
                         }
+                        tc_commit(bar(ACC_FULL + buf));
+                        ++nacc_total[buf];
                     }
-                    tc_commit(bar(ACC_FULL + buf));
-                    ++nacc_total[buf];
                     // streamed blocks: the next step, if it needs another block, may overwrite this one once
                     // these MMAs are done
-                    if (!resident) {
+                    if (ok && !resident) {
                         int nsb = sb + 1;
                         bool more = true;
-                        if (nsb >= n_sb) { nsb = 0; more = rep + 1 < n_pass || n + 1 < nu; }
+                        if (nsb >= n_sb) { nsb = 0; more = rep + 1 < n_pass || n1 < nu; }
                         if (more && nsb != sb) tc_commit(bar(D_EMPTY));
                     }
                 }
-                if (ok) tc_commit(bar(Q_EMPTY + st));
+                for (int n = n0; ok && n < n1; ++n) tc_commit(bar(Q_EMPTY + n % p.q_stages));
             }
         }
     } else if (warp < 2 + 4 * NG) {
@@ -320,11 +337,14 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
         };
         // the sorted list of this pass's picks lives in registers (a 64-entry list leaves room for one selection group)
         constexpr int KR = KMAX;
-        // With few chunks the list append of a unit is finished after the next unit's selection, so the
-        // round trip of the range-reserving atomics is hidden; `pend` is the unit whose append is open.
-        const bool deferred = KMAX <= 8 && p.C <= 256;
-        struct Pending { int h, i, j[KR], rank[KR], base0, base1; bool live, open; } pend;
-        pend.open = false; pend.live = false; pend.h = 0; pend.i = 0; pend.base0 = 0; pend.base1 = 0;
+        // With at most kRtDeferredChunks chunks the list append of a unit is finished after the next unit's selection,
+        // so the round trip of the range-reserving atomics is hidden; `pend` is the unit whose append is open.
+        const bool deferred = KMAX <= 8 && p.C <= kRtDeferredChunks;
+        constexpr int NB = kRtDeferredChunks / 128;           // chunks a thread owns in the deferred append
+        struct Pending { int h, i, j[KR], rank[KR], base[NB]; bool live, open; } pend;
+        pend.open = false; pend.live = false; pend.h = 0; pend.i = 0;
+#pragma unroll
+        for (int y = 0; y < NB; ++y) pend.base[y] = 0;
         // Deferred append, one group barrier per unit.  Unit n uses histogram n & 1 and base table n & 1:
         //   before the barrier: the bases that unit n - 1's range-reserving atomics returned go into the table,
         //     and unit n's picks take their tile-local ranks from the histogram;
@@ -334,8 +354,9 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
         int ndef = 0;                          // units this group has appended so far
         auto write_bases = [&]() {
             int *baseb = hist + (2 + (ndef & 1)) * p.C;
-            if (gt < p.C) baseb[gt] = pend.base0;
-            if (gt + 128 < p.C) baseb[gt + 128] = pend.base1;
+#pragma unroll
+            for (int y = 0; y < NB; ++y)
+                if (gt + 128 * y < p.C) baseb[gt + 128 * y] = pend.base[y];
         };
         auto write_entries = [&]() {
             const int *baseb = hist + (2 + (ndef & 1)) * p.C;
@@ -353,26 +374,43 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             for (int x = gt; x < 2 * p.C; x += 128) hist[x] = 0;
             ok = group_sync();
         }
-        int nx_ci = 0;
-        uint32_t nx_aw = 0u;
+        // Candidates of a row, over score columns.  Prefix mode (the causal rule): the columns [0, lim); else a
+        // bitmap row.  Both are fetched a unit ahead, so that these dependent loads are never waited for.
+        int nx_ci = 0, nx_lim = 0;
+        uint32_t nx_w0 = 0u;
+        auto fetch_row = [&](int i0, bool live0) {
+            nx_ci = live0 ? p.tok_chunk[i0] : 0;
+        };
+        auto fetch_cand = [&](bool live0) {
+            nx_lim = live0 ? (p.prefix ? p.lim[nx_ci] : 0) : 0;
+            nx_w0 = (live0 && !p.prefix) ? p.cand_c[(size_t)nx_ci * p.cwords] : 0u;
+        };
         if (sg < nu) {
             const int i0 = unit_of(sg) * kRtRows + r;
-            nx_ci = i0 < p.L ? p.tok_chunk[i0] : 0;
-            nx_aw = i0 < p.L ? p.anc_bits[(size_t)nx_ci * p.words] : 0u;
+            fetch_row(i0, i0 < p.L);
+            fetch_cand(i0 < p.L);
         }
         for (int n = sg; ok && n < nu; n += NG) {
             const int u = unit_of(n);
-            const int reach = s_reach[n], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a chunk in reach
+            const int reach = s_reach[n], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a column in reach
             const int i = u * kRtRows + r;
             const bool live = i < p.L;
-            const int ci = nx_ci;
-            const uint32_t aw_next = nx_aw;
+            const int ci = nx_ci, lim_i = nx_lim;
+            const uint32_t w0 = nx_w0;
             const int i2 = unit_of(n + NG) * kRtRows + r;
             const bool live2 = n + NG < nu && i2 < p.L;
-            if (live2) nx_ci = p.tok_chunk[i2];       // the next unit's chunk, loaded a unit ahead (its anchor word follows below)
+            fetch_row(i2, live2);       // the next unit's chunk, loaded a unit ahead (its candidates follow below)
+            // candidate bits of the 32 columns from j0 on
+            auto cand_bits = [&](int j0) -> uint32_t {
+                if (p.prefix) {
+                    const int m = lim_i - j0;
+                    return m <= 0 ? 0u : (m >= 32 ? 0xffffffffu : ((1u << m) - 1u));
+                }
+                return j0 == 0 ? w0 : (live ? p.cand_c[(size_t)ci * p.cwords + (j0 >> 5)] : 0u);
+            };
             // More than 64 picks are taken 64 at a time: every pass sees the tile's scores again (the issuer
-            // recomputes them) and considers only the chunks that come after the previous pass's last pick in
-            // the order of the result (score descending, then chunk index ascending).
+            // recomputes them) and considers only the columns that come after the previous pass's last pick in
+            // the order of the result (score descending, then column ascending).
             [[maybe_unused]] float prev_s = INFINITY;
             [[maybe_unused]] int prev_j = -1;
             for (int pass = 0; ok && pass < n_pass; ++pass) {
@@ -380,6 +418,28 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             TopK<KMAX> top;
             top.init();
             [[maybe_unused]] float kth = -INFINITY;
+            // One candidate into the sorted list (descending; equal scores keep their arrival order, which is
+            // ascending column): it goes behind every entry that is at least as large, the entries after it move
+            // down one slot and the last falls off.  Every slot is decided on its own from the compare of its
+            // entry and of the entry before it, so the slots do not wait for one another.
+            auto insert = [&](float cv, int cj) {
+                bool ge[KR];
+#pragma unroll
+                for (int x = 0; x < KR; ++x) ge[x] = top.s[x] >= cv;
+#pragma unroll
+                for (int x = KR - 1; x >= 0; --x) {
+                    const bool here = x == 0 ? true : ge[x - 1];             // the new entry's slot is x, or before x
+                    const float ps = x == 0 ? cv : top.s[x - 1];
+                    const int pj = x == 0 ? cj : top.j[x - 1];
+                    top.s[x] = ge[x] ? top.s[x] : (here ? cv : ps);
+                    top.j[x] = ge[x] ? top.j[x] : (here ? cj : pj);
+                }
+            };
+            auto update_kth = [&]() {
+                kth = top.s[0];
+#pragma unroll
+                for (int x = 1; x < KR; ++x) kth = (x < kp) ? top.s[x] : kth;
+            };
             for (int sb = 0; ok && sb < n_sb; ++sb) {
                 ok = mbar_wait_spin(bar(ACC_FULL + sg), nacc & 1, abort_flag, p.status, RW_ACCFULL);
                 ok = __all_sync(0xffffffffu, ok);
@@ -388,14 +448,9 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 tc_fence_after();
                 const int rows_sb = max(16, min(min(p.sb_rows, p.c_pad - sb * p.sb_rows), (reach - sb * p.sb_rows + 15) & ~15));
                 if (FEW) {
-                    // at most 32 chunks, all in this block.  Candidate bits: a real chunk, not an anchor, strictly
-                    // earlier if causal.  The scores of the chunks in the tile's reach come eight at a time, each the
-                    // sum of its three terms (hi, mid, lo, in that order), and sink through the sorted list (strict
-                    // '>' keeps equal scores in arrival order, which is ascending chunk index).
-                    uint32_t cand = ~aw_next;
-                    const int lim = min(p.C, p.causal ? ci : p.C);
-                    cand = lim <= 0 ? 0u : (lim >= 32 ? cand : (cand & ((1u << lim) - 1u)));
-                    if (!live) cand = 0u;
+                    // at most 32 columns, all in this block.  The scores of the columns in the tile's reach come eight
+                    // at a time, each the sum of its three terms (hi, mid, lo, in that order), and go into the list.
+                    const uint32_t cand = cand_bits(0);
                     uint32_t a[8], b[8], c3[8];
                     tmem_ld8(acc, a);
                     tmem_ld8(acc + p.c_pad, b);
@@ -414,58 +469,12 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                             }
 #pragma unroll
                             for (int c = 0; c < 8; ++c) {
-                                float cv = ((cand >> (g * 8 + c)) & 1u) ? f[c] : -INFINITY;
-                                int cj = g * 8 + c;
-                                bool placed = false;
-#pragma unroll
-                                for (int x = 0; x < KR; ++x) {
-                                    // the new score takes the first slot it beats (strict '>': equal scores keep
-                                    // their arrival order, ascending chunk index); from there on every entry moves
-                                    // down one slot, equal ones included, and the last falls off
-                                    const bool up = placed || cv > top.s[x];
-                                    placed = up;
-                                    const float ts = top.s[x];
-                                    const int tj = top.j[x];
-                                    top.s[x] = up ? cv : ts;
-                                    top.j[x] = up ? cj : tj;
-                                    cv = up ? ts : cv;
-                                    cj = up ? tj : cj;
-                                }
+                                insert(((cand >> (g * 8 + c)) & 1u) ? f[c] : -INFINITY, g * 8 + c);     // -inf changes nothing
                             }
                         }
                     }
                 } else {
-                // candidate bits of the 32 chunks from j0 on: a real chunk, not an anchor, strictly earlier if causal
-                auto cand_bits = [&](int j0) {
-                    const uint32_t aw = j0 == 0 ? aw_next : (live ? p.anc_bits[(size_t)ci * p.words + (j0 >> 5)] : 0u);
-                    uint32_t cand = ~aw;
-                    const int lim = min(p.C, p.causal ? ci : p.C) - j0;     // chunks j0 .. j0 + lim - 1 may be picked
-                    cand = lim <= 0 ? 0u : (lim >= 32 ? cand : (cand & ((1u << lim) - 1u)));
-                    return live ? cand : 0u;
-                };
-                // one candidate into the sorted list: it takes the first slot it beats (strict '>': equal scores keep
-                // their arrival order, ascending chunk index); from there on every entry moves down one slot, equal
-                // ones included, and the last falls off
-                auto insert = [&](float cv, int cj) {
-                    bool placed = false;
-#pragma unroll
-                    for (int x = 0; x < KR; ++x) {
-                        const bool up = placed || cv > top.s[x];
-                        placed = up;
-                        const float ts = top.s[x];
-                        const int tj = top.j[x];
-                        top.s[x] = up ? cv : ts;
-                        top.j[x] = up ? cj : tj;
-                        cv = up ? ts : cv;
-                        cj = up ? tj : cj;
-                    }
-                };
-                auto update_kth = [&]() {
-                    kth = top.s[0];
-#pragma unroll
-                    for (int x = 1; x < KR; ++x) kth = (x < kp) ? top.s[x] : kth;
-                };
-                // Best-first extraction: up to k members of a 32-chunk block can enter the list; they are taken one
+                // Best-first extraction: up to k members of a 32-column block can enter the list; they are taken one
                 // per round, the block's best first, while any row of the warp still has one above its k-th score.
                 auto extract_blocks = [&]() {
                 for (int cc = 0; cc < rows_sb; cc += 32) {
@@ -514,84 +523,165 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 };
                 // Threshold selection (lists of at most 16 picks).  A lower bound `thr` of the row's final k-th score
                 // is known before any candidate is inserted: in the tile's first scoring step it is the k-th largest
-                // of G group maxima (group = chunks with equal index mod G: k groups whose maximum is at least thr
+                // of G group maxima (group = columns with equal index mod G: k groups whose maximum is at least thr
                 // hold k different candidates at least thr), later the list's own k-th score.  Only the candidates at
                 // least thr - a few more than k per row - go through the sorted insertion, which is where the work
-                // is: each row's survivors are queued in shared memory (score and column, in chunk order) and the
-                // warp inserts every row's e-th survivor together, so the insertion runs max-over-rows(survivors)
-                // times per warp instead of once per chunk.  A row with more survivors than slots (many equal scores)
-                // sends its warp through the best-first extraction instead, which needs no queue.
+                // is: each row's survivors are queued in shared memory (score and column, in column order: the lower
+                // half of the step's blocks fills the queue from the front, the upper half from the back, two
+                // independent streams of instructions) and the warp inserts every row's e-th survivor together, so
+                // the insertion runs max-over-rows(survivors) times per warp instead of once per column.  A row with
+                // more survivors than slots (many equal scores) sends its warp through the best-first extraction
+                // instead, which needs no queue.  A block all of whose columns are candidates for all 32 rows (most
+                // blocks: the candidates are a prefix of the columns) skips the candidate masks.
                 bool fast = KMAX <= 16 && p.surv_cap > 0;
                 if (fast) {
                     constexpr int G = KMAX <= 8 ? 16 : 32;
+                    const int jb = sb * p.sb_rows;
                     float thr = kth;
                     if (sb == 0) {
                         float gm[G];
 #pragma unroll
                         for (int x = 0; x < G; ++x) gm[x] = -INFINITY;
 #pragma unroll 1
-                        for (int cc = 0; cc < rows_sb; cc += 32) {
-                            uint32_t v[32];
+                        for (int cc = 0; cc < rows_sb; cc += 64) {          // two blocks of 32 columns in flight
+                            const bool two = cc + 32 < rows_sb;
+                            uint32_t v[32], w[32];
                             tmem_ld32(acc + cc, v);
-                            const uint32_t cand = cand_bits(sb * p.sb_rows + cc);
+                            if (two) tmem_ld32(acc + cc + 32, w);
+                            const uint32_t cand = cand_bits(jb + cc), cand2 = two ? cand_bits(jb + cc + 32) : 0u;
                             tmem_wait_ld();
-                            if (__all_sync(0xffffffffu, cand == 0xffffffffu)) {
+                            if (__all_sync(0xffffffffu, cand == 0xffffffffu && (!two || cand2 == 0xffffffffu))) {
 #pragma unroll
                                 for (int x = 0; x < G; ++x)
                                     gm[x] = G == 16 ? max3(gm[x], __uint_as_float(v[x]), __uint_as_float(v[x + 16])) : fmaxf(gm[x], __uint_as_float(v[x]));
+                                if (two) {
+#pragma unroll
+                                    for (int x = 0; x < G; ++x)
+                                        gm[x] = G == 16 ? max3(gm[x], __uint_as_float(w[x]), __uint_as_float(w[x + 16])) : fmaxf(gm[x], __uint_as_float(w[x]));
+                                }
                             } else {
 #pragma unroll
                                 for (int c = 0; c < 32; ++c) {
                                     const float f = ((cand >> c) & 1u) ? __uint_as_float(v[c]) : -INFINITY;
-                                    gm[c % G] = fmaxf(gm[c % G], f);
+                                    const float f2 = ((cand2 >> c) & 1u) ? __uint_as_float(w[c]) : -INFINITY;
+                                    gm[c % G] = max3(gm[c % G], f, f2);
                                 }
                             }
                         }
-                        float t[KR];           // the KR largest group maxima, descending
+                        // sort the group maxima, descending (bitonic network: a fixed sequence of compare-exchange
+                        // steps, every index a compile-time constant), and take the k-th
 #pragma unroll
-                        for (int y = 0; y < KR; ++y) t[y] = -INFINITY;
+                        for (int k2 = 2; k2 <= G; k2 <<= 1)
 #pragma unroll
-                        for (int x = 0; x < G; ++x) {
-                            float cv = gm[x];
+                            for (int jj = k2 >> 1; jj > 0; jj >>= 1)
 #pragma unroll
-                            for (int y = 0; y < KR; ++y) {
-                                const float hi = fmaxf(t[y], cv);
-                                cv = fminf(t[y], cv);
-                                t[y] = hi;
-                            }
-                        }
-                        thr = t[0];
+                                for (int ii = 0; ii < G; ++ii) {
+                                    const int ll = ii ^ jj;
+                                    if (ll > ii) {
+                                        const float hi = fmaxf(gm[ii], gm[ll]), lo = fminf(gm[ii], gm[ll]);
+                                        const bool desc = (ii & k2) == 0;
+                                        gm[ii] = desc ? hi : lo;
+                                        gm[ll] = desc ? lo : hi;
+                                    }
+                                }
+                        thr = gm[0];
 #pragma unroll
-                        for (int y = 1; y < KR; ++y) thr = (y < kp) ? t[y] : thr;
+                        for (int y = 1; y < KR; ++y) thr = (y < kp) ? gm[y] : thr;
                     }
-                    thr = fmaxf(thr, -FLT_MAX);          // a chunk that is not a candidate (-inf) never survives
-                    float *sv = surv_base + (size_t)sg * p.surv_cap * 160 + gt;          // 128 floats + 128 bytes per slot
-                    uint8_t *sj = reinterpret_cast<uint8_t *>(surv_base + (size_t)sg * p.surv_cap * 160 + (size_t)p.surv_cap * 128) + gt;
-                    int cnt = 0;
+                    thr = fmaxf(thr, -FLT_MAX);          // a column that is not a candidate (-inf) never survives
+                    const int cap = p.surv_cap;
+                    float *sv = surv_base + (size_t)sg * cap * 160 + gt;          // 128 floats + 128 bytes per slot
+                    uint8_t *sj = reinterpret_cast<uint8_t *>(surv_base + (size_t)sg * cap * 160 + (size_t)cap * 128) + gt;
+                    const int nblk = (rows_sb + 31) >> 5, half = (nblk + 1) >> 1;
+                    // Queue cursors as shared-memory addresses: the front stream moves up from slot 0, the back stream
+                    // down from slot cap - 1.  A survivor is stored while its stream's cursor is inside the queue and the
+                    // cursor moves whether it was stored or not, so the count stays exact; the two streams have run into
+                    // each other (or out of the queue) exactly when the counts add up to more than cap.  The stores are
+                    // predicated instructions, written out so that no branch is made of them.
+                    const uint32_t q_v = smem_u32(sv), q_j = smem_u32(sj);
+                    uint32_t lo_v = q_v, lo_j = q_j, hi_v = q_v + (cap - 1) * 512, hi_j = q_j + (cap - 1) * 128;
+                    const uint32_t lo_end = q_v + cap * 512;
+                    // the cursors advance by multiply-add with a factor of one the compiler cannot see through: that
+                    // instruction runs on the multiply-add pipe, while the compares around it fill the other one
+                    int one;
+                    asm volatile("mov.u32 %0, 1;" : "=r"(one));
 #pragma unroll 1
-                    for (int cc = 0; cc < rows_sb; cc += 32) {
-                        uint32_t v[32];
-                        tmem_ld32(acc + cc, v);
-                        const uint32_t cand = cand_bits(sb * p.sb_rows + cc);
+                    for (int b = 0; b < half; ++b) {
+                        const bool two = b + half < nblk;
+                        const int cl = b * 32, ch = (b + half) * 32;
+                        uint32_t vl[32], vh[32];
+                        tmem_ld32(acc + cl, vl);
+                        if (two) tmem_ld32(acc + ch, vh);
+                        const uint32_t cand_l = cand_bits(jb + cl), cand_h = two ? cand_bits(jb + ch) : 0u;
                         tmem_wait_ld();
+                        const bool plain = __all_sync(0xffffffffu, cand_l == 0xffffffffu && (!two || cand_h == 0xffffffffu));
+                        if (!plain) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            const float f = ((cand >> c) & 1u) ? __uint_as_float(v[c]) : -INFINITY;
-                            const bool keep = f >= thr;
-                            if (keep && cnt < p.surv_cap) {
-                                sv[cnt * 128] = f;
-                                sj[cnt * 128] = (uint8_t)(cc + c);
+                            for (int c = 0; c < 32; ++c) {
+                                vl[c] = ((cand_l >> c) & 1u) ? vl[c] : 0xff800000u;      // -inf
+                                vh[c] = ((cand_h >> c) & 1u) ? vh[c] : 0xff800000u;
                             }
-                            cnt += keep ? 1 : 0;
+                        }
+                        if (two) {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) {
+                                asm volatile(
+                                    "{\n\t.reg .pred p, q;\n\t"
+                                    "setp.ge.f32 p, %3, %4;\n\t"
+                                    "setp.lt.and.u32 q, %0, %5, p;\n\t"
+                                    "@q st.shared.f32 [%0], %3;\n\t"
+                                    "@q st.shared.u8 [%1], %2;\n\t"
+                                    "@p mad.lo.s32 %0, %6, 512, %0;\n\t"
+                                    "@p mad.lo.s32 %1, %6, 128, %1;\n\t}"
+                                    : "+r"(lo_v), "+r"(lo_j)
+                                    : "r"(cl + c), "f"(__uint_as_float(vl[c])), "f"(thr), "r"(lo_end), "r"(one)
+                                    : "memory");
+                                asm volatile(
+                                    "{\n\t.reg .pred p, q;\n\t"
+                                    "setp.ge.f32 p, %3, %4;\n\t"
+                                    "setp.ge.and.s32 q, %0, %5, p;\n\t"
+                                    "@q st.shared.f32 [%0], %3;\n\t"
+                                    "@q st.shared.u8 [%1], %2;\n\t"
+                                    "@p mad.lo.s32 %0, %6, -512, %0;\n\t"
+                                    "@p mad.lo.s32 %1, %6, -128, %1;\n\t}"
+                                    : "+r"(hi_v), "+r"(hi_j)
+                                    : "r"(ch + c), "f"(__uint_as_float(vh[c])), "f"(thr), "r"(q_v), "r"(one)
+                                    : "memory");
+                            }
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                asm volatile(
+                                    "{\n\t.reg .pred p, q;\n\t"
+                                    "setp.ge.f32 p, %3, %4;\n\t"
+                                    "setp.lt.and.u32 q, %0, %5, p;\n\t"
+                                    "@q st.shared.f32 [%0], %3;\n\t"
+                                    "@q st.shared.u8 [%1], %2;\n\t"
+                                    "@p mad.lo.s32 %0, %6, 512, %0;\n\t"
+                                    "@p mad.lo.s32 %1, %6, 128, %1;\n\t}"
+                                    : "+r"(lo_v), "+r"(lo_j)
+                                    : "r"(cl + c), "f"(__uint_as_float(vl[c])), "f"(thr), "r"(lo_end), "r"(one)
+                                    : "memory");
                         }
                     }
-                    fast = !__any_sync(0xffffffffu, cnt > p.surv_cap);
+                    const int cnt_lo = (int)(lo_v - q_v) >> 9, cnt_hi = (int)(q_v + (cap - 1) * 512 - hi_v) >> 9;
+                    fast = !__any_sync(0xffffffffu, cnt_lo + cnt_hi > cap);
                     if (fast) {
-                        const int nmax = __reduce_max_sync(0xffffffffu, cnt);
-                        const int jb = sb * p.sb_rows;
+                        // every row's e-th survivor goes into its list together; a row that has none left inserts
+                        // -inf, which changes nothing, so there is no branch; the next survivor is fetched ahead
+                        const int nlo = __reduce_max_sync(0xffffffffu, cnt_lo), nhi = __reduce_max_sync(0xffffffffu, cnt_hi);
+                        const int ntot = nlo + nhi;
+                        auto slot_of = [&](int e) { return e < nlo ? e : cap - 1 - (e - nlo); };
+                        auto live_of = [&](int e) { return e < nlo ? e < cnt_lo : e - nlo < cnt_hi; };
+                        float nv = 0.f;
+                        int nj = 0;
+                        if (ntot > 0) { nv = sv[slot_of(0) * 128]; nj = sj[slot_of(0) * 128]; }
 #pragma unroll 1
-                        for (int e = 0; e < nmax; ++e) {
-                            if (e < cnt) insert(sv[e * 128], jb + (int)sj[e * 128]);
+                        for (int e = 0; e < ntot; ++e) {
+                            const float cv = live_of(e) ? nv : -INFINITY;
+                            const int cj = jb + nj;
+                            if (e + 1 < ntot) { nv = sv[slot_of(e + 1) * 128]; nj = sj[slot_of(e + 1) * 128]; }
+                            insert(cv, cj);
                         }
                         update_kth();
                     }
@@ -602,8 +692,15 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 mbar_arrive(bar(ACC_EMPTY + sg));
             }
             if (!ok) break;
-            nx_aw = live2 ? p.anc_bits[(size_t)nx_ci * p.words] : 0u;
-            // sel_idx and the empty slots' partial log-sum-exp
+            fetch_cand(live2);
+            if (KMAX == 64) {                           // the next pass starts after this pass's last pick
+#pragma unroll
+                for (int x = 0; x < KR; ++x)
+                    if (x == kp - 1) { prev_s = top.s[x]; prev_j = top.j[x]; }
+            }
+            // columns -> chunks; sel_idx and the empty slots' partial log-sum-exp
+#pragma unroll
+            for (int x = 0; x < KR; ++x) top.j[x] = top.j[x] >= 0 ? s_col[top.j[x]] : -1;
             int32_t *out = p.sel + ((size_t)h * p.L + i) * p.k + pass * 64;
             float *pl = p.part_lse + ((size_t)h * p.L + i) * p.k + pass * 64;
             if (live) {
@@ -613,11 +710,6 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                         out[x] = top.j[x];
                         if (top.j[x] < 0) pl[x] = -INFINITY;
                     }
-            }
-            if (KMAX == 64) {                           // the next pass starts after this pass's last pick
-#pragma unroll
-                for (int x = 0; x < KR; ++x)
-                    if (x == kp - 1) { prev_s = top.s[x]; prev_j = top.j[x]; }
             }
             if (deferred) {
                 int *cntb = hist + (ndef & 1) * p.C;
@@ -631,14 +723,13 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 ok = group_sync();
                 if (!ok) break;
                 if (pend.open) write_entries();
-                pend.base0 = 0; pend.base1 = 0;
-                if (gt < p.C) {
-                    const int n = cntb[gt];
-                    if (n) { pend.base0 = atomicAdd(&p.cnt[h * p.C + gt], n); cntb[gt] = 0; }
-                }
-                if (gt + 128 < p.C) {
-                    const int n = cntb[gt + 128];
-                    if (n) { pend.base1 = atomicAdd(&p.cnt[h * p.C + gt + 128], n); cntb[gt + 128] = 0; }
+#pragma unroll
+                for (int y = 0; y < NB; ++y) {
+                    pend.base[y] = 0;
+                    if (gt + 128 * y < p.C) {
+                        const int n = cntb[gt + 128 * y];
+                        if (n) { pend.base[y] = atomicAdd(&p.cnt[h * p.C + gt + 128 * y], n); cntb[gt + 128 * y] = 0; }
+                    }
                 }
 #pragma unroll
                 for (int x = 0; x < KR; ++x) pend.j[x] = njr[x];
@@ -802,7 +893,7 @@ int launch_lists_from_sel(const moc_plan *p, int32_t *sel, void *ws, cudaStream_
     int *cnt = ws_ptr<int>(ws, p->ws.cnt);
     int *status = ws_ptr<int>(ws, p->ws.status);
     const size_t n = std::max((size_t)p->H * p->C, (size_t)kStatusWords);
-    route_prep_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(nullptr, nullptr, cnt, status, p->H, p->C, p->c_pad, p->d, p->wait_us);
+    route_prep_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(nullptr, nullptr, cnt, status, nullptr, p->H, p->C, p->ncol, p->c_pad, p->d, p->wait_us);
     MOC_LAUNCH_CHECK();
     if (p->k > 0) {
         const size_t smem = 2 * sizeof(int) * (size_t)p->C;
@@ -824,16 +915,17 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
     __nv_bfloat16 *desc3 = ws_ptr<__nv_bfloat16>(ws, p->ws.desc3);
     {
         const size_t n = std::max((size_t)p->H * p->c_pad * D, (size_t)kStatusWords);   // covers H * C too
-        route_prep_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(desc, desc3, cnt, status, p->H, p->C, p->c_pad, D, p->wait_us);
+        route_prep_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(desc, desc3, cnt, status, p->d_col_chunk, p->H, p->C, p->ncol, p->c_pad, D, p->wait_us);
         MOC_LAUNCH_CHECK();
     }
     if (p->k > 0) {
         RouteParams a;
         a.sel = sel; a.part_lse = ws_ptr<float>(ws, p->ws.part_lse); a.cnt = cnt;
         a.qlist = ws_ptr<int32_t>(ws, p->ws.qlist);
-        a.tok_chunk = p->d_tok_chunk; a.anc_bits = p->d_anc_bits; a.cap_off = p->d_cap_off; a.status = status;
-        a.H = p->H; a.L = p->L; a.C = p->C; a.c_pad = p->c_pad; a.k = p->k; a.words = p->words;
-        a.causal = (p->flags & MOC_FLAG_CAUSAL) ? 1 : 0;
+        a.tok_chunk = p->d_tok_chunk; a.cand_c = p->d_cand_c; a.lim = p->d_lim; a.reach = p->d_reach;
+        a.col_chunk = p->d_col_chunk; a.cap_off = p->d_cap_off; a.status = status;
+        a.H = p->H; a.L = p->L; a.C = p->C; a.ncol = p->ncol; a.c_pad = p->c_pad; a.k = p->k; a.cwords = p->cwords;
+        a.prefix = p->prefix_mode;
         a.tiles_per_head = (p->L + kRtRows - 1) / kRtRows;
         a.d_rows = p->c_pad <= kRtResident ? p->c_pad : kRtBlock;
         // a scoring step fills one accumulator: a quarter of TMEM (128 chunks) with four selection groups, half of it
@@ -849,7 +941,8 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         const int ng = few ? 4 : p->k > 32 ? 1 : 2;
         a.n_pass = p->k > 64 ? (p->k + 63) / 64 : 1;
         // one histogram per group, the list offsets, and one byte per unit of a CTA
-        const size_t hist = (ng * (p->k <= 8 && p->C <= 256 ? 4 : 1) + 1) * sizeof(int) * (size_t)p->C + 2 * (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
+        const size_t hist = (ng * (p->k <= 8 && p->C <= kRtDeferredChunks ? 4 : 1) + 1) * sizeof(int) * (size_t)p->C + sizeof(int) * (size_t)p->ncol +
+                            2 * (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
         if (d_block + q_tile + hist > budget) return MOC_ERR_SHAPE;
         // threshold selection (lists of at most 16 picks, not the few-chunk case): survivor slots per row, as many
         // as fit beside two Q stages, at least k + 4 (else the best-first extraction alone is used)
@@ -862,6 +955,7 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
             surv = 16 + a.surv_cap * per_slot;
         }
         a.q_stages = (int)std::min<size_t>(4, (budget - d_block - hist - surv) / q_tile);
+        if (a.d_rows != p->c_pad && a.q_stages < ng) return MOC_ERR_SHAPE;      // streamed blocks: a round's Q tiles are held together
         const size_t smem = 1024 + d_block + a.q_stages * q_tile + hist + surv;
         CUtensorMap tmQ, tmD;
         if (int r = make_tmap_2d_bf16(&tmQ, Q, (uint64_t)p->H * p->L, D, kRtRows)) return r;
@@ -872,6 +966,7 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         route_tc_kernel<D, KM, NG, FW><<<grid, rt_threads(NG), smem, s>>>(tmQ, tmD, a);                                     \
     } while (0)
         if (p->k <= 4) { if (few) MOC_ROUTE_CASE(4, 4, true); else MOC_ROUTE_CASE(4, 2, false); }
+        else if (p->k <= 6 && !few) MOC_ROUTE_CASE(6, 2, false);
         else if (p->k <= 8) { if (few) MOC_ROUTE_CASE(8, 4, true); else MOC_ROUTE_CASE(8, 2, false); }
         else if (p->k <= 16) MOC_ROUTE_CASE(16, 2, false);
         else if (p->k <= 32) MOC_ROUTE_CASE(32, 2, false);
