@@ -153,6 +153,22 @@ int moc_route(const moc_plan *plan, const void *Q, const float *desc, int32_t *s
  * Slots need not be sorted or packed to the front. */
 int moc_lists_from_sel(const moc_plan *plan, int32_t *sel_idx, void *ws, void *stream);
 
+/* Sec. 3.1, "Context drop-off" and "Context drop-in": the training-time regularisers of the routed
+ * selection, applied in place to a sel_idx that moc_route wrote (or moc_lists_from_sel checked), after
+ * which the lists in ws are rebuilt for the edited selection (as by moc_lists_from_sel).  Per query:
+ *   drop-off: p_drop = U p_max, U ~ Uniform[0, 1); floor(p_drop k) of the query's picks are removed (at
+ *             most all it has), each chosen uniformly among the picks still there;
+ *   drop-in:  m ~ Poisson(lambda) chunks are added, each chosen uniformly among the chunks the query may
+ *             route to (not an anchor, strictly earlier if causal) that are neither picks of the query
+ *             (kept or just removed) nor added already; they go into the free slots, lowest first, and
+ *             stop when the k slots are full or no chunk is left.
+ * The paper gives neither p_max nor lambda; here 0 <= p_max <= 1 and 0 <= lambda <= 8 (MOC_ERR_SHAPE
+ * otherwise); p_max = 0 and lambda = 0 leave the selection as it is.  The draws are a pure function of
+ * (seed, head, token): Philox4x32-10 with the seed as key and (token, head, draw / 4, 0) as counter, so a
+ * run is reproducible and independent of launch shape. */
+int moc_context_drop(const moc_plan *plan, int32_t *sel_idx, float p_max, float lambda, uint64_t seed, void *ws,
+                     void *stream);
+
 /* Step 6 - sparse attention (Eq. 2): O_i = softmax(scale q_i K_Omega^T) V_Omega over the
  * tokens of the chunks in Omega(i) = anchors(c(i)) U sel_idx[i]; lse as defined above.
  * bf16 products, fp32 accumulation and softmax.
@@ -183,6 +199,35 @@ int moc_selected_pairs(const moc_plan *plan, const void *ws, void *stream, int64
  * or MOC_ERR_WORKSPACE, with `detail` (optional) receiving a kernel-specific code (for a
  * timeout, which wait gave up). */
 int moc_get_status(const moc_plan *plan, const void *ws, void *stream, int *device_status, int *detail);
+
+/* Outer-loop context routing (the paper's appendix of that name): before any attention, whole shots of the
+ * context are pre-selected for one query block; the selected shots, the mandatory text and the block's own
+ * shots form a reduced stream on which the calls above then run with a plan of its own.
+ *   High-level chunk Psi_s = every token of shot s (all chunks with that chunk_shot value); S shots.
+ *   phi(Psi_s) = mean of the context features over the shot: computed here as the token-weighted mean of
+ *                `desc`, the chunk descriptors that moc_chunk_pool made of the context features;
+ *   x_g        = mean of the query features Xq ([H][L][d] bf16, each of the H streams on its own) over the
+ *                block of tokens [q_tok0, q_tok1);
+ *   scores     = <x_g, phi(Psi_s)> for every shot ([H][S], fp32); shot_desc [H][S][d] fp32;
+ *   sel_shot   = [H][top_m] int32: the top_m best shots among those that END before the block begins (a
+ *                shot holding a token >= q_tok0 is not history), best first, equal scores to the earlier
+ *                shot, -1 padded.  ws: scratch of moc_workspace_bytes (its pooling area is used). */
+int moc_outer_num_shots(const moc_plan *plan, int32_t *n_shots);
+int moc_outer_route(const moc_plan *plan, const void *Xq, const float *desc, int32_t q_tok0, int32_t q_tok1, int32_t top_m,
+                    float *shot_desc, float *scores, int32_t *sel_shot, void *ws, void *stream);
+
+/* HOST only (no device work): the chunk table of the reduced stream for one selection.  Kept, in stream
+ * order: every text chunk (the mandatory elements), the chunks of the n_sel shots in sel_shot (HOST, -1
+ * entries skipped) and the chunks of the shots that overlap the block [q_tok0, q_tok1).  Outputs (HOST,
+ * sized by the caller for the original stream: C + 1, C, C and L entries): the reduced chunk_off /
+ * chunk_shot / chunk_mod, ready for moc_plan_create, and tok_map[r] = original token of reduced token r. */
+int moc_outer_reduced_layout(const moc_plan *plan, const int32_t *sel_shot, int32_t n_sel, int32_t q_tok0, int32_t q_tok1,
+                             int32_t *n_chunks, int32_t *n_tokens, int32_t *chunk_off, int32_t *chunk_shot,
+                             uint8_t *chunk_mod, int32_t *tok_map);
+
+/* out[h][r][:] = X[h][tok_map[r]][:] for r < n_out: the rows of a [H][L][d] bf16 tensor that the reduced
+ * stream keeps (tok_map: DEVICE int32; out: DEVICE [H][n_out][d] bf16). */
+int moc_gather_tokens(const moc_plan *plan, const void *X, const int32_t *tok_map, int32_t n_out, void *out, void *stream);
 
 /* How many kernel launches the library has enqueued since it was loaded. */
 int64_t moc_launch_count(void);

@@ -144,6 +144,21 @@ class Oracle:
                                         C.c_int(len(rows)), _p(rows), _p(O), _p(lse))
         return O, lse
 
+    def num_shots(self) -> int:
+        return int(self.lib.moc_oracle_num_shots(C.byref(self.cfg)))
+
+    def outer_route(self, Xq, Xk, q0, q1, top_m):
+        """Outer-loop routing of the query block [q0, q1): (shot descriptors [H, S, d], scores [H, S],
+        selected shots [H, M], -1 padded)."""
+        Xq, Xk = self._u16(Xq), self._u16(Xk)
+        S = self.num_shots()
+        desc = np.empty((self.H, S, self.d), np.float64)
+        sc = np.empty((self.H, S), np.float64)
+        sel = np.empty((self.H, int(top_m)), np.int32)
+        self.lib.moc_oracle_outer_route(C.byref(self.cfg), _p(Xq), _p(Xk), C.c_int(int(q0)), C.c_int(int(q1)),
+                                        C.c_int(int(top_m)), _p(desc), _p(sc), _p(sel))
+        return desc, sc, sel
+
     def context_drop(self, sel_idx, p_max, lam, seed):
         """Context drop-off / drop-in (Sec. 3.1) applied to a copy of sel_idx.  Returns
         (edited sel_idx, n_dropped, n_drawn, n_added), the last three [H, L] int32."""

@@ -428,6 +428,61 @@ void moc_oracle_context_drop(const moc_oracle_cfg *p, int32_t *sel_idx, float p_
         }
 }
 
+
+/* ---- Appendix "Outer Loop Context Routing": a coarse pre-selection of whole shots for one query block.
+ * High-level chunk Psi_s = every token of shot s (all of its chunks, in stream order).  Per feature stream h:
+ *   phi(Psi_s) = mean of Xk over the tokens of shot s;   x_g = mean of Xq over the query block [q0, q1);
+ *   s_s = <x_g, phi(Psi_s)>;   Omega_g = the M shots of largest s_s among the shots that END before the block
+ *   begins (a shot holding a token >= q0 is the block's own present or future and is not a candidate); equal
+ *   scores go to the earlier shot; fewer than M candidates: all of them, -1 padded.
+ * shot_desc [H][S][d], scores [H][S] (every shot, unmasked), sel [H][M]; S = number of distinct shot ids. ---- */
+int moc_oracle_num_shots(const moc_oracle_cfg *p) {
+    int S = 0;
+    for (int c = 0; c < p->C; ++c)
+        if (c == 0 || p->shot[c] != p->shot[c - 1]) ++S;
+    return S;
+}
+
+void moc_oracle_outer_route(const moc_oracle_cfg *p, const uint16_t *Xq, const uint16_t *Xk, int q0, int q1, int M,
+                            double *shot_desc, double *scores, int32_t *sel) {
+    int S = moc_oracle_num_shots(p), d = p->d, L = p->L;
+    int *t0 = (int *)malloc(sizeof(int) * (size_t)S), *t1 = (int *)malloc(sizeof(int) * (size_t)S);
+    for (int c = 0, s = -1; c < p->C; ++c) {
+        if (c == 0 || p->shot[c] != p->shot[c - 1]) { ++s; t0[s] = p->off[c]; }
+        t1[s] = p->off[c + 1];
+    }
+    for (int h = 0; h < p->H; ++h) {
+        double *xg = (double *)calloc((size_t)d, sizeof(double));
+        for (int t = q0; t < q1; ++t)
+            for (int x = 0; x < d; ++x) xg[x] += bf16_to_f64(Xq[((size_t)h * L + t) * d + x]);
+        for (int x = 0; x < d; ++x) xg[x] /= (double)(q1 - q0);
+        for (int s = 0; s < S; ++s) {
+            double *f = shot_desc + ((size_t)h * S + s) * d;
+            for (int x = 0; x < d; ++x) {
+                double a = 0.0;
+                for (int t = t0[s]; t < t1[s]; ++t) a += bf16_to_f64(Xk[((size_t)h * L + t) * d + x]);
+                f[x] = a / (double)(t1[s] - t0[s]);
+            }
+            double sc = 0.0;
+            for (int x = 0; x < d; ++x) sc += xg[x] * f[x];
+            scores[(size_t)h * S + s] = sc;
+        }
+        char *avail = (char *)malloc((size_t)S);
+        for (int s = 0; s < S; ++s) avail[s] = (char)(t1[s] <= q0);
+        for (int r = 0; r < M; ++r) {
+            int best = -1;
+            for (int s = 0; s < S; ++s)
+                if (avail[s] && (best < 0 || scores[(size_t)h * S + s] > scores[(size_t)h * S + best])) best = s;
+            sel[(size_t)h * M + r] = best;
+            if (best >= 0) avail[best] = 0;
+        }
+        free(avail);
+        free(xg);
+    }
+    free(t0);
+    free(t1);
+}
+
 int moc_oracle_num_threads(void) {
     int n = 1;
 #ifdef _OPENMP

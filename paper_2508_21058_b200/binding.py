@@ -54,6 +54,12 @@ def load_library():
     lib.moc_plan_set_workspace_budget.argtypes = [vp, sz]
     lib.moc_route.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.moc_lists_from_sel.argtypes = [vp, vp, vp, vp]
+    lib.moc_outer_num_shots.argtypes = [vp, C.POINTER(C.c_int32)]
+    lib.moc_outer_route.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, vp, vp, vp, vp, vp]
+    lib.moc_outer_reduced_layout.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
+                                             vp, vp, vp, vp]
+    lib.moc_gather_tokens.argtypes = [vp, vp, vp, C.c_int32, vp, vp]
+    lib.moc_context_drop.argtypes = [vp, vp, C.c_float, C.c_float, C.c_uint64, vp, vp]
     # test hooks (exported, not in the public header)
     lib.moc_debug_use_cuda_core_attention.argtypes = [vp, i32]
     lib.moc_debug_set_wait_limit_us.argtypes = [vp, C.c_uint]
@@ -153,6 +159,9 @@ class MocPlan:
     def moc_lists_from_sel(self, sel_idx, ws):
         _check(self._lib.moc_lists_from_sel(self._h, _ptr(sel_idx), _ptr(ws), _stream()))
 
+    def moc_context_drop(self, sel_idx, p_max, lam, seed, ws):
+        _check(self._lib.moc_context_drop(self._h, _ptr(sel_idx), float(p_max), float(lam), int(seed), _ptr(ws), _stream()))
+
     def moc_attend(self, Q, K, V, sel_idx, O, lse, ws):
         _check(self._lib.moc_attend(self._h, _ptr(Q), _ptr(K), _ptr(V), _ptr(sel_idx), _ptr(O), _ptr(lse), _ptr(ws),
                                     _stream()))
@@ -170,6 +179,30 @@ class MocPlan:
         st, det = C.c_int(0), C.c_int(0)
         _check(self._lib.moc_get_status(self._h, _ptr(ws), _stream(), C.byref(st), C.byref(det)))
         return int(st.value), int(det.value)
+
+    def moc_outer_num_shots(self) -> int:
+        n = C.c_int32(0)
+        _check(self._lib.moc_outer_num_shots(self._h, C.byref(n)))
+        return int(n.value)
+
+    def moc_outer_route(self, Xq, desc, q_tok0, q_tok1, top_m, shot_desc, scores, sel_shot, ws):
+        _check(self._lib.moc_outer_route(self._h, _ptr(Xq), _ptr(desc), int(q_tok0), int(q_tok1), int(top_m), _ptr(shot_desc),
+                                         _ptr(scores), _ptr(sel_shot), _ptr(ws), _stream()))
+
+    def moc_outer_reduced_layout(self, sel_shot, q_tok0, q_tok1):
+        """Host only: (chunk_off, chunk_shot, chunk_mod, tok_map) of the reduced stream for one row of sel_shot."""
+        sel = np.ascontiguousarray(sel_shot, np.int32).reshape(-1)
+        off = np.zeros(self.C + 1, np.int32)
+        shot = np.zeros(self.C, np.int32)
+        mod = np.zeros(self.C, np.uint8)
+        tok = np.zeros(self.L, np.int32)
+        nc, nt = C.c_int32(0), C.c_int32(0)
+        _check(self._lib.moc_outer_reduced_layout(self._h, sel.ctypes.data, len(sel), int(q_tok0), int(q_tok1), C.byref(nc),
+                                                  C.byref(nt), off.ctypes.data, shot.ctypes.data, mod.ctypes.data, tok.ctypes.data))
+        return off[:nc.value + 1].copy(), shot[:nc.value].copy(), mod[:nc.value].copy(), tok[:nt.value].copy()
+
+    def moc_gather_tokens(self, X, tok_map, out):
+        _check(self._lib.moc_gather_tokens(self._h, _ptr(X), _ptr(tok_map), int(tok_map.numel()), _ptr(out), _stream()))
 
     # test hooks
     def debug_set_wait_limit_us(self, us: int):

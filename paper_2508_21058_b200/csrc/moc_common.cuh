@@ -64,6 +64,7 @@ struct moc_plan {
     std::vector<moc::WorkItem> qitems;       // anchor-pass work items of one head
     std::vector<moc::KTile> ktiles;          // key tiles of one head, chunk by chunk
     std::vector<int32_t> pool_unit_off;      // [C+1] prefix of pool units per chunk
+    std::vector<moc::KeyRange> shot_chunks;  // [S] chunk range [t0, t1) of every shot (outer-loop routing)
     int words;                               // uint32 words per anchor bitmap row
     std::vector<int32_t> cap_off;            // [C+1] start of chunk c's query list inside a head's list area
     // Routing scores only the chunks that can ever be picked: text chunks are anchors of every query, so the score
@@ -88,6 +89,7 @@ struct moc_plan {
     moc::WorkItem *d_qitems;
     moc::KeyRange *d_chunk_rng;              // [C] token range of every chunk
     moc::KTile *d_ktiles;
+    moc::KeyRange *d_shot_chunks;            // [S]
     moc::WsLayout ws;
 };
 
@@ -162,6 +164,7 @@ static inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<u
 int launch_chunk_pool(const moc_plan *p, const __nv_bfloat16 *K, float *desc, void *ws, cudaStream_t s);
 int launch_route(const moc_plan *p, const __nv_bfloat16 *Q, const float *desc, int32_t *sel, void *ws, cudaStream_t s);
 int launch_lists_from_sel(const moc_plan *p, int32_t *sel, void *ws, cudaStream_t s);
+int launch_context_drop(const moc_plan *p, int32_t *sel, float p_max, float lambda, uint64_t seed, cudaStream_t s);
 int pool_scratch_prepare(int device);     // looks up (once per device) the fixed scratch array of moc_chunk_pool_noalloc
 int launch_attend_scalar(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
                          const int32_t *sel, __nv_bfloat16 *O, float *lse, void *ws, cudaStream_t s);

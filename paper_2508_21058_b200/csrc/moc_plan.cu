@@ -195,6 +195,10 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
         if (lim[c] < 0) p->prefix_mode = 0;
         reach[c] = std::max(top, c ? reach[c - 1] : 0);
     }
+    for (int c = 0; c < C; ++c) {
+        if (c == 0 || p->shot[c] != p->shot[c - 1]) p->shot_chunks.push_back(KeyRange{c, c});
+        p->shot_chunks.back().t1 = c + 1;
+    }
     p->partials_budget = (size_t)6 << 30;
     p->wait_us = 0;
     p->cookie = plan_cookie(p);
@@ -209,6 +213,7 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
     size_t o_bits = take(4 * bits.size()), o_aoff = take(4 * (C + 1)), o_arng = take(sizeof(KeyRange) * p->anc_rng.size());
     size_t o_roff = take(4 * (C + 1)), o_ranc = take(4 * p->ranc.size()), o_qt = take(sizeof(WorkItem) * p->qitems.size());
     size_t o_puo = take(4 * (C + 1)), o_puc = take(4 * unit_chunk.size()), o_cap = take(4 * (C + 1)), o_crng = take(sizeof(KeyRange) * C), o_kt = take(sizeof(KTile) * p->ktiles.size());
+    size_t o_shots = take(sizeof(KeyRange) * p->shot_chunks.size());
     size_t o_candc = take(4 * cand_c.size()), o_lim = take(4 * C), o_reach = take(4 * C), o_colc = take(4 * std::max<size_t>(col_chunk.size(), 1));
     cudaError_t e = cudaMalloc(&p->d_blob, o);
     if (e != cudaSuccess) { set_cuda_error(e, "cudaMalloc(plan tables)"); delete p; return MOC_ERR_CUDA; }
@@ -225,7 +230,8 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
                         up(o_cap, p->cap_off.data(), 4 * (C + 1)), up(o_crng, chunk_rng.data(), sizeof(KeyRange) * C),
                         up(o_kt, p->ktiles.data(), sizeof(KTile) * p->ktiles.size()),
                         up(o_candc, cand_c.data(), 4 * cand_c.size()), up(o_lim, lim.data(), 4 * C), up(o_reach, reach.data(), 4 * C),
-                        up(o_colc, col_chunk.data(), 4 * col_chunk.size())};
+                        up(o_colc, col_chunk.data(), 4 * col_chunk.size()),
+                        up(o_shots, p->shot_chunks.data(), sizeof(KeyRange) * p->shot_chunks.size())};
     for (cudaError_t x : es)
         if (x != cudaSuccess) { set_cuda_error(x, "cudaMemcpy(plan tables)"); cudaFree(p->d_blob); delete p; return MOC_ERR_CUDA; }
     p->d_off = (int32_t *)(b + o_off); p->d_shot = (int32_t *)(b + o_shot); p->d_mod = (uint8_t *)(b + o_mod);
@@ -238,6 +244,7 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
     p->d_ktiles = (KTile *)(b + o_kt);
     p->d_cand_c = (uint32_t *)(b + o_candc); p->d_lim = (int32_t *)(b + o_lim); p->d_reach = (int32_t *)(b + o_reach);
     p->d_col_chunk = (int32_t *)(b + o_colc);
+    p->d_shot_chunks = (KeyRange *)(b + o_shots);
     *out = p;
     return MOC_OK;
 }
@@ -310,6 +317,17 @@ extern "C" int moc_lists_from_sel(const moc_plan *p, int32_t *sel_idx, void *ws,
     if (p->k > 0) { if (int r = check_dev_ptrs({sel_idx}, 4)) return r; }
     if (!ws) return MOC_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return MOC_ERR_ALIGN;
+    return launch_lists_from_sel(p, sel_idx, ws, (cudaStream_t)stream);
+}
+
+extern "C" int moc_context_drop(const moc_plan *p, int32_t *sel_idx, float p_max, float lambda, uint64_t seed, void *ws,
+                                void *stream) {
+    if (int r = enter(p)) return r;
+    if (!(p_max >= 0.f && p_max <= 1.f) || !(lambda >= 0.f && lambda <= 8.f)) return MOC_ERR_SHAPE;
+    if (p->k > 0) { if (int r = check_dev_ptrs({sel_idx}, 4)) return r; }
+    if (!ws) return MOC_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return MOC_ERR_ALIGN;
+    if (int r = launch_context_drop(p, sel_idx, p_max, lambda, seed, (cudaStream_t)stream)) return r;
     return launch_lists_from_sel(p, sel_idx, ws, (cudaStream_t)stream);
 }
 
