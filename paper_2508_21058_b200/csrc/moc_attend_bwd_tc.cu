@@ -353,13 +353,26 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                         reinterpret_cast<uint4 *>(dst)[q4] = out;
                     }
                 };
+                // the routed dQ partials use the forward's layout of routed partials: query-innermost pieces
+                constexpr int NP = D / 8;
+                const int LB = (p.L + 127) >> 7;
+                uint4 *part16 = reinterpret_cast<uint4 *>(p.part);
                 if (MODE == DQ_ROUTED) {
-                    if (qi >= 0) store_row(p.part + (((size_t)(h - p.h0) * p.L + qi) * p.k + slot) * D + ch * 32);
+                    if (qi >= 0) {
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            uint4 out;
+                            out.x = bf16x2(acc[q4 * 8 + 0], acc[q4 * 8 + 1]);
+                            out.y = bf16x2(acc[q4 * 8 + 2], acc[q4 * 8 + 3]);
+                            out.z = bf16x2(acc[q4 * 8 + 4], acc[q4 * 8 + 5]);
+                            out.w = bf16x2(acc[q4 * 8 + 6], acc[q4 * 8 + 7]);
+                            part16[part_piece(h - p.h0, LB, p.k, NP, qi, slot, ch * 4 + q4)] = out;
+                        }
+                    }
                 } else if (MODE == DQ_ANCHOR) {
                     if (qi >= 0) {
                         // the routed partials of this query, four slots requested together; a slot is in use
                         // if the forward left a finite log-sum-exp for it
-                        const uint4 *src = reinterpret_cast<const uint4 *>(p.part + ((size_t)(h - p.h0) * p.L + qi) * p.k * D + ch * 32);
                         const float *pl = p.part_lse + ((size_t)h * p.L + qi) * p.k;
                         for (int s0 = 0; s0 < p.k; s0 += 4) {
                             uint4 raw[4][4];
@@ -368,7 +381,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                                 const bool used = s0 + u < p.k && pl[s0 + u] != -INFINITY;
 #pragma unroll
                                 for (int q4 = 0; q4 < 4; ++q4)
-                                    raw[u][q4] = used ? __ldcg(src + (size_t)(s0 + u) * (D / 8) + q4) : make_uint4(0, 0, 0, 0);
+                                    raw[u][q4] = used ? __ldcg(part16 + part_piece(h - p.h0, LB, p.k, NP, qi, s0 + u, ch * 4 + q4)) : make_uint4(0, 0, 0, 0);
                             }
 #pragma unroll
                             for (int u = 0; u < 4; ++u)

@@ -1,32 +1,41 @@
-// Tensor-core sparse attention forward (tcgen05 MMA, TMEM accumulators, TMA-fed K/V).
+// Tensor-core sparse attention forward (tcgen05 MMA, TMEM accumulators, TMA-fed Q/K/V), one persistent
+// kernel over a single queue of work items.
 //
-// Two passes share one kernel:
-//   routed pass (key-chunk stationary): work item = (head, chunk c, up to 256 entries of the
-//     list of (query, slot) pairs that picked c).  The Q rows are gathered into shared
-//     memory, the keys are exactly the tokens of chunk c, and each (query, slot) gets a
-//     partial result (normalised output + log-sum-exp) in the workspace.
-//   anchor pass (query-tile stationary): work item = (head, up to 256 consecutive rows of
-//     one chunk); keys are the chunk's mandatory anchors (merged token ranges).  Its
-//     epilogue merges the row's <= k routed partials by log-sum-exp and writes O and LSE.
+// Two kinds of items:
+//   routed (key-chunk stationary): (head, chunk c, up to 256 entries of the list of (query, slot) pairs that
+//     picked c).  The Q rows are gathered by TMA (four rows per copy), the keys are exactly the tokens of chunk
+//     c, and each (query, slot) gets a partial result (normalised output + log-sum-exp) in the workspace;
+//   anchor (query-tile stationary): (head, up to 256 consecutive rows of one chunk); keys are the chunk's
+//     mandatory anchors (merged token ranges).  Its epilogue merges the row's <= k routed partials by
+//     log-sum-exp and writes O and LSE.
+// The queue holds, group of heads by group of heads, the group's routed items and then its anchor items.  One
+// CTA per SM claims items in queue order (a global counter), so the two kinds need no separate launches and no
+// CTA is set up or torn down per item: the tensor memory, the barriers and the K/V ring live for the whole
+// kernel, and the next item's Q tiles and first K/V tiles are on their way while the current item finishes.
+// What an anchor item needs from the routed items of its group (their partials) is awaited late, just before
+// its merge, on a count of completed rows; by then every routed item of the group has long been claimed, by a
+// CTA that is running, so the wait ends.  Partials of consecutive groups alternate between two buffers; a
+// routed item waits, before it stores, for the anchor items that read its buffer two groups ago.
 //
-// One CTA per SM, 12 warps in three warpgroups (the third gives most of its registers to the
-// other two), two 128-row query tiles that share every K/V tile:
-//   warps 0-3 / 4-7  softmax group of query tile 0 / 1, one row per thread (TMEM lane = row):
-//              load or gather Q into the swizzled shared tile, read S from TMEM, online
-//              softmax, write P back to TMEM as packed bf16 (aliasing S; the first 64 keys are
-//              released to the issuer before the exponentials of the other 64), lazily rescale
-//              O, epilogue.  The exponentials of the two tiles take turns;
-//   warp 8     TMA producer: K and V tiles of 128 keys, two stages each, 128-byte swizzle;
-//   warps 9, 10  one MMA-issuing thread per query tile g:  S_g(0), then  O_g += P_g V(j),
-//              S_g(j + 1)  per key tile.  The tensor pipe takes the next MMA only as the
-//              previous one retires, so an issuer that waits on a barrier idles the pipe; with
-//              one issuer per tile the other tile's MMAs fill that time, and one tile's softmax
-//              overlaps the other tile's MMAs.  S = Q K^T takes both operands from shared
-//              memory, O += P V takes P from TMEM and V as an MN-major shared-memory operand;
-//              all accumulators live in TMEM (S0, S1, O0, O1 = 512 columns);
-//   warp 11    idle (fills the third warpgroup).
-// Every mbarrier wait is bounded; a wait that runs out flags the workspace status word
-// and the CTA drains and leaves.
+// 12 warps in three warpgroups (the third gives most of its registers to the other two); an item is two 128-row
+// query tiles that share every K/V tile:
+//   warps 0-3 / 4-7  softmax group of query tile 0 / 1, one row per thread (TMEM lane = row): read S from TMEM,
+//              online softmax, write P back to TMEM as packed bf16 (aliasing S; the first 64 keys are released
+//              to the issuer before the exponentials of the other 64), lazily rescale O, epilogue.  The
+//              exponentials of the two tiles take turns;
+//   warp 8     lane 0, TMA producer: the K and V tiles of 128 keys, two stages each, 128-byte swizzle; the ring
+//              runs across items.  Lane 16, bookkeeping: waits for what an item depends on, and when the item's
+//              rows are stored adds them to the queue's count of completed rows (the one thread that pays for
+//              a device-wide fence per item);
+//   warps 9, 10  one MMA-issuing thread per query tile g:  S_g(0), then  O_g += P_g V(j),  S_g(j + 1)  per key
+//              tile.  S = Q K^T takes both operands from shared memory, O += P V takes P from TMEM and V as an
+//              MN-major shared-memory operand; all accumulators live in TMEM (S0, S1, O0, O1 = 512 columns);
+//   warp 11    scheduler and Q loader: lane 0 claims the next item and hands its description to the others
+//              through a two-slot ring; then the warp loads the item's Q tiles (plain tiles for anchor items,
+//              row gathers, four rows per lane, for routed ones) into a ring of three tile buffers, so the next
+//              item's first query tile is in place before the current item ends.
+// Every wait (mbarrier or global counter) is bounded; one that runs out flags the workspace status word and
+// the CTA drains its copies and leaves.
 #include <algorithm>
 
 #include "moc_common.cuh"
@@ -40,98 +49,148 @@ struct AttendParams {
     const __nv_bfloat16 *Q;
     __nv_bfloat16 *O;
     float *lse;
-    __nv_bfloat16 *part_o;
-    float *part_lse;
-    const KeyRange *rng;        // key ranges the items index: merged anchor ranges, or the chunks
-    const WorkItem *items;      // anchor pass: one head's items (blockIdx.y = head - h0); routed pass: every item
-    const int *item_lo_dev, *item_hi_dev;   // routed pass: the group's item range [*lo, *hi) lives on the device
-    int h0;                     // first head of the group in flight (its partials are part_o[h - h0])
-    uint32_t cookie;            // what the workspace's status area must hold
+    __nv_bfloat16 *part_o;      // [2 or 1] buffers of the group in flight's partials (even / odd groups alternate), laid
+                                // out query-innermost in blocks of 128 queries (part_piece)
+    float *part_lse;            // [H][L][k]
+    size_t part_stride;         // elements between the two partial buffers (0 with a single group)
+    const KeyRange *chunk_rng;  // [C] key range of a routed item (its chunk)
+    const KeyRange *anc_rng;    // merged anchor ranges, indexed by the anchor items
+    const WorkItem *ritems;     // routed items of every head, (head, chunk) order
+    const WorkItem *aitems;     // anchor items of one head
+    const int *tile_off;        // [H C + 1] running count of routed items over (head, chunk)
     const int32_t *qlist;       // [H][cap_total]
+    int *queue;
     size_t cap_total;
     int *status;
-    int H, L, k;
-    float scale_log2;       // softmax scale * log2(e)
+    int H, L, C, k, hg, n_groups, n_aitems;
+    float scale_log2;           // softmax scale * log2(e)
+    uint32_t cookie;
 };
 
 constexpr int kBN = 128;               // keys per tile
-constexpr int kThreads = 384;          // three warpgroups: softmax 0, softmax 1, {producer, two MMA issuers, one idle warp}
+constexpr int kThreads = 384;          // three warpgroups: softmax 0, softmax 1, {producer, two MMA issuers, scheduler}
 constexpr int kTmemCols = 512;         // S0/P0 [0,128) S1/P1 [128,256) O0 [256,384) O1 [384,512)
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr float kRescaleThreshold = 8.0f;
-   // log2 units: O is rescaled only when the row max grows by more
+constexpr float kRescaleThreshold = 8.0f;    // log2 units: O is rescaled only when the row max grows by more
 
-enum WaitCode { W_QFULL = 1, W_KFULL, W_VFULL, W_SFULL, W_PFULL, W_OFULL, W_KEMPTY, W_VEMPTY, W_TURN, W_PHALF };
+enum WaitCode { W_QFULL = 1, W_KFULL, W_VFULL, W_SFULL, W_PFULL, W_OFULL, W_KEMPTY, W_VEMPTY, W_TURN, W_PHALF,
+                W_QEMPTY, W_OFREE, W_ITEMFULL, W_ITEMEMPTY, W_ROWSDONE, W_DEPEND };
 
-template <int D, bool ROUTED>
-__global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+// One claimed item, as the scheduler hands it over.
+struct ItemSlot {
+    int valid;          // 0: the queue is empty, everyone leaves
+    int routed, h, first, rows, nrng, ntiles, phase;
+    const KeyRange *rng;
+};
+
+// Queue bookkeeping in the workspace (kQueueHeader ints, then three per phase: first item, rows that must
+// complete, rows completed), written before the persistent kernel starts.  Phase 2 g is the routed items of head
+// group g (rows = the group's list entries), phase 2 g + 1 its anchor items (rows = its query rows).  One block.
+__global__ void attend_queue_kernel(int *__restrict__ queue, const int *__restrict__ tile_off, const int *__restrict__ cnt,
+                                    const int *__restrict__ status, uint32_t cookie, int H, int L, int C, int k, int hg, int n_groups,
+                                    int n_aitems) {
+    __shared__ int red[256];
+    const bool routed_ok = status[ST_STATUS] == 0 && (uint32_t)status[ST_COOKIE] == cookie;     // else nothing may be read
+    int first = 0;
+    for (int g = 0; g < n_groups; ++g) {
+        const int h0 = g * hg, h1 = min(H, h0 + hg);
+        int entries = 0;
+        if (routed_ok && k > 0)
+            for (int x = h0 * C + threadIdx.x; x < h1 * C; x += blockDim.x) entries += cnt[x];
+        red[threadIdx.x] = entries;
+        __syncthreads();
+        for (int o = 128; o > 0; o >>= 1) {
+            if ((int)threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) {
+            const int n_r = (routed_ok && k > 0) ? tile_off[h1 * C] - tile_off[h0 * C] : 0;
+            int *ph = queue + kQueueHeader + 3 * (2 * g);
+            ph[0] = first; ph[1] = red[0]; ph[2] = 0;
+            first += n_r;
+            ph[3] = first; ph[4] = (h1 - h0) * L; ph[5] = 0;
+            first += (h1 - h0) * n_aitems;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) { queue[0] = 0; queue[1] = routed_ok ? first : 0; queue[2] = 2 * n_groups; queue[3] = 0; }
+}
+
+// a bounded wait on a counter in global memory (another CTA adds to it)
+__device__ __forceinline__ bool wait_count(const int *ctr, int need, volatile int *abort_flag, int *status, int code) {
+    if (*(volatile const int *)ctr >= need) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (*(volatile const int *)ctr >= need) return true;
+        __nanosleep(200);
+        if ((it & 0x3f) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > wait_limit_ns(status)) {
+                *abort_flag = 1;
+                if (atomicCAS(status, 0, MOC_ERR_TIMEOUT) == 0) status[ST_DETAIL] = code;
+                return false;
+            }
+        }
+    }
+}
+
+// four rows of a 2-D tensor, 64 columns from column x on, into four consecutive 128-byte rows of shared memory
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap *map, int x, int r0, int r1, int r2, int r3, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
+                 : "memory");
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
+                                                                const __grid_constant__ CUtensorMap tmQrow,
+                                                                const __grid_constant__ CUtensorMap tmK,
                                                                 const __grid_constant__ CUtensorMap tmV,
                                                                 const AttendParams p) {
     constexpr int TILE_BYTES = 128 * D * 2;
     constexpr int SUB = D / 64;            // 64-column (128-byte) sub-tiles per row
     constexpr int SUB_BYTES = 128 * 128;   // one sub-tile: 128 rows of 128 bytes
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[20];
+    __shared__ __align__(8) uint64_t bars[36];
     __shared__ uint32_t tmem_slot;
     __shared__ int s_abort;
-    __shared__ int w_valid, w_h, w_rows, w_first, w_nrng, w_ntiles;
-    __shared__ int s_qrow[kQTileRows];              // query row behind each row of the item (-1 = padding)
-    __shared__ const KeyRange *w_rng;
+    __shared__ ItemSlot s_item[2];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t *gbase = smem_raw + (sbase - smem_u32(smem_raw));
-    // shared tiles: Q0 Q1 | K stage 0,1 | V stage 0,1
-    const uint32_t sQ = sbase, sK = sbase + 2 * TILE_BYTES, sV = sbase + 4 * TILE_BYTES;
+    // shared tiles: Q ring of three | K stage 0,1 | V stage 0,1
+    const uint32_t sQ = sbase, sK = sbase + 3 * TILE_BYTES, sV = sbase + 5 * TILE_BYTES;
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
-    // barrier indices
-    constexpr int Q_FULL = 0, K_FULL = 2, K_EMPTY = 4, V_FULL = 6, V_EMPTY = 8, S_FULL = 10, P_FULL = 12, O_FULL = 14, TURN = 16, P_HALF = 18;
+    // barrier indices (pairs: per query tile g, per K/V stage, or per item slot)
+    constexpr int Q_FULL = 0, Q_EMPTY = 3, K_FULL = 6, K_EMPTY = 8, V_FULL = 10, V_EMPTY = 12, S_FULL = 14, P_HALF = 16, P_FULL = 18,
+                  O_FULL = 20, O_FREE = 22, TURN = 24, ITEM_FULL = 26, ITEM_EMPTY = 28, ROWS_DONE = 30, DEPEND = 32;
+    constexpr int kItemReaders = 2 + 2 + 256;          // producer and bookkeeping lanes, two issuers, every softmax thread
 
     if (threadIdx.x == 0) {
         s_abort = 0;
-        int valid = (*(volatile int *)p.status == 0);
-        if (valid && (uint32_t)((volatile int *)p.status)[ST_COOKIE] != p.cookie) {
-            // the workspace does not hold this plan's lists: report, touch nothing else
-            atomicCAS(p.status, 0, MOC_ERR_WORKSPACE);
-            valid = 0;
+        for (int t = 0; t < 3; ++t) {
+            mbar_init(bar(Q_FULL + t), 1);
+            mbar_init(bar(Q_EMPTY + t), 1);
         }
-        int item = blockIdx.x;
-        if (ROUTED && valid) {
-            item += *p.item_lo_dev;
-            if (item >= *p.item_hi_dev) valid = 0;
-        }
-        WorkItem w = {};
-        if (valid) {
-            w = p.items[item];
-            if (ROUTED && !index_ok((unsigned)w.h < (unsigned)p.H && w.rows > 0 && w.rows <= kQTileRows && w.first >= 0 &&
-                                    (size_t)w.first + w.rows <= p.cap_total && w.nrng == 1, p.status, IX_ITEM_FIELDS))
-                valid = 0;
-        }
-        if (valid) {
-            w_h = ROUTED ? w.h : p.h0 + (int)blockIdx.y;
-            w_first = w.first;
-            w_rows = w.rows;
-            w_rng = p.rng + w.rng_off;
-            w_nrng = w.nrng;
-            w_ntiles = w.ntiles;
-        }
-        w_valid = valid;
+        mbar_init(bar(DEPEND), 1);
         for (int t = 0; t < 2; ++t) {
-            mbar_init(bar(Q_FULL + t), 128);
             mbar_init(bar(K_FULL + t), 1);
-            mbar_init(bar(K_EMPTY + t), valid && w_rows > 128 ? 2 : 1);   // one commit per MMA issuer
+            mbar_init(bar(K_EMPTY + t), 2);            // one arrival per MMA issuer
             mbar_init(bar(V_FULL + t), 1);
-            mbar_init(bar(V_EMPTY + t), valid && w_rows > 128 ? 2 : 1);
+            mbar_init(bar(V_EMPTY + t), 2);
             mbar_init(bar(S_FULL + t), 1);
+            mbar_init(bar(P_HALF + t), 128);
             mbar_init(bar(P_FULL + t), 128);
             mbar_init(bar(O_FULL + t), 1);
+            mbar_init(bar(O_FREE + t), 128);
             mbar_init(bar(TURN + t), 128);
-            mbar_init(bar(P_HALF + t), 128);
+            mbar_init(bar(ITEM_FULL + t), 1);
+            mbar_init(bar(ITEM_EMPTY + t), kItemReaders);
+            mbar_init(bar(ROWS_DONE + t), 128);
         }
         fence_barrier_init();
     }
     __syncthreads();
-    if (!w_valid) return;
     if (warp == 8) {
         tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
         tmem_relinquish();
@@ -139,11 +198,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-
     const uint32_t tmem = tmem_slot;
-    const int h = w_h, rows = w_rows, first = w_first, n_tiles = w_ntiles;
-    const bool two = rows > 128;            // is query tile 1 populated?
     volatile int *abort_flag = &s_abort;
+    int *phase_tab = p.queue + kQueueHeader;
 
     if (warp < 8) {
         // ------------------------------------------------------------ softmax / epilogue groups
@@ -154,55 +211,58 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
         const int r = threadIdx.x & 127;               // row within the tile = TMEM lane
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + g * 128 + lane_off, tP = tS, tO = tmem + 256 + g * 128 + lane_off;
-        if (g == 0 || two) {
-            const int rt = g * 128 + r;                // row within the work item
+        const float c = p.scale_log2;
+        // running counts that give every barrier's phase: items seen, items this group worked on, key tiles it
+        // processed, key tiles processed in two-tile items (the turn-taking of the exponentials)
+        int n_item = 0, n_mine = 0, n_s = 0, n_turn = 0;
+        bool ok = true;
+        while (ok) {
+            const int sl = n_item & 1;
+            ok = mbar_wait(bar(ITEM_FULL + sl), (n_item >> 1) & 1, abort_flag, p.status, W_ITEMFULL);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const ItemSlot it_ = s_item[sl];
+            mbar_arrive(bar(ITEM_EMPTY + sl));
+            ++n_item;
+            if (!it_.valid) break;
+            const int h = it_.h, rows = it_.rows, first = it_.first, group = it_.phase >> 1;
+            const bool routed = it_.routed != 0, two = rows > 128;
+            if (g == 1 && !two) continue;               // this item has one query tile
+            const int rt = g * 128 + r;                 // row within the work item
             int qi = -1, slot = 0;
             if (rt < rows) {
-                if (ROUTED) {
-                    const int e = p.qlist[(size_t)h * p.cap_total + first + rt];
+                if (routed) {
+                    const bool at_ok = index_ok((size_t)first + rt < p.cap_total, p.status, IX_LIST_POSITION);
+                    const int e = at_ok ? p.qlist[(size_t)h * p.cap_total + first + rt] : -1;
                     qi = e / p.k;
                     slot = e - qi * p.k;
                     (void)index_ok(e >= 0 && qi < p.L, p.status, IX_LIST_ENTRY);
-                    if ((unsigned)qi >= (unsigned)p.L) qi = -1;      // never follow an entry that is not a row of this head
+                    if (e < 0 || qi >= p.L) qi = -1;         // never follow an entry that is not a row of this head
                 } else {
                     qi = first + rt;
                 }
             }
-            {
-                // The group stages its Q tile together: consecutive threads take consecutive 16-byte pieces
-                // of a row, so every request covers whole 128-byte lines even when the rows are gathered.
-                s_qrow[g * 128 + r] = qi;
-                asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory");     // the group's 128 threads; nothing can have failed yet
-                constexpr int CH = D / 8, RP = 128 / CH;       // pieces per row, rows per pass
-                const int c16 = r % CH;
-                uint8_t *dstq = gbase + g * TILE_BYTES + (c16 >> 3) * SUB_BYTES;
-                uint4 v[CH];
-#pragma unroll
-                for (int ps = 0; ps < CH; ++ps) {
-                    const int rr = ps * RP + r / CH, q = s_qrow[g * 128 + rr];
-                    v[ps] = make_uint4(0, 0, 0, 0);
-                    if (q >= 0) v[ps] = __ldg(reinterpret_cast<const uint4 *>(p.Q + ((size_t)h * p.L + q) * D) + c16);
-                }
-#pragma unroll
-                for (int ps = 0; ps < CH; ++ps)
-                    *reinterpret_cast<uint4 *>(dstq + sw128_offset(ps * RP + r / CH, c16 & 7)) = v[ps];
-            }
-            fence_proxy_async_smem();
-            mbar_arrive(bar(Q_FULL + g));
-            if (!ROUTED && qi >= 0) {
-                // the epilogue will merge this row's routed partials: start them on their way into L2 now
-                const char *po = reinterpret_cast<const char *>(p.part_o + ((size_t)(h - p.h0) * p.L + qi) * p.k * D);
-                for (int b = 0; b < p.k * D * 2; b += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(po + b));
+            // partials of the group in flight: even and odd groups alternate between two buffers
+            __nv_bfloat16 *part_o = p.part_o + (size_t)(group & 1) * p.part_stride;
+            const int h_loc = h - group * p.hg;
+            constexpr int NP = D / 8;                   // 16-byte pieces per row
+            const int LB = (p.L + 127) >> 7;
+            uint4 *part16 = reinterpret_cast<uint4 *>(part_o);
+            if (!routed && qi >= 0 && p.k > 0) {
+                // the epilogue will merge this row's routed partials: start them on their way into L2 now.  A 128-byte
+                // line holds one piece of eight consecutive queries: every eighth query (and the tile's first) asks
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(p.part_lse + ((size_t)h * p.L + qi) * p.k));
+                if ((qi & 7) == 0 || r == 0)
+                    for (int s = 0; s < p.k; ++s)
+                        for (int cc = 0; cc < NP; ++cc)
+                            asm volatile("prefetch.global.L2 [%0];" ::"l"(part16 + part_piece(h_loc, LB, p.k, NP, qi, s, cc)));
             }
 
             float m_run = -INFINITY, l_run = 0.f;
-            const float c = p.scale_log2;
-            TileIter it(w_rng, w_nrng);
+            TileIter it(it_.rng, it_.nrng);
             int t0, valid, jt = 0;
-            bool ok = true;
             while (it.next(t0, valid)) {
-                ok = mbar_wait(bar(S_FULL + g), jt & 1, abort_flag, p.status, W_SFULL);
+                ok = mbar_wait(bar(S_FULL + g), n_s & 1, abort_flag, p.status, W_SFULL);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
@@ -235,9 +295,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 // The exponentials of the two query tiles take turns (tile 0 of key tile j, tile 1
                 // of j, tile 0 of j + 1, ...): each then has the arithmetic pipes to itself while
                 // the other tile's MMAs run, instead of both drifting into lock step.
-                // TURN + g is arrived on by group g when its exponentials of a key tile are done.
-                if (two && (g == 1 || jt > 0)) {
-                    ok = mbar_wait(bar(TURN + (g ^ 1)), (g == 1 ? jt : jt - 1) & 1, abort_flag, p.status, W_TURN);
+                // TURN + g is arrived on by group g when its exponentials of a key tile are done.  (Tile 0 waits for
+                // tile 1's previous turn even at the start of an item: the barrier must never get two phases ahead of
+                // a group that has yet to wait on it.)
+                if (two && (g == 1 || n_turn > 0)) {
+                    ok = mbar_wait(bar(TURN + (g ^ 1)), (g == 1 ? n_turn : n_turn - 1) & 1, abort_flag, p.status, W_TURN);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                 }
@@ -286,7 +348,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 unpack2(add2(sum_a, sum_b), s0, s1);
                 l_run = l_run * alpha + (s0 + s1);
                 ++jt;
+                ++n_s;
+                if (two) ++n_turn;
             }
+            if (!ok) break;
             // ---- epilogue
             // The merge weights of the routed partials depend only on log-sum-exps: have them ready before
             // the last P V lands.  wslot[s] = exp(lse_s - lse_total), w_own likewise for this pass's own part.
@@ -298,14 +363,18 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
 #pragma unroll
             for (int s = 0; s < KW; ++s) wslot[s] = 0.f;
             const float *pl = nullptr;
-            const __nv_bfloat16 *po = nullptr;
-            if (!ROUTED && ok && qi >= 0 && p.k > 0) {
+            // what this item depends on (an anchor item: the routed items of its group have stored all their partials;
+            // a routed item: the anchor items two groups back have read the buffer it is about to store into) has been
+            // awaited by the bookkeeping lane, which then arrives on DEPEND, once per item
+            ok = mbar_wait(bar(DEPEND), (n_item - 1) & 1, abort_flag, p.status, W_DEPEND);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (!routed && qi >= 0 && p.k > 0) {
                 pl = p.part_lse + ((size_t)h * p.L + qi) * p.k;
-                po = p.part_o + ((size_t)(h - p.h0) * p.L + qi) * p.k * D;
                 if (p.k <= KW) {
                     float plv[KW];
 #pragma unroll
-                    for (int s = 0; s < KW; ++s) plv[s] = s < p.k ? pl[s] : -INFINITY;
+                    for (int s = 0; s < KW; ++s) plv[s] = s < p.k ? __ldcg(pl + s) : -INFINITY;
 #pragma unroll
                     for (int s = 0; s < KW; ++s) big = fmaxf(big, plv[s]);
                     wsum = __expf(lse_own - big);
@@ -314,65 +383,49 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
 #pragma unroll
                     for (int s = 0; s < KW; ++s) wslot[s] /= wsum;
                 } else {
-                    for (int s = 0; s < p.k; ++s) big = fmaxf(big, pl[s]);
+                    for (int s = 0; s < p.k; ++s) big = fmaxf(big, __ldcg(pl + s));
                     wsum = __expf(lse_own - big);
-                    for (int s = 0; s < p.k; ++s) wsum += __expf(pl[s] - big);
+                    for (int s = 0; s < p.k; ++s) wsum += __expf(__ldcg(pl + s) - big);
                 }
                 w_own = __expf(lse_own - big) / wsum * inv_l;
             }
-            if (ok) {
-                ok = mbar_wait(bar(O_FULL + g), 0, abort_flag, p.status, W_OFULL);
-                ok = __all_sync(0xffffffffu, ok);
-            }
-            if (ok) {
-                tc_fence_after();
+            ok = mbar_wait(bar(O_FULL + g), n_mine & 1, abort_flag, p.status, W_OFULL);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
 #pragma unroll 1
-                for (int ch = 0; ch < D / 32; ++ch) {
-                    uint32_t v[32];
-                    __syncwarp();
-                    tmem_ld32(tO + ch * 32, v);
-                    tmem_wait_ld();
-                    float acc[32];
+            for (int ch = 0; ch < D / 32; ++ch) {
+                uint32_t v[32];
+                __syncwarp();
+                tmem_ld32(tO + ch * 32, v);
+                tmem_wait_ld();
+                if (ch == D / 32 - 1) {
+                    // O has been read: the issuer may start the next item's P V (which overwrites it)
+                    tc_fence_before();
+                    mbar_arrive(bar(O_FREE + g));
+                }
+                float acc[32];
 #pragma unroll
-                    for (int x = 0; x < 32; ++x) acc[x] = __uint_as_float(v[x]) * w_own;
-                    if (pl && p.k <= KW) {
-                        // four slots' pieces of this column block are requested together: one round trip, not four
+                for (int x = 0; x < 32; ++x) acc[x] = __uint_as_float(v[x]) * w_own;
+                if (pl && p.k <= KW) {
+                    // four slots' pieces of this column block are requested together: one round trip, not four
 #pragma unroll
-                        for (int s0 = 0; s0 < KW; s0 += 4) {
-                            if (s0 >= p.k) break;
-                            uint4 raw[4][4];
+                    for (int s0 = 0; s0 < KW; s0 += 4) {
+                        if (s0 >= p.k) break;
+                        uint4 raw[4][4];
 #pragma unroll
-                            for (int s = 0; s < 4; ++s)
+                        for (int s = 0; s < 4; ++s)
 #pragma unroll
-                                for (int q4 = 0; q4 < 4; ++q4)
-                                    raw[s][q4] = (s0 + s < p.k && wslot[s0 + s] != 0.f)
-                                                     ? __ldcg(reinterpret_cast<const uint4 *>(po + (size_t)(s0 + s) * D + ch * 32) + q4)
-                                                     : make_uint4(0, 0, 0, 0);
+                            for (int q4 = 0; q4 < 4; ++q4)
+                                raw[s][q4] = (s0 + s < p.k && wslot[s0 + s] != 0.f)
+                                                 ? __ldcg(part16 + part_piece(h_loc, LB, p.k, NP, qi, s0 + s, ch * 4 + q4))
+                                                 : make_uint4(0, 0, 0, 0);
 #pragma unroll
-                            for (int s = 0; s < 4; ++s) {
-                                const float w = wslot[s0 + s];
-#pragma unroll
-                                for (int q4 = 0; q4 < 4; ++q4) {
-                                    const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&raw[s][q4]);
-#pragma unroll
-                                    for (int y = 0; y < 4; ++y) {
-                                        const float2 f = __bfloat1622float2(b[y]);
-                                        acc[q4 * 8 + 2 * y] = fmaf(w, f.x, acc[q4 * 8 + 2 * y]);
-                                        acc[q4 * 8 + 2 * y + 1] = fmaf(w, f.y, acc[q4 * 8 + 2 * y + 1]);
-                                    }
-                                }
-                            }
-                        }
-                    } else if (pl) {
-                        for (int s = 0; s < p.k; ++s) {
-                            const float ls = pl[s];
-                            if (ls == -INFINITY) continue;
-                            const float w = __expf(ls - big) / wsum;
-                            const uint4 *src = reinterpret_cast<const uint4 *>(po + (size_t)s * D + ch * 32);
+                        for (int s = 0; s < 4; ++s) {
+                            const float w = wslot[s0 + s];
 #pragma unroll
                             for (int q4 = 0; q4 < 4; ++q4) {
-                                const uint4 raw = __ldcg(src + q4);
-                                const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+                                const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&raw[s][q4]);
 #pragma unroll
                                 for (int y = 0; y < 4; ++y) {
                                     const float2 f = __bfloat1622float2(b[y]);
@@ -382,52 +435,84 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                             }
                         }
                     }
-                    if (qi < 0) continue;
-                    __nv_bfloat16 *dst = ROUTED ? p.part_o + (((size_t)(h - p.h0) * p.L + qi) * p.k + slot) * D + ch * 32
-                                                : p.O + ((size_t)h * p.L + qi) * D + ch * 32;
+                } else if (pl) {
+                    for (int s = 0; s < p.k; ++s) {
+                        const float ls = __ldcg(pl + s);
+                        if (ls == -INFINITY) continue;
+                        const float w = __expf(ls - big) / wsum;
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        uint4 out;
-                        uint32_t *o32 = reinterpret_cast<uint32_t *>(&out);
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            const uint4 raw = __ldcg(part16 + part_piece(h_loc, LB, p.k, NP, qi, s, ch * 4 + q4));
+                            const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&raw);
 #pragma unroll
-                        for (int y = 0; y < 4; ++y) {
-                            __nv_bfloat162 b = __floats2bfloat162_rn(acc[q4 * 8 + 2 * y], acc[q4 * 8 + 2 * y + 1]);
-                            o32[y] = *reinterpret_cast<uint32_t *>(&b);
+                            for (int y = 0; y < 4; ++y) {
+                                const float2 f = __bfloat1622float2(b[y]);
+                                acc[q4 * 8 + 2 * y] = fmaf(w, f.x, acc[q4 * 8 + 2 * y]);
+                                acc[q4 * 8 + 2 * y + 1] = fmaf(w, f.y, acc[q4 * 8 + 2 * y + 1]);
+                            }
                         }
-                        reinterpret_cast<uint4 *>(dst)[q4] = out;
                     }
                 }
-                if (qi >= 0) {
-                    if (ROUTED) p.part_lse[((size_t)h * p.L + qi) * p.k + slot] = lse_own;
-                    else p.lse[(size_t)h * p.L + qi] = (pl ? big + __logf(wsum) : lse_own);
+                if (qi < 0) continue;
+                uint4 *dst_row = reinterpret_cast<uint4 *>(p.O + ((size_t)h * p.L + qi) * D + ch * 32);
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    uint4 out;
+                    uint32_t *o32 = reinterpret_cast<uint32_t *>(&out);
+#pragma unroll
+                    for (int y = 0; y < 4; ++y) {
+                        __nv_bfloat162 b = __floats2bfloat162_rn(acc[q4 * 8 + 2 * y], acc[q4 * 8 + 2 * y + 1]);
+                        o32[y] = *reinterpret_cast<uint32_t *>(&b);
+                    }
+                    if (routed) part16[part_piece(h_loc, LB, p.k, NP, qi, slot, ch * 4 + q4)] = out;
+                    else dst_row[q4] = out;
                 }
             }
+            if (qi >= 0) {
+                if (routed) p.part_lse[((size_t)h * p.L + qi) * p.k + slot] = lse_own;
+                else p.lse[(size_t)h * p.L + qi] = (pl ? big + __logf(wsum) : lse_own);
+            }
+            // this tile's rows are stored; the bookkeeping lane counts them once all 128 threads are here
+            mbar_arrive(bar(ROWS_DONE + g));
+            ++n_mine;
         }
     } else if (warp == 8) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-        // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
+            // ------------------------------------------------------------ TMA producer of the K and V tiles
             prefetch_tensormap(&tmK);
             prefetch_tensormap(&tmV);
-            TileIter it(w_rng, w_nrng);
-            int t0, valid, jt = 0;
-            int k_last = -1, v_last = -1;   // last tile whose K / V copy was issued
-            while (it.next(t0, valid)) {
-                const int st = jt & 1;
-                const uint32_t ph = (jt >> 1) & 1;
-                if (!mbar_wait(bar(K_EMPTY + st), ph ^ 1, abort_flag, p.status, W_KEMPTY)) break;
-                mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
+            int n_item = 0, n_kv = 0;                         // items seen, K/V tiles issued
+            int k_last = -1, v_last = -1;                     // last tile whose K / V copy was issued
+            bool ok = true;
+            while (ok) {
+                const int sl = n_item & 1;
+                if (!mbar_wait(bar(ITEM_FULL + sl), (n_item >> 1) & 1, abort_flag, p.status, W_ITEMFULL)) break;
+                const ItemSlot it_ = s_item[sl];
+                mbar_arrive(bar(ITEM_EMPTY + sl));
+                ++n_item;
+                if (!it_.valid) break;
+                const int h = it_.h;
+                // the ring of stages runs on from the previous item
+                TileIter it(it_.rng, it_.nrng);
+                int t0, valid;
+                while (it.next(t0, valid)) {
+                    const int st = n_kv & 1;
+                    const uint32_t ph = (n_kv >> 1) & 1;
+                    if (!mbar_wait(bar(K_EMPTY + st), ph ^ 1, abort_flag, p.status, W_KEMPTY)) { ok = false; break; }
+                    mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
 #pragma unroll
-                for (int sub = 0; sub < SUB; ++sub)
-                    tma_load_2d(sK + st * TILE_BYTES + sub * SUB_BYTES, &tmK, sub * 64, h * p.L + t0, bar(K_FULL + st));
-                k_last = jt;
-                if (!mbar_wait(bar(V_EMPTY + st), ph ^ 1, abort_flag, p.status, W_VEMPTY)) break;
-                mbar_expect_tx(bar(V_FULL + st), TILE_BYTES);
+                    for (int sub = 0; sub < SUB; ++sub)
+                        tma_load_2d(sK + st * TILE_BYTES + sub * SUB_BYTES, &tmK, sub * 64, h * p.L + t0, bar(K_FULL + st));
+                    k_last = n_kv;
+                    if (!mbar_wait(bar(V_EMPTY + st), ph ^ 1, abort_flag, p.status, W_VEMPTY)) { ok = false; break; }
+                    mbar_expect_tx(bar(V_FULL + st), TILE_BYTES);
 #pragma unroll
-                for (int sub = 0; sub < SUB; ++sub)
-                    tma_load_2d(sV + st * TILE_BYTES + sub * SUB_BYTES, &tmV, sub * 64, h * p.L + t0, bar(V_FULL + st));
-                v_last = jt;
-                ++jt;
+                    for (int sub = 0; sub < SUB; ++sub)
+                        tma_load_2d(sV + st * TILE_BYTES + sub * SUB_BYTES, &tmV, sub * 64, h * p.L + t0, bar(V_FULL + st));
+                    v_last = n_kv;
+                    ++n_kv;
+                }
             }
             if (*abort_flag) {
                 // drain: copies already issued must land before the CTA's shared memory is released
@@ -438,12 +523,45 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                     if (vj >= 0) mbar_wait(bar(V_FULL + (vj & 1)), (vj >> 1) & 1, &dummy_flag, p.status, W_VFULL);
                 }
             }
+        } else if (lane == 16) {
+            // ------------------------------------------------------------ bookkeeping, item by item:
+            // first what the item depends on - an anchor item: the routed items of its group have stored all their
+            // partials; a routed item: the anchor items two groups back have read the buffer it will store into -
+            // then, when the softmax groups have stored the item's rows, the rows join the phase's count.  The
+            // groups' arrivals order their stores before this thread (CTA scope); its fence makes them visible
+            // device-wide before the count moves.
+            int n_item = 0, n_tile[2] = {0, 0};
+            bool ok = true;
+            while (ok) {
+                const int sl = n_item & 1;
+                if (!mbar_wait(bar(ITEM_FULL + sl), (n_item >> 1) & 1, abort_flag, p.status, W_ITEMFULL)) break;
+                const ItemSlot it_ = s_item[sl];
+                mbar_arrive(bar(ITEM_EMPTY + sl));
+                ++n_item;
+                if (!it_.valid) break;
+                const int group = it_.phase >> 1;
+                if (!it_.routed && p.k > 0)
+                    ok = wait_count(&phase_tab[3 * (2 * group) + 2], phase_tab[3 * (2 * group) + 1], abort_flag, p.status, W_DEPEND);
+                if (it_.routed && group >= 2)
+                    ok = wait_count(&phase_tab[3 * (2 * (group - 2) + 1) + 2], phase_tab[3 * (2 * (group - 2) + 1) + 1], abort_flag, p.status, W_DEPEND);
+                if (!ok) break;
+                __threadfence();
+                mbar_arrive(bar(DEPEND));
+                const int n_qt = it_.rows > 128 ? 2 : 1;
+                for (int g = 0; ok && g < n_qt; ++g) {
+                    ok = mbar_wait(bar(ROWS_DONE + g), n_tile[g] & 1, abort_flag, p.status, W_ROWSDONE);
+                    ++n_tile[g];
+                }
+                if (!ok) break;
+                __threadfence();
+                atomicAdd(&phase_tab[3 * it_.phase + 2], it_.rows);
+            }
         }
-    } else {
+    } else if (warp < 11) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-        // ------------------------------------------------------------ MMA issuers (one per query tile); warp 11 idles
+        // ------------------------------------------------------------ MMA issuers (one per query tile)
         const int g = warp - 9;
-        if (lane == 0 && g < 2 && (g == 0 || two)) {
+        if (lane == 0) {
             constexpr uint32_t IDESC_PV = idesc_bf16_f32(128, D, 0, 1);
             // Descriptors are built once; inside the issue loops only the 14-bit start-address field
             // (low word, 16-byte units) moves, so one tcgen05.mma costs the issuing thread a few
@@ -451,10 +569,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             const uint64_t q_desc0 = smem_desc_sw128(sQ, 16, 1024), k_desc0 = smem_desc_sw128(sK, 16, 1024);
             const uint64_t v_desc0 = smem_desc_sw128(sV, SUB_BYTES, 1024);
             constexpr uint64_t STAGE = TILE_BYTES >> 4;   // next tile / next stage, in address-field units
-            auto issue_qk = [&](int g, int st, int valid) {
+            int qb = 0;                                   // Q buffer of this tile in the current item
+            auto issue_qk = [&](int st, int valid) {
                 const int n_qk = max(16, (valid + 15) & ~15);
                 const uint32_t idesc_qk = idesc_bf16_f32(128, n_qk, 0, 0);
-                const uint64_t qd = q_desc0 + (g ? STAGE : 0), kd = k_desc0 + (st ? STAGE : 0);
+                const uint64_t qd = q_desc0 + qb * STAGE, kd = k_desc0 + (st ? STAGE : 0);
                 const uint32_t q_lo = (uint32_t)qd, q_hi = (uint32_t)(qd >> 32), k_lo = (uint32_t)kd, k_hi = (uint32_t)(kd >> 32);
                 const uint32_t d_s = tmem + g * 128;
 #pragma unroll
@@ -464,7 +583,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 }
             };
             // k-steps [ks0, ks1) of  O_g += P_g V(stage st)  (16 keys each)
-            auto issue_pv = [&](int g, int st, int ks0, int ks1, bool accumulate) {
+            auto issue_pv = [&](int st, int ks0, int ks1, bool accumulate) {
                 const uint64_t vd = v_desc0 + (st ? STAGE : 0);
                 const uint32_t v_lo = (uint32_t)vd, v_hi = (uint32_t)(vd >> 32);
                 const uint32_t d_o = tmem + 256 + g * 128, a_p = tmem + g * 128;
@@ -476,42 +595,176 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                     for (int ks = ks0; ks < ks1; ++ks) mma_ts_lo(d_o, a_p + ks * 8, v_lo + ks * (2048 >> 4), v_hi, IDESC_PV, accumulate || ks > ks0);
                 }
             };
-            // this issuer serves query tile g: S_g(0), then per key tile  O_g += P_g V(j),  S_g(j + 1)
-            TileIter it(w_rng, w_nrng);
-            int t0, valid, valid_next = 0;
-            bool ok = it.next(t0, valid);
-            ok = ok && mbar_wait(bar(Q_FULL + g), 0, abort_flag, p.status, W_QFULL);
-            ok = ok && mbar_wait(bar(K_FULL + 0), 0, abort_flag, p.status, W_KFULL);
-            if (ok) {
-                tc_fence_after();
-                issue_qk(g, 0, valid);
-                tc_commit(bar(S_FULL + g));
-                tc_commit(bar(K_EMPTY + 0));
-            }
-            for (int jt = 0; ok && jt < n_tiles; ++jt) {
-                const int st = jt & 1, sn = (jt + 1) & 1;
-                const uint32_t ph = (jt >> 1) & 1, phn = ((jt + 1) >> 1) & 1;
-                const bool more = it.next(t0, valid_next);
-                if (!mbar_wait(bar(V_FULL + st), ph, abort_flag, p.status, W_VFULL)) break;
-                if (more && !mbar_wait(bar(K_FULL + sn), phn, abort_flag, p.status, W_KFULL)) break;
-                const int steps = (valid + 15) >> 4, half = min(steps, 4);
-                if (!mbar_wait(bar(P_HALF + g), jt & 1, abort_flag, p.status, W_PHALF)) break;
-                tc_fence_after();
-                issue_pv(g, st, 0, half, jt > 0);
-                if (!mbar_wait(bar(P_FULL + g), jt & 1, abort_flag, p.status, W_PFULL)) break;
-                tc_fence_after();
-                if (steps > half) issue_pv(g, st, half, steps, true);
-                // a commit between two groups of MMAs leaves the pipe idle: the next S goes out first, then all commits
-                if (more) {
-                    issue_qk(g, sn, valid_next);
-                    tc_commit(bar(S_FULL + g));
-                    tc_commit(bar(V_EMPTY + st));
-                    tc_commit(bar(K_EMPTY + sn));
-                } else {
-                    tc_commit(bar(V_EMPTY + st));
-                    tc_commit(bar(O_FULL + g));
+            // items seen, items with this tile, K/V tiles seen, P tiles consumed, query tiles loaded before this item
+            int n_item = 0, n_mine = 0, n_kv = 0, n_p = 0, n_qtile = 0;
+            bool ok = true;
+            while (ok) {
+                const int sl = n_item & 1;
+                if (!mbar_wait(bar(ITEM_FULL + sl), (n_item >> 1) & 1, abort_flag, p.status, W_ITEMFULL)) break;
+                const ItemSlot it_ = s_item[sl];
+                mbar_arrive(bar(ITEM_EMPTY + sl));
+                ++n_item;
+                if (!it_.valid) break;
+                const int n_tiles = it_.ntiles;
+                const int q_seq = n_qtile + g;                      // this tile's place in the sequence of Q loads
+                n_qtile += it_.rows > 128 ? 2 : 1;
+                if (g == 1 && it_.rows <= 128) {
+                    // no second query tile: this issuer only keeps the K/V ring's accounting (each stage is
+                    // released by two arrivals)
+                    for (int jt = 0; ok && jt < n_tiles; ++jt) {
+                        const int st = n_kv & 1;
+                        const uint32_t ph = (n_kv >> 1) & 1;
+                        ok = mbar_wait(bar(K_FULL + st), ph, abort_flag, p.status, W_KFULL) &&
+                             mbar_wait(bar(V_FULL + st), ph, abort_flag, p.status, W_VFULL);
+                        if (!ok) break;
+                        mbar_arrive(bar(K_EMPTY + st));
+                        mbar_arrive(bar(V_EMPTY + st));
+                        ++n_kv;
+                    }
+                    continue;
                 }
-                valid = valid_next;
+                qb = q_seq % 3;
+                // this issuer serves query tile g: S_g(0), then per key tile  O_g += P_g V(j),  S_g(j + 1)
+                TileIter it(it_.rng, it_.nrng);
+                int t0, valid, valid_next = 0;
+                ok = it.next(t0, valid);
+                ok = ok && mbar_wait(bar(Q_FULL + qb), (q_seq / 3) & 1, abort_flag, p.status, W_QFULL);
+                ok = ok && mbar_wait(bar(K_FULL + (n_kv & 1)), (n_kv >> 1) & 1, abort_flag, p.status, W_KFULL);
+                if (!ok) break;
+                tc_fence_after();
+                issue_qk(n_kv & 1, valid);
+                tc_commit(bar(S_FULL + g));
+                tc_commit(bar(K_EMPTY + (n_kv & 1)));
+                if (n_tiles == 1) tc_commit(bar(Q_EMPTY + qb));       // that was the item's only S: its Q buffer may be refilled
+                for (int jt = 0; ok && jt < n_tiles; ++jt) {
+                    const int st = n_kv & 1, sn = (n_kv + 1) & 1;
+                    const uint32_t ph = (n_kv >> 1) & 1, phn = ((n_kv + 1) >> 1) & 1;
+                    const bool more = it.next(t0, valid_next);
+                    if (!mbar_wait(bar(V_FULL + st), ph, abort_flag, p.status, W_VFULL)) { ok = false; break; }
+                    if (more && !mbar_wait(bar(K_FULL + sn), phn, abort_flag, p.status, W_KFULL)) { ok = false; break; }
+                    const int steps = (valid + 15) >> 4, half = min(steps, 4);
+                    if (!mbar_wait(bar(P_HALF + g), n_p & 1, abort_flag, p.status, W_PHALF)) { ok = false; break; }
+                    // the first P V of an item overwrites O: the previous item's epilogue must have read it
+                    if (jt == 0 && n_mine > 0 && !mbar_wait(bar(O_FREE + g), (n_mine - 1) & 1, abort_flag, p.status, W_OFREE)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_pv(st, 0, half, jt > 0);
+                    if (!mbar_wait(bar(P_FULL + g), n_p & 1, abort_flag, p.status, W_PFULL)) { ok = false; break; }
+                    tc_fence_after();
+                    if (steps > half) issue_pv(st, half, steps, true);
+                    // a commit between two groups of MMAs leaves the pipe idle: the next S goes out first, then all commits
+                    if (more) {
+                        issue_qk(sn, valid_next);
+                        tc_commit(bar(S_FULL + g));
+                        tc_commit(bar(V_EMPTY + st));
+                        tc_commit(bar(K_EMPTY + sn));
+                        if (jt + 2 == n_tiles) tc_commit(bar(Q_EMPTY + qb));      // the item's last S: its Q buffer may be refilled
+                    } else {
+                        tc_commit(bar(V_EMPTY + st));
+                        tc_commit(bar(O_FULL + g));
+                    }
+                    valid = valid_next;
+                    ++n_kv;
+                    ++n_p;
+                }
+                ++n_mine;
+            }
+        }
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        // ------------------------------------------------------------ scheduler (lane 0 claims items in queue order) and
+        // Q loader (the whole warp): a claimed item is published at once, then its query tiles are loaded as their
+        // buffers come free, which for the first tile is before the previous item has finished
+        bool usable = false;
+        int total = 0, n_phases = 0;
+        if (lane == 0) {
+            usable = *(volatile int *)p.status == 0 && (uint32_t)((volatile int *)p.status)[ST_COOKIE] == p.cookie;
+            if (!usable) atomicCAS(p.status, 0, MOC_ERR_WORKSPACE);      // not this plan's lists: report, touch nothing else
+            total = usable ? p.queue[1] : 0;
+            n_phases = p.queue[2];
+            prefetch_tensormap(&tmQ);
+            prefetch_tensormap(&tmQrow);
+        }
+        int n_item = 0, n_qtile = 0;
+        bool ok = true;
+        while (ok) {
+            const int sl = n_item & 1;
+            ItemSlot s;
+            s.valid = 0; s.routed = 0; s.h = 0; s.first = 0; s.rows = 0; s.nrng = 0; s.ntiles = 0; s.phase = 0; s.rng = nullptr;
+            if (lane == 0) {
+                if (n_item >= 2) ok = mbar_wait(bar(ITEM_EMPTY + sl), ((n_item - 2) >> 1) & 1, abort_flag, p.status, W_ITEMEMPTY);
+                const int t = (ok && usable && !*abort_flag && *(volatile int *)p.status == 0) ? atomicAdd(&p.queue[0], 1) : total;
+                if (t < total) {
+                    int ph = 0;
+                    while (ph + 1 < n_phases && phase_tab[3 * (ph + 1)] <= t) ++ph;
+                    const int local = t - phase_tab[3 * ph], group = ph >> 1, h0 = group * p.hg;
+                    WorkItem w;
+                    s.routed = (ph & 1) == 0;
+                    if (s.routed) {
+                        w = p.ritems[p.tile_off[(size_t)h0 * p.C] + local];
+                        s.h = w.h;
+                        s.rng = p.chunk_rng + w.rng_off;
+                    } else {
+                        w = p.aitems[local % p.n_aitems];
+                        s.h = h0 + local / p.n_aitems;
+                        s.rng = p.anc_rng + w.rng_off;
+                    }
+                    s.first = w.first; s.rows = w.rows; s.nrng = w.nrng; s.ntiles = w.ntiles; s.phase = ph;
+                    s.valid = 1;
+                    if (s.routed && !index_ok((unsigned)w.h < (unsigned)p.H && w.rows > 0 && w.rows <= kQTileRows && w.first >= 0 &&
+                                              (size_t)w.first + w.rows <= p.cap_total && w.nrng == 1, p.status, IX_ITEM_FIELDS))
+                        s.valid = 0;
+                }
+                s_item[sl] = s;
+                __threadfence_block();
+                mbar_arrive(bar(ITEM_FULL + sl));
+            }
+            ++n_item;
+            // the rest of the warp learns the item from lane 0
+            const int valid = __shfl_sync(0xffffffffu, s.valid, 0), routed = __shfl_sync(0xffffffffu, s.routed, 0);
+            const int h = __shfl_sync(0xffffffffu, s.h, 0), first = __shfl_sync(0xffffffffu, s.first, 0), rows = __shfl_sync(0xffffffffu, s.rows, 0);
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+            if (!valid || !ok) break;
+            const int n_qt = rows > 128 ? 2 : 1;
+            for (int g = 0; ok && g < n_qt; ++g) {
+                const int qb = n_qtile % 3;
+                ok = mbar_wait(bar(Q_EMPTY + qb), ((n_qtile / 3) & 1) ^ 1, abort_flag, p.status, W_QEMPTY);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (lane == 0) mbar_expect_tx(bar(Q_FULL + qb), TILE_BYTES);
+                __syncwarp();
+                if (!routed) {
+                    if (lane == 0) {
+#pragma unroll
+                        for (int sub = 0; sub < SUB; ++sub)
+                            tma_load_2d(sQ + qb * TILE_BYTES + sub * SUB_BYTES, &tmQ, sub * 64, h * p.L + first + g * 128, bar(Q_FULL + qb));
+                    }
+                } else {
+                    // lane l gathers rows 4 l .. 4 l + 3 of the tile; a row past the item's end repeats the item's
+                    // first query (its result is never stored)
+                    int row[4];
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        const int rt = g * 128 + lane * 4 + x;
+                        const size_t at = (size_t)first + (rt < rows ? rt : 0);
+                        const int e = at < p.cap_total ? p.qlist[(size_t)h * p.cap_total + at] : 0;
+                        int qi = e / p.k;
+                        if (e < 0 || qi >= p.L) qi = 0;
+                        row[x] = h * p.L + qi;
+                    }
+#pragma unroll
+                    for (int sub = 0; sub < SUB; ++sub)
+                        tma_gather4(sQ + qb * TILE_BYTES + sub * SUB_BYTES + lane * 512, &tmQrow, sub * 64, row[0], row[1], row[2], row[3],
+                                    bar(Q_FULL + qb));
+                }
+                ++n_qtile;
+            }
+        }
+        if (*abort_flag && lane == 0) {
+            // drain: the Q copies already issued must land before the CTA's shared memory is released
+            int dummy_flag = 0;
+            for (int b = 1; b <= 3; ++b) {
+                const int qj = n_qtile - b;
+                if (qj >= 0) mbar_wait(bar(Q_FULL + qj % 3), (qj / 3) & 1, &dummy_flag, p.status, W_QFULL);
             }
         }
     }
@@ -548,48 +801,41 @@ int make_tmap_2d_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_
 template <int D>
 static int attend_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
                        __nv_bfloat16 *O, float *lse, void *ws, cudaStream_t s) {
-    CUtensorMap tmK, tmV;
+    CUtensorMap tmQ, tmQrow, tmK, tmV;
+    if (int r = make_tmap_2d_bf16(&tmQ, Q, (uint64_t)p->H * p->L, D, 128)) return r;
+    if (int r = make_tmap_2d_bf16(&tmQrow, Q, (uint64_t)p->H * p->L, D, 1)) return r;      // row gathers: a box one row high
     if (int r = make_tmap_2d_bf16(&tmK, K, (uint64_t)p->H * p->L, D, kBN)) return r;
     if (int r = make_tmap_2d_bf16(&tmV, V, (uint64_t)p->H * p->L, D, kBN)) return r;
+    const int n_groups = (p->H + p->heads_per_group - 1) / p->heads_per_group;
     AttendParams a;
     a.Q = Q; a.O = O; a.lse = lse;
     a.part_o = ws_ptr<__nv_bfloat16>(ws, p->ws.part_o);
     a.part_lse = ws_ptr<float>(ws, p->ws.part_lse);
+    a.part_stride = n_groups > 1 ? (size_t)p->heads_per_group * ((p->L + 127) / 128 * 128) * p->k * D : 0;
+    a.chunk_rng = p->d_chunk_rng; a.anc_rng = p->d_anc_rng;
+    a.ritems = ws_ptr<WorkItem>(ws, p->ws.rtiles);
+    a.aitems = p->d_qitems;
+    a.tile_off = ws_ptr<int>(ws, p->ws.tile_off);
     a.qlist = ws_ptr<int32_t>(ws, p->ws.qlist);
+    a.queue = ws_ptr<int>(ws, p->ws.queue);
     a.cap_total = (size_t)p->cap_off[p->C];
     a.status = ws_ptr<int>(ws, p->ws.status);
-    a.H = p->H; a.L = p->L; a.k = p->k;
+    a.H = p->H; a.L = p->L; a.C = p->C; a.k = p->k; a.hg = p->heads_per_group; a.n_groups = n_groups;
+    a.n_aitems = (int)p->qitems.size();
     a.scale_log2 = p->scale * 1.4426950408889634f;
     a.cookie = p->cookie;
+    attend_queue_kernel<<<1, 256, 0, s>>>(a.queue, a.tile_off, ws_ptr<int>(ws, p->ws.cnt), a.status, p->cookie, p->H, p->L, p->C, p->k,
+                                          p->heads_per_group, n_groups, a.n_aitems);
+    MOC_LAUNCH_CHECK();
     // always the d = 128 footprint: more than half an SM's shared memory, so CTAs (which each
     // take all 512 TMEM columns) never share an SM
-    const size_t smem = 6 * (size_t)128 * 128 * 2 + 1024;
-    MOC_CUDA_TRY(cudaFuncSetAttribute(attend_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    MOC_CUDA_TRY(cudaFuncSetAttribute(attend_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    // group by group of heads: the routed pass leaves the group's partials in the workspace, the anchor
-    // pass merges them
-    const int *tile_off = ws_ptr<int>(ws, p->ws.tile_off);
-    for (int h0 = 0; h0 < p->H; h0 += p->heads_per_group) {
-        const int hg = std::min(p->heads_per_group, p->H - h0);
-        a.h0 = h0;
-        if (p->k > 0) {
-            // routed pass: the items and their count were left in the workspace with the lists; the grid
-            // covers the most the group can have
-            a.rng = p->d_chunk_rng;
-            a.items = ws_ptr<WorkItem>(ws, p->ws.rtiles);
-            a.item_lo_dev = tile_off + (size_t)h0 * p->C;
-            a.item_hi_dev = tile_off + (size_t)(h0 + hg) * p->C;
-            const long long bound = (long long)hg * (((long long)p->L * p->k + kQTileRows - 1) / kQTileRows + p->C);
-            attend_tc_kernel<D, true><<<(unsigned)bound, kThreads, smem, s>>>(tmK, tmV, a);
-            MOC_LAUNCH_CHECK();
-        }
-        a.rng = p->d_anc_rng;
-        a.items = p->d_qitems;
-        a.item_lo_dev = a.item_hi_dev = nullptr;
-        dim3 grid((unsigned)p->qitems.size(), (unsigned)hg);
-        attend_tc_kernel<D, false><<<grid, kThreads, smem, s>>>(tmK, tmV, a);
-        MOC_LAUNCH_CHECK();
-    }
+    const size_t smem = 7 * (size_t)128 * 128 * 2 + 1024;      // Q ring of three, K and V two stages each
+    MOC_CUDA_TRY(cudaFuncSetAttribute(attend_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    // one CTA per SM, never more than there are anchor items (the least the queue can hold)
+    const long long most = (long long)p->H * a.n_aitems;
+    const unsigned grid = (unsigned)std::max(1LL, std::min<long long>(p->n_sm, most));
+    attend_tc_kernel<D><<<grid, kThreads, smem, s>>>(tmQ, tmQrow, tmK, tmV, a);
+    MOC_LAUNCH_CHECK();
     return MOC_OK;
 }
 

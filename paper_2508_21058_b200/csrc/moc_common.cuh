@@ -16,6 +16,7 @@ constexpr int kStatusWords = 16;    // status area at the head of the workspace 
 // [0] device status (a moc_status), [1] detail code, [2] cookie of the plan whose lists the workspace holds,
 // [3] limit of every bounded wait in microseconds (0 = the default of one second)
 enum StatusWord { ST_STATUS = 0, ST_DETAIL = 1, ST_COOKIE = 2, ST_WAIT_US = 3 };
+constexpr int kQueueHeader = 4;     // queue area: [0] next item to claim, [1] items, [2] phases, [3] spare; then 3 ints per phase
 constexpr unsigned kPrivFlagCudaCoreAttend = 0x80000000u;   // plan flag outside the public header: test hook
 
 // One contiguous range of key tokens [t0, t1).
@@ -39,7 +40,9 @@ struct WsLayout {
     size_t desc3;       // bf16 [H][3][Cpad][d]  descriptors split into three bf16 terms (hi + mid + lo)
     size_t pool_part;   // float[H][n_pool_units][d] partial key sums
     size_t pool_done;   // int32[H][C] arrival counters (cleared at the start of every pooling call)
-    size_t part_o;      // bf16 [Hg][L][k][d] routed partial outputs (normalised) of one group of Hg heads at a time
+    size_t queue;       // int32[kQueueHeader + 6 groups] work queue of the forward attention kernel
+    size_t part_o;      // bf16 [1 or 2][Hg][L][k][d] routed partial outputs (normalised) of one group of Hg heads; with
+                        // several groups, two buffers that consecutive groups alternate between
     size_t part_lse;    // float[H][L][k]    routed partial log-sum-exp (-inf = unused slot)
     size_t fwd_end;
     size_t delta;       // float[H][L]       rowsum(dO * O)
@@ -136,6 +139,17 @@ __device__ __forceinline__ bool index_ok(bool cond, int *status, int code) {
 #else
 __device__ __forceinline__ bool index_ok(bool, int *, int) { return true; }
 #endif
+
+// Layout of the routed partial outputs.  The row of one (query, slot) is written by one thread of a routed item
+// and read by one thread of the query's anchor item, 16 bytes (a "piece": eight columns) at a time.  Anchor items
+// hold consecutive queries in consecutive lanes, so the pieces are laid out query-innermost: within a block of 128
+// queries, piece c of slot s of the block's queries is 128 x 16 contiguous bytes.  A warp's load of one piece for
+// its 32 queries is then 512 contiguous bytes instead of 32 scattered 16-byte requests.
+//   index (in 16-byte units) of piece c of (head-in-group hl, query qi, slot s); NP = d / 8 pieces per row,
+//   LB = ceil(L / 128) blocks per head
+__device__ __forceinline__ size_t part_piece(int hl, int LB, int k, int NP, int qi, int s, int c) {
+    return ((((size_t)hl * LB + (qi >> 7)) * k + s) * NP + c) * 128 + (qi & 127);
+}
 
 // Walks the 128-key tiles of a list of key ranges (a tile never straddles two ranges).
 struct TileIter {

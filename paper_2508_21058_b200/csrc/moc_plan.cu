@@ -34,16 +34,23 @@ static bool is_anchor(const moc_plan *p, int c, int j) {
 }
 
 // Workspace layout.  The routed partial outputs ([heads][L][k][d] bf16, k times the size of O) are held for
-// one group of Hg heads at a time; attention and its backward run group by group.  Hg is the largest
-// even split of the heads whose partials stay within the plan's budget (at least one head).
+// one group of Hg heads at a time; attention and its backward run group by group.  If all heads fit the plan's
+// budget there is one group and one buffer; otherwise two buffers of Hg heads each (consecutive groups
+// alternate, so that one group's routed items can run while the previous group's anchor items still merge),
+// Hg the largest even split of the heads for which both stay within the budget (at least one head).
 void layout_workspace(moc_plan *p) {
     WsLayout &w = p->ws;
     const size_t H = p->H, L = p->L, d = p->d, C = p->C, k = p->k;
-    const size_t per_head = sizeof(__nv_bfloat16) * L * k * d;
-    size_t hg = per_head ? std::max<size_t>(1, p->partials_budget / per_head) : H;
-    hg = std::min(hg, H);
-    const size_t groups = (H + hg - 1) / hg;
-    p->heads_per_group = (int)((H + groups - 1) / groups);
+    const size_t per_head = sizeof(__nv_bfloat16) * ((L + 127) / 128 * 128) * k * d;      // whole blocks of 128 queries
+    size_t groups = 1, buffers = 1;
+    p->heads_per_group = (int)H;
+    if (per_head * H > p->partials_budget) {
+        const size_t hg = std::max<size_t>(1, p->partials_budget / (2 * per_head));
+        groups = (H + hg - 1) / hg;
+        p->heads_per_group = (int)((H + groups - 1) / groups);
+        groups = (H + p->heads_per_group - 1) / p->heads_per_group;
+        buffers = groups > 1 ? 2 : 1;
+    }
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
     w.status = take(sizeof(int32_t) * kStatusWords);
@@ -54,7 +61,8 @@ void layout_workspace(moc_plan *p) {
     w.desc3 = take(sizeof(__nv_bfloat16) * H * 3 * (size_t)p->c_pad * d);
     w.pool_part = take(sizeof(float) * H * (size_t)p->n_pool_units * d);
     w.pool_done = take(sizeof(int32_t) * H * C);
-    w.part_o = take(per_head * (size_t)p->heads_per_group);
+    w.queue = take(sizeof(int32_t) * (kQueueHeader + 6 * groups));
+    w.part_o = take(per_head * (size_t)p->heads_per_group * buffers);
     w.part_lse = take(sizeof(float) * H * L * (k ? k : 1));
     w.fwd_end = o;
     w.delta = take(sizeof(float) * H * L);
@@ -258,18 +266,20 @@ extern "C" int moc_plan_destroy(moc_plan *p) {
 
 extern "C" int moc_plan_set_workspace_budget(moc_plan *p, size_t max_bytes) {
     if (!p) return MOC_ERR_NULL;
-    const size_t per_head = sizeof(__nv_bfloat16) * (size_t)p->L * p->k * p->d;
+    const size_t per_head = sizeof(__nv_bfloat16) * (((size_t)p->L + 127) / 128 * 128) * p->k * p->d;
     const size_t old = p->partials_budget;
-    p->partials_budget = per_head;                       // one head at a time: the smallest workspace there is
+    // the smallest workspace there is: one head at a time (two buffers of one head, or one if there is one head)
+    p->partials_budget = p->H > 1 ? 2 * per_head : per_head;
     layout_workspace(p);
-    const size_t rest = p->ws.fwd_end - per_head;
+    const size_t rest = p->ws.fwd_end - p->partials_budget;
     if (p->ws.fwd_end > max_bytes) {
         p->partials_budget = old;
         layout_workspace(p);
         return MOC_ERR_TOO_LARGE;
     }
-    p->partials_budget = std::max(per_head, max_bytes - rest - 4096);
+    p->partials_budget = std::max(p->partials_budget, max_bytes - rest - 65536);
     layout_workspace(p);
+    if (p->ws.fwd_end > max_bytes) return MOC_ERR_TOO_LARGE;       // cannot happen: the partials only shrank
     return MOC_OK;
 }
 
