@@ -140,9 +140,11 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     const int hist_ints = (KMAX <= 8 && p.C <= kRtDeferredChunks ? 4 : 1) * p.C;
     int *s_cap = hist_base + NG * hist_ints;                             // copy of cap_off[0 .. C)
     int *s_col = s_cap + p.C;                                            // copy of col_chunk[0 .. ncol)
-    uint16_t *s_reach = reinterpret_cast<uint16_t *>(s_col + p.ncol);   // columns in reach of each of this CTA's units
+    // per unit of this CTA, packed: columns in reach (bits 0-15), scoring steps (16-23), Q stage (24-27) and the parity
+    // of that stage's use (28): worked out once by all threads, so that the single threads that load and issue never divide
+    uint32_t *s_unit = reinterpret_cast<uint32_t *>(s_col + p.ncol);
     // threshold selection: per group, surv_cap slots of (score, column) per query row; slot e of row r at [e][r]
-    float *surv_base = reinterpret_cast<float *>(reinterpret_cast<uintptr_t>(s_reach + p.tiles_per_head / p.ctas_per_head + 16) + 15 & ~(uintptr_t)15);
+    float *surv_base = reinterpret_cast<float *>(reinterpret_cast<uintptr_t>(s_unit + p.tiles_per_head / p.ctas_per_head + 16) + 15 & ~(uintptr_t)15);
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     constexpr int Q_FULL = 0, Q_EMPTY = kMaxStages, D_FULL = 2 * kMaxStages, D_EMPTY = D_FULL + 1, ACC_FULL = D_FULL + 2,
                   ACC_EMPTY = ACC_FULL + NG, GROUP = ACC_EMPTY + NG;
@@ -179,7 +181,15 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     auto unit_of = [&](int n) { return part + n * p.ctas_per_head; };
     for (int x = threadIdx.x; x < p.C; x += kRtThreads) s_cap[x] = p.cap_off[x];
     for (int x = threadIdx.x; x < p.ncol; x += kRtThreads) s_col[x] = p.col_chunk[x];
-    for (int x = threadIdx.x; x < nu; x += kRtThreads) s_reach[x] = (uint16_t)chunks_in_reach(p, unit_of(x));
+    for (int x = threadIdx.x; x < nu; x += kRtThreads) {
+        const int reach = chunks_in_reach(p, unit_of(x));
+        s_unit[x] = (uint32_t)reach | (uint32_t)max(1, (reach + p.sb_rows - 1) / p.sb_rows) << 16 | (uint32_t)(x % p.q_stages) << 24 |
+                    (uint32_t)((x / p.q_stages) & 1) << 28;
+    }
+    auto reach_of = [&](int n) { return (int)(s_unit[n] & 0xffffu); };
+    auto steps_of = [&](int n) { return (int)((s_unit[n] >> 16) & 0xffu); };
+    auto qstage_of = [&](int n) { return (int)((s_unit[n] >> 24) & 0xfu); };
+    auto qparity_of = [&](int n) { return (int)((s_unit[n] >> 28) & 1u); };
     __syncthreads();
     constexpr int ACC_COLS = 512 / NG;   // TMEM columns per accumulator (NG = 4 only with sb_rows <= 128)
     const int n_pass = KMAX == 64 ? p.n_pass : 1;     // only the 64-entry list is used for more picks than it holds
@@ -199,10 +209,10 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             for (int n0 = 0; ok && n0 < nu; n0 += grp) {
                 const int n1 = min(n0 + grp, nu);
                 int n_sb = 1;
-                for (int n = n0; n < n1; ++n) n_sb = max(n_sb, (s_reach[n] + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a column in reach
+                for (int n = n0; n < n1; ++n) n_sb = max(n_sb, steps_of(n));   // blocks that hold a column in reach
                 for (int n = n0; ok && n < n1; ++n) {
-                    const int st = qn % p.q_stages;
-                    ok = mbar_wait(bar(Q_EMPTY + st), ((qn / p.q_stages) & 1) ^ 1, abort_flag, p.status, RW_QEMPTY);
+                    const int st = qstage_of(n);                          // qn == n: one Q tile per unit, in unit order
+                    ok = mbar_wait(bar(Q_EMPTY + st), qparity_of(n) ^ 1, abort_flag, p.status, RW_QEMPTY);
                     if (!ok) break;
                     mbar_expect_tx(bar(Q_FULL + st), Q_TILE_BYTES);
 #pragma unroll
@@ -261,9 +271,9 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
             for (int n0 = first; ok && n0 < nu; n0 += resident ? stride : grp) {
                 const int n1 = min(n0 + grp, nu);
                 int n_sb = 1;
-                for (int n = n0; n < n1; ++n) n_sb = max(n_sb, (s_reach[n] + p.sb_rows - 1) / p.sb_rows);
+                for (int n = n0; n < n1; ++n) n_sb = max(n_sb, steps_of(n));
                 for (int n = n0; ok && n < n1; ++n)
-                    ok = mbar_wait(bar(Q_FULL + n % p.q_stages), (n / p.q_stages) & 1, abort_flag, p.status, RW_QFULL);
+                    ok = mbar_wait(bar(Q_FULL + qstage_of(n)), qparity_of(n), abort_flag, p.status, RW_QFULL);
                 for (int rep = 0; ok && rep < n_pass; ++rep)
                 for (int sb = 0; ok && sb < n_sb; ++sb) {
                     if (resident ? dn == 0 : sb != res_sb) {
@@ -273,10 +283,12 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                         res_sb = sb;
                     }
                     for (int n = n0; ok && n < n1; ++n) {
-                        const int reach = s_reach[n];
-                        if (sb >= max(1, (reach + p.sb_rows - 1) / p.sb_rows)) continue;       // this unit needs no such block
-                        const int buf = n % NG, st = n % p.q_stages;
-                        const int uses = nacc_total[buf];
+                        const int reach = reach_of(n);
+                        if (sb >= steps_of(n)) continue;       // this unit needs no such block
+                        const int buf = n % NG, st = qstage_of(n);
+                        int uses = 0;                          // how often this accumulator has been filled (no indexed array:
+#pragma unroll                                                 // the counters stay in registers)
+                        for (int x = 0; x < NG; ++x) uses = x == buf ? nacc_total[x] : uses;
                         ok = mbar_wait(bar(ACC_EMPTY + buf), (uses & 1) ^ 1, abort_flag, p.status, RW_ACCEMPTY);
                         if (!ok) break;
                         tc_fence_after();
@@ -305,7 +317,8 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                             }
                         }
                         tc_commit(bar(ACC_FULL + buf));
-                        ++nacc_total[buf];
+#pragma unroll
+                        for (int x = 0; x < NG; ++x) nacc_total[x] += x == buf ? 1 : 0;
                     }
                     // streamed blocks: the next step, if it needs another block, may overwrite this one once
                     // these MMAs are done
@@ -316,7 +329,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                         if (more && nsb != sb) tc_commit(bar(D_EMPTY));
                     }
                 }
-                for (int n = n0; ok && n < n1; ++n) tc_commit(bar(Q_EMPTY + n % p.q_stages));
+                for (int n = n0; ok && n < n1; ++n) tc_commit(bar(Q_EMPTY + qstage_of(n)));
             }
         }
     } else if (warp < 2 + 4 * NG) {
@@ -392,7 +405,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
         }
         for (int n = sg; ok && n < nu; n += NG) {
             const int u = unit_of(n);
-            const int reach = s_reach[n], n_sb = max(1, (reach + p.sb_rows - 1) / p.sb_rows);   // blocks that hold a column in reach
+            const int reach = reach_of(n), n_sb = steps_of(n);   // blocks that hold a column in reach
             const int i = u * kRtRows + r;
             const bool live = i < p.L;
             const int ci = nx_ci, lim_i = nx_lim;
@@ -942,7 +955,7 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         a.n_pass = p->k > 64 ? (p->k + 63) / 64 : 1;
         // one histogram per group, the list offsets, and one byte per unit of a CTA
         const size_t hist = (ng * (p->k <= 8 && p->C <= kRtDeferredChunks ? 4 : 1) + 1) * sizeof(int) * (size_t)p->C + sizeof(int) * (size_t)p->ncol +
-                            2 * (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
+                            4 * (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
         if (d_block + q_tile + hist > budget) return MOC_ERR_SHAPE;
         // threshold selection (lists of at most 16 picks, not the few-chunk case): survivor slots per row, as many
         // as fit beside two Q stages, at least k + 4 (else the best-first extraction alone is used)
