@@ -14,8 +14,8 @@ constexpr int kQTileRows = 256;     // query rows per attention work item (two 1
 constexpr int kPoolSlice = 256;     // tokens per chunk-pool work unit
 constexpr int kStatusWords = 16;    // status area at the head of the workspace (int32 each):
 // [0] device status (a moc_status), [1] detail code, [2] cookie of the plan whose lists the workspace holds,
-// [3] limit of every bounded wait in microseconds (0 = the default of one second)
-enum StatusWord { ST_STATUS = 0, ST_DETAIL = 1, ST_COOKIE = 2, ST_WAIT_US = 3 };
+// [3] limit of every bounded wait in microseconds (0 = the default of one second), [4] routing blocks that have finished
+enum StatusWord { ST_STATUS = 0, ST_DETAIL = 1, ST_COOKIE = 2, ST_WAIT_US = 3, ST_ARRIVE = 4 };
 constexpr int kQueueHeader = 4;     // queue area: [0] next item to claim, [1] items, [2] phases, [3] spare; then 3 ints per phase
 constexpr unsigned kPrivFlagCudaCoreAttend = 0x80000000u;   // plan flag outside the public header: test hook
 

@@ -103,6 +103,8 @@ struct RouteParams {
     int q_stages;
     int n_pass;             // selection passes over a tile's scores: 64 picks each (the scores are recomputed per pass)
     int surv_cap;           // threshold selection: survivor slots per query row in shared memory (0 = not used)
+    int *tile_off;          // [H C + 1] running tile counts, written by the last block to finish
+    uint32_t cookie;
     size_t cap_total;
 };
 
@@ -797,6 +799,40 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, 512);
+    // The last block to get here turns the pick counts into the running counts of attention tiles over the (head,
+    // chunk) pairs and marks the workspace (what route_tiles_kernel does on the paths that have no such block): one
+    // launch less.  Every block's counts are in place before it arrives (the atomics that made them have
+    // returned), and the fence orders them before the arrival.
+    __shared__ int s_last, s_wsum[32];
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(&p.status[ST_ARRIVE], 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const int HC = p.H * p.C, T = kRtThreads, t = threadIdx.x;
+    const int per = (HC + T - 1) / T, i0 = min(t * per, HC), i1 = min(i0 + per, HC);
+    int mine = 0;
+    for (int i = i0; i < i1; ++i) mine += (__ldcg(p.cnt + i) + kQTileRows - 1) / kQTileRows;
+    int incl = mine;                                     // inclusive scan over the block: warps by shuffles, then warp totals
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    if (lane == 31) s_wsum[warp] = incl;
+    __syncthreads();
+    int at = incl - mine;
+    for (int w = 0; w < warp; ++w) at += s_wsum[w];
+    for (int i = i0; i < i1; ++i) {
+        p.tile_off[i] = at;
+        at += (__ldcg(p.cnt + i) + kQTileRows - 1) / kQTileRows;
+    }
+    if (t == T - 1) {
+        p.tile_off[HC] = at;
+        p.status[ST_COOKIE] = (int)p.cookie;
+    }
 }
 
 // gtile[i] = attention tiles (of kQTileRows picks) before (head, chunk) pair i, with a final total;
@@ -840,10 +876,12 @@ __global__ void route_items_kernel(const int *__restrict__ cnt, const int *__res
 
 
 // Tile counts, routed work items and the cookie, from the per-(head, chunk) pick counts and lists.
-static int finish_lists(const moc_plan *p, void *ws, cudaStream_t s) {
+static int finish_lists(const moc_plan *p, void *ws, cudaStream_t s, bool count_tiles) {
     int *cnt = ws_ptr<int>(ws, p->ws.cnt);
-    route_tiles_kernel<<<1, 1024, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off), ws_ptr<int>(ws, p->ws.status), p->H * p->C, p->cookie);
-    MOC_LAUNCH_CHECK();
+    if (count_tiles) {
+        route_tiles_kernel<<<1, 1024, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off), ws_ptr<int>(ws, p->ws.status), p->H * p->C, p->cookie);
+        MOC_LAUNCH_CHECK();
+    }
     if (p->k > 0) {
         route_items_kernel<<<(unsigned)((p->H * p->C + 3) / 4), 128, 0, s>>>(cnt, ws_ptr<int>(ws, p->ws.tile_off),
                                                                                ws_ptr<WorkItem>(ws, p->ws.rtiles), p->d_off,
@@ -917,7 +955,7 @@ int launch_lists_from_sel(const moc_plan *p, int32_t *sel, void *ws, cudaStream_
             p->d_cap_off, status, p->L, p->C, p->k, p->words, (p->flags & MOC_FLAG_CAUSAL) ? 1 : 0, (size_t)p->cap_off[p->C]);
         MOC_LAUNCH_CHECK();
     }
-    return finish_lists(p, ws, s);
+    return finish_lists(p, ws, s, true);
 }
 
 template <int D>
@@ -945,6 +983,8 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         // (256 chunks) with two, which is every case but the few-chunk one; streamed blocks are 128 chunks
         a.sb_rows = std::min(a.d_rows, p->c_pad <= 32 ? kRtBlock : 2 * kRtBlock);
         a.cap_total = (size_t)p->cap_off[p->C];
+        a.tile_off = ws_ptr<int>(ws, p->ws.tile_off);
+        a.cookie = p->cookie;
         const size_t q_tile = (size_t)kRtRows * D * 2, d_block = ((size_t)3 * a.d_rows * D * 2 + 1023) & ~(size_t)1023;
         a.ctas_per_head = std::max(1, std::min(p->n_sm / p->H, a.tiles_per_head));
         const unsigned grid = (unsigned)(p->H * a.ctas_per_head);
@@ -986,8 +1026,9 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         else MOC_ROUTE_CASE(64, 1, false);                 // beyond 64 picks: several passes of 64
 #undef MOC_ROUTE_CASE
         MOC_LAUNCH_CHECK();
+        return finish_lists(p, ws, s, false);       // the routing kernel's last block has counted the tiles
     }
-    return finish_lists(p, ws, s);
+    return finish_lists(p, ws, s, true);
 }
 
 int launch_route(const moc_plan *p, const __nv_bfloat16 *Q, const float *desc, int32_t *sel, void *ws, cudaStream_t s) {
