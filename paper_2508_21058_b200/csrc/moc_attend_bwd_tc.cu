@@ -50,6 +50,7 @@ struct BwdParams {
     int h0;                       // first head of the group in flight
     uint32_t cookie;              // what the workspace's status area must hold
     const KTile *ktiles;          // dK/dV mode
+    int n_ktiles, n_long;         // tiles per head, and how many of them come first for every head
     const int32_t *off, *ranc_off, *ranc, *cap_off;
     const int *cnt;
     const int32_t *qlist;
@@ -129,8 +130,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 if (w_rows <= 0) valid = 0;
             }
         } else {
-            const KTile kt = p.ktiles[blockIdx.x];
-            w_h = blockIdx.y;
+            // block order: the long key tiles of every head, then the others head by head (tiles of one chunk next
+            // to each other: they stream the same query rows)
+            const int n_long_all = p.n_long * p.H;
+            int b = blockIdx.x, hh, ti;
+            if (b < n_long_all) { hh = b / p.n_long; ti = b - hh * p.n_long; }
+            else { b -= n_long_all; const int n_rest = p.n_ktiles - p.n_long; hh = b / n_rest; ti = p.n_long + b - hh * n_rest; }
+            const KTile kt = p.ktiles[ti];
+            w_h = hh;
             w_chunk = kt.chunk;
             w_t0 = kt.t0;
             w_rows = kt.valid;
@@ -661,7 +668,7 @@ static int attend_bwd_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv
     a.cookie = p->cookie; a.h0 = 0; a.item_lo_dev = a.item_hi_dev = nullptr;
     a.dQ = dQ; a.dK = dK; a.dV = dV;
     a.part = ws_ptr<__nv_bfloat16>(ws, p->ws.part_o);      // the forward's partial outputs are no longer needed
-    a.ktiles = p->d_ktiles; a.off = p->d_off; a.ranc_off = p->d_ranc_off; a.ranc = p->d_ranc; a.cap_off = p->d_cap_off;
+    a.ktiles = p->d_ktiles; a.n_ktiles = (int)p->ktiles.size(); a.n_long = p->n_long_ktiles; a.off = p->d_off; a.ranc_off = p->d_ranc_off; a.ranc = p->d_ranc; a.cap_off = p->d_cap_off;
     a.cnt = ws_ptr<int>(ws, p->ws.cnt);
     a.qlist = ws_ptr<int32_t>(ws, p->ws.qlist);
     a.cap_total = (size_t)p->cap_off[p->C];
@@ -706,7 +713,7 @@ static int attend_bwd_tc_d(const moc_plan *p, const __nv_bfloat16 *Q, const __nv
         attend_bwd_tc_kernel<D, DQ_ANCHOR><<<dim3((unsigned)(2 * p->qitems.size()), (unsigned)hg), kBwdThreads, smem[DQ_ANCHOR], s>>>(tmK, tmV, a);
         MOC_LAUNCH_CHECK();
     }
-    attend_bwd_tc_kernel<D, DKV><<<dim3((unsigned)p->ktiles.size(), (unsigned)p->H), kBwdThreads, smem[DKV], s>>>(tmK, tmV, a);
+    attend_bwd_tc_kernel<D, DKV><<<(unsigned)(p->ktiles.size() * (size_t)p->H), kBwdThreads, smem[DKV], s>>>(tmK, tmV, a);
     MOC_LAUNCH_CHECK();
     return MOC_OK;
 }

@@ -65,7 +65,8 @@ struct moc_plan {
     std::vector<int64_t> anc_tokens;         // [C] anchor key tokens per query chunk
     std::vector<int32_t> ranc_off, ranc;     // reverse anchors: key chunk -> query chunks
     std::vector<moc::WorkItem> qitems;       // anchor-pass work items of one head
-    std::vector<moc::KTile> ktiles;          // key tiles of one head, chunk by chunk
+    std::vector<moc::KTile> ktiles;          // key tiles of one head: the long ones (see moc_plan_create) first, then chunk by chunk
+    int n_long_ktiles = 0;
     std::vector<int32_t> pool_unit_off;      // [C+1] prefix of pool units per chunk
     std::vector<moc::KeyRange> shot_chunks;  // [S] chunk range [t0, t1) of every shot (outer-loop routing)
     int words;                               // uint32 words per anchor bitmap row

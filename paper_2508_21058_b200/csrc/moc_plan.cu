@@ -162,12 +162,34 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
             p->qitems.push_back(WorkItem{0, r, std::min(kQTileRows, p->off[c + 1] - r), anc_tiles, p->anc_off[c],
                                          p->anc_off[c + 1] - p->anc_off[c], p->anc_rng[p->anc_off[c]].t0,
                                          p->anc_rng[p->anc_off[c]].t1});
-        for (int t = p->off[c]; t < p->off[c + 1]; t += 128) p->ktiles.push_back(KTile{c, t, std::min(128, p->off[c + 1] - t), 0});
         int units = (p->off[c + 1] - p->off[c] + kPoolSlice - 1) / kPoolSlice;
         p->pool_unit_off[c + 1] = p->pool_unit_off[c] + units;
         for (int u = 0; u < units; ++u) unit_chunk.push_back(c);
     }
     p->n_pool_units = p->pool_unit_off[C];
+    // Key tiles of the backward's key-stationary pass.  A tile's block streams every query that attends its chunk:
+    // the rows of the chunks that have it as an anchor (known here) and the routed list.  Tiles of chunks whose
+    // anchor rows are far above the average (a caption, which every query attends) go first, for all heads, so
+    // that the longest blocks start at once instead of forming the tail of the launch.
+    {
+        std::vector<int64_t> anc_rows(C, 0);
+        int64_t total = 0, tiles = 0;
+        for (int c = 0; c < C; ++c) {
+            for (int a = p->ranc_off[c]; a < p->ranc_off[c + 1]; ++a) anc_rows[c] += p->off[p->ranc[a] + 1] - p->off[p->ranc[a]];
+            const int nt = (p->off[c + 1] - p->off[c] + 127) / 128;
+            total += anc_rows[c] * nt;
+            tiles += nt;
+        }
+        const int64_t mean_rows = total / std::max<int64_t>(tiles, 1);
+        for (int pass = 0; pass < 2; ++pass) {
+            for (int c = 0; c < C; ++c) {
+                const bool is_long = anc_rows[c] > 4 * mean_rows;
+                if (is_long != (pass == 0)) continue;
+                for (int t = p->off[c]; t < p->off[c + 1]; t += 128) p->ktiles.push_back(KTile{c, t, std::min(128, p->off[c + 1] - t), 0});
+            }
+            if (pass == 0) p->n_long_ktiles = (int)p->ktiles.size();
+        }
+    }
     // Query-list capacities: chunk c can be picked by at most the rows after it (causal) or by
     // every row (non-causal); the lists sit back to back at these fixed offsets, so routing can
     // append to them without a counting pass.
