@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
         const float c = p.scale_log2;
         // running counts that give every barrier's phase: items seen, items this group worked on, key tiles it
         // processed, key tiles processed in two-tile items (the turn-taking of the exponentials)
-        int n_item = 0, n_mine = 0, n_s = 0, n_turn = 0;
+        int n_item = 0, n_mine = 0, n_s = 0, n_turn = 0, n_dep = 0;
         bool ok = true;
         while (ok) {
             const int sl = n_item & 1;
@@ -227,6 +227,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             if (!it_.valid) break;
             const int h = it_.h, rows = it_.rows, first = it_.first, group = it_.phase >> 1;
             const bool routed = it_.routed != 0, two = rows > 128;
+            // an item that depends on other items' rows (see the bookkeeping lane) is released through DEPEND, whose
+            // phase counts those items only
+            const bool dep = routed ? group >= 2 : p.k > 0;
+            const int dep_phase = n_dep & 1;
+            if (dep) ++n_dep;
             if (g == 1 && !two) continue;               // this item has one query tile
             const int rt = g * 128 + r;                 // row within the work item
             int qi = -1, slot = 0;
@@ -250,11 +255,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             uint4 *part16 = reinterpret_cast<uint4 *>(part_o);
             if (!routed && qi >= 0 && p.k > 0) {
                 // the epilogue will merge this row's routed partials: start them on their way into L2 now.  A 128-byte
-                // line holds one piece of eight consecutive queries: every eighth query (and the tile's first) asks
+                // line holds one pair of pieces of four consecutive queries: every fourth query (and the tile's first) asks
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(p.part_lse + ((size_t)h * p.L + qi) * p.k));
-                if ((qi & 7) == 0 || r == 0)
+                if ((qi & 3) == 0 || r == 0)
                     for (int s = 0; s < p.k; ++s)
-                        for (int cc = 0; cc < NP; ++cc)
+                        for (int cc = 0; cc < NP; cc += 2)
                             asm volatile("prefetch.global.L2 [%0];" ::"l"(part16 + part_piece(h_loc, LB, p.k, NP, qi, s, cc)));
             }
 
@@ -366,9 +371,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             // what this item depends on (an anchor item: the routed items of its group have stored all their partials;
             // a routed item: the anchor items two groups back have read the buffer it is about to store into) has been
             // awaited by the bookkeeping lane, which then arrives on DEPEND, once per item
-            ok = mbar_wait(bar(DEPEND), (n_item - 1) & 1, abort_flag, p.status, W_DEPEND);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+            if (dep) {
+                ok = mbar_wait(bar(DEPEND), dep_phase, abort_flag, p.status, W_DEPEND);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+            }
             if (!routed && qi >= 0 && p.k > 0) {
                 pl = p.part_lse + ((size_t)h * p.L + qi) * p.k;
                 if (p.k <= KW) {
@@ -416,10 +423,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
 #pragma unroll
                         for (int s = 0; s < 4; ++s)
 #pragma unroll
-                            for (int q4 = 0; q4 < 4; ++q4)
-                                raw[s][q4] = (s0 + s < p.k && wslot[s0 + s] != 0.f)
-                                                 ? __ldcg(part16 + part_piece(h_loc, LB, p.k, NP, qi, s0 + s, ch * 4 + q4))
-                                                 : make_uint4(0, 0, 0, 0);
+                            for (int q4 = 0; q4 < 4; q4 += 2) {
+                                raw[s][q4] = raw[s][q4 + 1] = make_uint4(0, 0, 0, 0);
+                                if (s0 + s < p.k && wslot[s0 + s] != 0.f)
+                                    ld_cg_256(part16 + part_piece(h_loc, LB, p.k, NP, qi, s0 + s, ch * 4 + q4), raw[s][q4], raw[s][q4 + 1]);
+                            }
 #pragma unroll
                         for (int s = 0; s < 4; ++s) {
                             const float w = wslot[s0 + s];
@@ -440,10 +448,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                         const float ls = __ldcg(pl + s);
                         if (ls == -INFINITY) continue;
                         const float w = __expf(ls - big) / wsum;
+                        uint4 raw[4];
+                        ld_cg_256(part16 + part_piece(h_loc, LB, p.k, NP, qi, s, ch * 4), raw[0], raw[1]);
+                        ld_cg_256(part16 + part_piece(h_loc, LB, p.k, NP, qi, s, ch * 4 + 2), raw[2], raw[3]);
 #pragma unroll
                         for (int q4 = 0; q4 < 4; ++q4) {
-                            const uint4 raw = __ldcg(part16 + part_piece(h_loc, LB, p.k, NP, qi, s, ch * 4 + q4));
-                            const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+                            const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&raw[q4]);
 #pragma unroll
                             for (int y = 0; y < 4; ++y) {
                                 const float2 f = __bfloat1622float2(b[y]);
@@ -455,17 +465,22 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 }
                 if (qi < 0) continue;
                 uint4 *dst_row = reinterpret_cast<uint4 *>(p.O + ((size_t)h * p.L + qi) * D + ch * 32);
+                uint4 out[4];
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
-                    uint4 out;
-                    uint32_t *o32 = reinterpret_cast<uint32_t *>(&out);
+                    uint32_t *o32 = reinterpret_cast<uint32_t *>(&out[q4]);
 #pragma unroll
                     for (int y = 0; y < 4; ++y) {
                         __nv_bfloat162 b = __floats2bfloat162_rn(acc[q4 * 8 + 2 * y], acc[q4 * 8 + 2 * y + 1]);
                         o32[y] = *reinterpret_cast<uint32_t *>(&b);
                     }
-                    if (routed) part16[part_piece(h_loc, LB, p.k, NP, qi, slot, ch * 4 + q4)] = out;
-                    else dst_row[q4] = out;
+                }
+                if (routed) {            // whole 32-byte sectors
+                    st_256(part16 + part_piece(h_loc, LB, p.k, NP, qi, slot, ch * 4), out[0], out[1]);
+                    st_256(part16 + part_piece(h_loc, LB, p.k, NP, qi, slot, ch * 4 + 2), out[2], out[3]);
+                } else {
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) dst_row[q4] = out[q4];
                 }
             }
             if (qi >= 0) {
@@ -530,7 +545,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
             // then, when the softmax groups have stored the item's rows, the rows join the phase's count.  The
             // groups' arrivals order their stores before this thread (CTA scope); its fence makes them visible
             // device-wide before the count moves.
+            // An item that depends on nothing does not go through DEPEND at all; the rows of an item are counted when
+            // the next item has been seen, so that the fence before the count (it waits for the item's stores to
+            // land) is not in the way of the next item.  DEPEND is arrived on after the previous item's rows were
+            // counted, that is after every softmax thread has passed its previous wait on it.
             int n_item = 0, n_tile[2] = {0, 0};
+            int pend_phase = -1, pend_rows = 0;                 // the item whose rows are still to be counted
             bool ok = true;
             while (ok) {
                 const int sl = n_item & 1;
@@ -538,23 +558,31 @@ __global__ void __launch_bounds__(kThreads, 1) attend_tc_kernel(const __grid_con
                 const ItemSlot it_ = s_item[sl];
                 mbar_arrive(bar(ITEM_EMPTY + sl));
                 ++n_item;
-                if (!it_.valid) break;
                 const int group = it_.phase >> 1;
-                if (!it_.routed && p.k > 0)
+                const bool dep_anchor = it_.valid && !it_.routed && p.k > 0, dep_routed = it_.valid && it_.routed && group >= 2;
+                if (pend_phase >= 0) {
+                    const int n_qt = pend_rows > 128 ? 2 : 1;
+                    for (int g = 0; ok && g < n_qt; ++g) {
+                        ok = mbar_wait(bar(ROWS_DONE + g), n_tile[g] & 1, abort_flag, p.status, W_ROWSDONE);
+                        ++n_tile[g];
+                    }
+                    if (!ok) break;
+                    __threadfence();
+                    atomicAdd(&phase_tab[3 * pend_phase + 2], pend_rows);
+                    pend_phase = -1;
+                }
+                if (!it_.valid) break;
+                if (dep_anchor)
                     ok = wait_count(&phase_tab[3 * (2 * group) + 2], phase_tab[3 * (2 * group) + 1], abort_flag, p.status, W_DEPEND);
-                if (it_.routed && group >= 2)
+                if (dep_routed)
                     ok = wait_count(&phase_tab[3 * (2 * (group - 2) + 1) + 2], phase_tab[3 * (2 * (group - 2) + 1) + 1], abort_flag, p.status, W_DEPEND);
                 if (!ok) break;
-                __threadfence();
-                mbar_arrive(bar(DEPEND));
-                const int n_qt = it_.rows > 128 ? 2 : 1;
-                for (int g = 0; ok && g < n_qt; ++g) {
-                    ok = mbar_wait(bar(ROWS_DONE + g), n_tile[g] & 1, abort_flag, p.status, W_ROWSDONE);
-                    ++n_tile[g];
+                if (dep_anchor || dep_routed) {
+                    __threadfence();
+                    mbar_arrive(bar(DEPEND));
                 }
-                if (!ok) break;
-                __threadfence();
-                atomicAdd(&phase_tab[3 * it_.phase + 2], it_.rows);
+                pend_phase = it_.phase;
+                pend_rows = it_.rows;
             }
         }
     } else if (warp < 11) {

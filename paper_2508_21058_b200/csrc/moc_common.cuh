@@ -144,12 +144,14 @@ __device__ __forceinline__ bool index_ok(bool, int *, int) { return true; }
 // Layout of the routed partial outputs.  The row of one (query, slot) is written by one thread of a routed item
 // and read by one thread of the query's anchor item, 16 bytes (a "piece": eight columns) at a time.  Anchor items
 // hold consecutive queries in consecutive lanes, so the pieces are laid out query-innermost: within a block of 128
-// queries, piece c of slot s of the block's queries is 128 x 16 contiguous bytes.  A warp's load of one piece for
-// its 32 queries is then 512 contiguous bytes instead of 32 scattered 16-byte requests.
+// queries, the pieces 2 c2 and 2 c2 + 1 (a pair: one 32-byte sector) of slot s of the block's queries are 128 x 32
+// contiguous bytes.  A warp's load of one pair for its 32 queries is then 1024 contiguous bytes instead of 32
+// scattered requests, and a routed item, whose rows are scattered queries, still writes whole sectors (a store of
+// half a sector makes the memory system read the other half first).
 //   index (in 16-byte units) of piece c of (head-in-group hl, query qi, slot s); NP = d / 8 pieces per row,
 //   LB = ceil(L / 128) blocks per head
 __device__ __forceinline__ size_t part_piece(int hl, int LB, int k, int NP, int qi, int s, int c) {
-    return ((((size_t)hl * LB + (qi >> 7)) * k + s) * NP + c) * 128 + (qi & 127);
+    return ((((((size_t)hl * LB + (qi >> 7)) * k + s) * (NP >> 1) + (c >> 1)) * 128 + (qi & 127)) << 1) + (c & 1);
 }
 
 // Walks the 128-key tiles of a list of key ranges (a tile never straddles two ranges).

@@ -280,6 +280,18 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N, int a_mn_maj
 // 128-byte rows whose base is 1024-byte aligned (the layout TMA SWIZZLE_128B produces)
 __device__ __forceinline__ uint32_t sw128_offset(int r, int c16) { return (uint32_t)(r * 128 + ((c16 ^ (r & 7)) << 4)); }
 
+// 32-byte (one sector) global load that is cached in L2 only, and 32-byte global store; addresses 32-byte aligned
+__device__ __forceinline__ void ld_cg_256(const void *ptr, uint4 &a, uint4 &b) {
+    asm volatile("ld.global.cg.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w)
+                 : "l"(ptr));
+}
+__device__ __forceinline__ void st_256(void *ptr, const uint4 &a, const uint4 &b) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(ptr), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
+                 : "memory");
+}
+
 }  // namespace tc
 
 // host: encode a 2-D bf16 tensor map [rows][cols], box {64 cols, box_rows}, 128-byte swizzle
