@@ -103,7 +103,7 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
     if any(r[1] for r in results):
         raise RuntimeError("nvcc failed building " + os.path.basename(lib))
     tmp = lib + f".{os.getpid()}.tmp"
-    res = subprocess.run([nvcc, "-shared", "-o", tmp, *[r[0] for r in results]], capture_output=True, text=True)
+    res = subprocess.run([nvcc, "-shared", "-o", tmp, *[r[0] for r in results], "-ldl"], capture_output=True, text=True)
     if res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)
         raise RuntimeError("link failed building " + os.path.basename(lib))

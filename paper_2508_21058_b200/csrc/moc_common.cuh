@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "../../include/moc.h"
+#include <nvtx3/nvToolsExt.h>
 
 namespace moc {
 
@@ -153,6 +154,14 @@ __device__ __forceinline__ bool index_ok(bool, int *, int) { return true; }
 __device__ __forceinline__ size_t part_piece(int hl, int LB, int k, int NP, int qi, int s, int c) {
     return ((((((size_t)hl * LB + (qi >> 7)) * k + s) * (NP >> 1) + (c >> 1)) * 128 + (qi & 127)) << 1) + (c & 1);
 }
+
+// A named range around a call of the boundary, for timeline tools (NVTX; a no-op when no tool is attached).
+struct NvtxRange {
+    explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange &) = delete;
+    NvtxRange &operator=(const NvtxRange &) = delete;
+};
 
 // Walks the 128-key tiles of a list of key ranges (a tile never straddles two ranges).
 struct TileIter {

@@ -117,6 +117,7 @@ extern "C" int moc_outer_num_shots(const moc_plan *p, int32_t *n_shots) {
 
 extern "C" int moc_outer_route(const moc_plan *p, const void *Xq, const float *desc, int32_t q_tok0, int32_t q_tok1, int32_t top_m,
                                float *shot_desc, float *scores, int32_t *sel_shot, void *ws, void *stream) {
+    moc::NvtxRange nvtx_range("moc_outer_route");
     if (!p) return MOC_ERR_NULL;
     int dev = -1;
     MOC_CUDA_TRY(cudaGetDevice(&dev));
@@ -180,6 +181,7 @@ extern "C" int moc_outer_reduced_layout(const moc_plan *p, const int32_t *sel_sh
 }
 
 extern "C" int moc_gather_tokens(const moc_plan *p, const void *X, const int32_t *tok_map, int32_t n_out, void *out, void *stream) {
+    moc::NvtxRange nvtx_range("moc_gather_tokens");
     if (!p) return MOC_ERR_NULL;
     int dev = -1;
     MOC_CUDA_TRY(cudaGetDevice(&dev));

@@ -328,6 +328,7 @@ static int enter(const moc_plan *p) {
 }
 
 extern "C" int moc_chunk_pool(const moc_plan *p, const void *K, float *desc, void *ws, void *stream) {
+    moc::NvtxRange nvtx_range("moc_chunk_pool");
     if (int r = enter(p)) return r;
     if (int r = check_dev_ptrs({K, desc}, 16)) return r;
     if (!ws) return MOC_ERR_WORKSPACE;
@@ -336,6 +337,7 @@ extern "C" int moc_chunk_pool(const moc_plan *p, const void *K, float *desc, voi
 }
 
 extern "C" int moc_route(const moc_plan *p, const void *Q, const float *desc, int32_t *sel_idx, void *ws, void *stream) {
+    moc::NvtxRange nvtx_range("moc_route");
     if (int r = enter(p)) return r;
     if (int r = check_dev_ptrs({Q, desc}, 16)) return r;
     if (p->k > 0) { if (int r = check_dev_ptrs({sel_idx}, 4)) return r; }
@@ -345,6 +347,7 @@ extern "C" int moc_route(const moc_plan *p, const void *Q, const float *desc, in
 }
 
 extern "C" int moc_lists_from_sel(const moc_plan *p, int32_t *sel_idx, void *ws, void *stream) {
+    moc::NvtxRange nvtx_range("moc_lists_from_sel");
     if (int r = enter(p)) return r;
     if (p->k > 0) { if (int r = check_dev_ptrs({sel_idx}, 4)) return r; }
     if (!ws) return MOC_ERR_WORKSPACE;
@@ -354,6 +357,7 @@ extern "C" int moc_lists_from_sel(const moc_plan *p, int32_t *sel_idx, void *ws,
 
 extern "C" int moc_context_drop(const moc_plan *p, int32_t *sel_idx, float p_max, float lambda, uint64_t seed, void *ws,
                                 void *stream) {
+    moc::NvtxRange nvtx_range("moc_context_drop");
     if (int r = enter(p)) return r;
     if (!(p_max >= 0.f && p_max <= 1.f) || !(lambda >= 0.f && lambda <= 8.f)) return MOC_ERR_SHAPE;
     if (p->k > 0) { if (int r = check_dev_ptrs({sel_idx}, 4)) return r; }
@@ -365,6 +369,7 @@ extern "C" int moc_context_drop(const moc_plan *p, int32_t *sel_idx, float p_max
 
 extern "C" int moc_attend(const moc_plan *p, const void *Q, const void *K, const void *V, const int32_t *sel_idx,
                           void *O, float *lse, void *ws, void *stream) {
+    moc::NvtxRange nvtx_range("moc_attend");
     if (int r = enter(p)) return r;
     if (int r = check_dev_ptrs({Q, K, V, O}, 16)) return r;
     if (int r = check_dev_ptrs({lse}, 4)) return r;
@@ -380,6 +385,7 @@ extern "C" int moc_attend(const moc_plan *p, const void *Q, const void *K, const
 extern "C" int moc_attend_bwd(const moc_plan *p, const void *Q, const void *K, const void *V, const void *O,
                               const float *lse, const void *dO, const int32_t *sel_idx, void *dQ, void *dK, void *dV,
                               void *ws, void *stream) {
+    moc::NvtxRange nvtx_range("moc_attend_bwd");
     if (int r = enter(p)) return r;
     if (int r = check_dev_ptrs({Q, K, V, O, dO, dQ, dK, dV}, 16)) return r;
     if (int r = check_dev_ptrs({lse}, 4)) return r;
