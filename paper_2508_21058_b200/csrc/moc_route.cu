@@ -491,8 +491,8 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 } else {
                 // Best-first extraction: up to k members of a 32-column block can enter the list; they are taken one
                 // per round, the block's best first, while any row of the warp still has one above its k-th score.
-                auto extract_blocks = [&]() {
-                for (int cc = 0; cc < rows_sb; cc += 32) {
+                auto extract_blocks = [&](int cc0, int cc1) {
+                for (int cc = cc0; cc < cc1; cc += 32) {
                     uint32_t v[32];
                     tmem_ld32(acc + cc, v);
                     const int j0 = sb * p.sb_rows + cc;
@@ -548,12 +548,12 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                 // more survivors than slots (many equal scores) sends its warp through the best-first extraction
                 // instead, which needs no queue.  A block all of whose columns are candidates for all 32 rows (most
                 // blocks: the candidates are a prefix of the columns) skips the candidate masks.
-                bool fast = KMAX <= 16 && p.surv_cap > 0;
+                bool fast = p.surv_cap > 0;
                 if (fast) {
                     constexpr int G = KMAX <= 8 ? 16 : 32;
                     const int jb = sb * p.sb_rows;
                     float thr = kth;
-                    if (sb == 0) {
+                    if (KMAX <= 16 && sb == 0) {
                         float gm[G];
 #pragma unroll
                         for (int x = 0; x < G; ++x) gm[x] = -INFINITY;
@@ -620,21 +620,28 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                     // instruction runs on the multiply-add pipe, while the compares around it fill the other one
                     int one;
                     asm volatile("mov.u32 %0, 1;" : "=r"(one));
-#pragma unroll 1
-                    for (int b = 0; b < half; ++b) {
-                        const bool two = b + half < nblk;
-                        const int cl = b * 32, ch = (b + half) * 32;
+                    // the 32-column blocks at cl (front stream) and, if `two`, at ch (back stream): survivors into the queue
+                    auto scan = [&](int cl, int ch, bool two) {
                         uint32_t vl[32], vh[32];
                         tmem_ld32(acc + cl, vl);
                         if (two) tmem_ld32(acc + ch, vh);
                         const uint32_t cand_l = cand_bits(jb + cl), cand_h = two ? cand_bits(jb + ch) : 0u;
                         tmem_wait_ld();
-                        const bool plain = __all_sync(0xffffffffu, cand_l == 0xffffffffu && (!two || cand_h == 0xffffffffu));
+                        const bool later_pass = KMAX == 64 && pass > 0;
+                        const bool plain = !later_pass && __all_sync(0xffffffffu, cand_l == 0xffffffffu && (!two || cand_h == 0xffffffffu));
                         if (!plain) {
 #pragma unroll
                             for (int c = 0; c < 32; ++c) {
                                 vl[c] = ((cand_l >> c) & 1u) ? vl[c] : 0xff800000u;      // -inf
                                 vh[c] = ((cand_h >> c) & 1u) ? vh[c] : 0xff800000u;
+                            }
+                            if (later_pass) {               // only what comes after the previous pass's last pick
+#pragma unroll
+                                for (int c = 0; c < 32; ++c) {
+                                    const float fl = __uint_as_float(vl[c]), fh = __uint_as_float(vh[c]);
+                                    vl[c] = (fl < prev_s || (fl == prev_s && jb + cl + c > prev_j)) ? vl[c] : 0xff800000u;
+                                    vh[c] = (fh < prev_s || (fh == prev_s && jb + ch + c > prev_j)) ? vh[c] : 0xff800000u;
+                                }
                             }
                         }
                         if (two) {
@@ -678,10 +685,13 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                                     : "r"(cl + c), "f"(__uint_as_float(vl[c])), "f"(thr), "r"(lo_end), "r"(one)
                                     : "memory");
                         }
-                    }
-                    const int cnt_lo = (int)(lo_v - q_v) >> 9, cnt_hi = (int)(q_v + (cap - 1) * 512 - hi_v) >> 9;
-                    fast = !__any_sync(0xffffffffu, cnt_lo + cnt_hi > cap);
-                    if (fast) {
+                    };
+                    // the queue's survivors into the list (front stream, then back stream: column order), unless a
+                    // row of the warp has more than fit; the cursors start again
+                    auto drain = [&]() -> bool {
+                        const int cnt_lo = (int)(lo_v - q_v) >> 9, cnt_hi = (int)(q_v + (cap - 1) * 512 - hi_v) >> 9;
+                        lo_v = q_v; lo_j = q_j; hi_v = q_v + (cap - 1) * 512; hi_j = q_j + (cap - 1) * 128;
+                        if (__any_sync(0xffffffffu, cnt_lo + cnt_hi > cap)) return false;
                         // every row's e-th survivor goes into its list together; a row that has none left inserts
                         // -inf, which changes nothing, so there is no branch; the next survivor is fetched ahead
                         const int nlo = __reduce_max_sync(0xffffffffu, cnt_lo), nhi = __reduce_max_sync(0xffffffffu, cnt_hi);
@@ -699,9 +709,29 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                             insert(cv, cj);
                         }
                         update_kth();
+                        return true;
+                    };
+                    if (KMAX <= 16) {
+                        // one scan of the whole step against the threshold found above, then one drain
+#pragma unroll 1
+                        for (int b = 0; b < half; ++b) scan(b * 32, (b + half) * 32, b + half < nblk);
+                        fast = drain();
+                    } else {
+                        // Long lists: no group maxima (a list of k needs more groups than registers hold); the columns
+                        // go 64 at a time against the list's own k-th score, which rises as they go: after n columns
+                        // about k / n of the next ones survive.  A pair of blocks whose survivors do not fit the
+                        // queue (the first ones, when everything survives and the queue is short) is extracted
+                        // best-first instead.
+#pragma unroll 1
+                        for (int b0 = 0; b0 < nblk; b0 += 2) {
+                            thr = fmaxf(kth, -FLT_MAX);
+                            const bool two = b0 + 1 < nblk;
+                            scan(b0 * 32, (b0 + 1) * 32, two);
+                            if (!drain()) extract_blocks(b0 * 32, min(rows_sb, (b0 + 2) * 32));
+                        }
                     }
                 }
-                if (!fast) extract_blocks();
+                if (!fast) extract_blocks(0, rows_sb);
                 }
                 tc_fence_before();
                 mbar_arrive(bar(ACC_EMPTY + sg));
@@ -995,16 +1025,20 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         a.n_pass = p->k > 64 ? (p->k + 63) / 64 : 1;
         // one histogram per group, the list offsets, and one byte per unit of a CTA
         const size_t hist = (ng * (p->k <= 8 && p->C <= kRtDeferredChunks ? 4 : 1) + 1) * sizeof(int) * (size_t)p->C + sizeof(int) * (size_t)p->ncol +
-                            4 * (size_t)(a.tiles_per_head / a.ctas_per_head + 16), budget = 227 * 1024 - 1024;
+                            4 * (size_t)(a.tiles_per_head / a.ctas_per_head + 16),
+                     budget = 227 * 1024 - 1024 - 512;      // what an SM has, less the alignment slack and the kernel's static variables
         if (d_block + q_tile + hist > budget) return MOC_ERR_SHAPE;
-        // threshold selection (lists of at most 16 picks, not the few-chunk case): survivor slots per row, as many
-        // as fit beside two Q stages, at least k + 4 (else the best-first extraction alone is used)
+        // threshold selection (not the few-chunk case): survivor slots per row, as many as fit beside two Q stages
+        // (too few: the best-first extraction alone is used)
         a.surv_cap = 0;
         size_t surv = 0;
-        if (!few && p->k <= 16 && budget > d_block + hist + 2 * q_tile + 16) {
+        if (!few && budget > d_block + hist + 2 * q_tile + 16) {
             const size_t room = budget - d_block - hist - 2 * q_tile - 16, per_slot = (size_t)ng * 160 * sizeof(float);
-            const int want = std::max(12, 2 * p->k + 4), have = (int)std::min<size_t>(room / per_slot, 255);
-            if (have >= p->k + 4) a.surv_cap = std::min(want, have);
+            // short lists: one scan per scoring step, a few more than k survive; long lists: 64 columns at a time,
+            // all of which survive at first
+            const int want = p->k <= 16 ? std::max(12, 2 * p->k + 4) : 64, need = p->k <= 16 ? p->k + 4 : 32;
+            const int have = (int)std::min<size_t>(room / per_slot, 255);
+            if (have >= need) a.surv_cap = std::min(want, have);
             surv = 16 + a.surv_cap * per_slot;
         }
         a.q_stages = (int)std::min<size_t>(4, (budget - d_block - hist - surv) / q_tile);
