@@ -366,15 +366,17 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                 uint4 *part16 = reinterpret_cast<uint4 *>(p.part);
                 if (MODE == DQ_ROUTED) {
                     if (qi >= 0) {
+                        uint4 out[4];
 #pragma unroll
                         for (int q4 = 0; q4 < 4; ++q4) {
-                            uint4 out;
-                            out.x = bf16x2(acc[q4 * 8 + 0], acc[q4 * 8 + 1]);
-                            out.y = bf16x2(acc[q4 * 8 + 2], acc[q4 * 8 + 3]);
-                            out.z = bf16x2(acc[q4 * 8 + 4], acc[q4 * 8 + 5]);
-                            out.w = bf16x2(acc[q4 * 8 + 6], acc[q4 * 8 + 7]);
-                            part16[part_piece(h - p.h0, LB, p.k, NP, qi, slot, ch * 4 + q4)] = out;
+                            out[q4].x = bf16x2(acc[q4 * 8 + 0], acc[q4 * 8 + 1]);
+                            out[q4].y = bf16x2(acc[q4 * 8 + 2], acc[q4 * 8 + 3]);
+                            out[q4].z = bf16x2(acc[q4 * 8 + 4], acc[q4 * 8 + 5]);
+                            out[q4].w = bf16x2(acc[q4 * 8 + 6], acc[q4 * 8 + 7]);
                         }
+                        // whole 32-byte sectors (pairs of pieces)
+                        st_256(part16 + part_piece(h - p.h0, LB, p.k, NP, qi, slot, ch * 4), out[0], out[1]);
+                        st_256(part16 + part_piece(h - p.h0, LB, p.k, NP, qi, slot, ch * 4 + 2), out[2], out[3]);
                     }
                 } else if (MODE == DQ_ANCHOR) {
                     if (qi >= 0) {
@@ -387,8 +389,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attend_bwd_tc_kernel(const __g
                             for (int u = 0; u < 4; ++u) {
                                 const bool used = s0 + u < p.k && pl[s0 + u] != -INFINITY;
 #pragma unroll
-                                for (int q4 = 0; q4 < 4; ++q4)
-                                    raw[u][q4] = used ? __ldcg(part16 + part_piece(h - p.h0, LB, p.k, NP, qi, s0 + u, ch * 4 + q4)) : make_uint4(0, 0, 0, 0);
+                                for (int q4 = 0; q4 < 4; q4 += 2) {
+                                    raw[u][q4] = raw[u][q4 + 1] = make_uint4(0, 0, 0, 0);
+                                    if (used) ld_cg_256(part16 + part_piece(h - p.h0, LB, p.k, NP, qi, s0 + u, ch * 4 + q4), raw[u][q4], raw[u][q4 + 1]);
+                                }
                             }
 #pragma unroll
                             for (int u = 0; u < 4; ++u)
