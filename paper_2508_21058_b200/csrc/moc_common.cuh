@@ -58,6 +58,7 @@ struct moc_plan {
     float scale;
     int device;
     int n_sm;
+    bool pool_direct = false;    // descriptors by one block per (head, chunk): every block resident at once, no long chunk
     std::vector<int32_t> off, shot;
     std::vector<uint8_t> mod;
     // host-side derived tables

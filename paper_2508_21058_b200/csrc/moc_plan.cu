@@ -167,6 +167,11 @@ extern "C" int moc_plan_create(const moc_problem *pr, moc_plan **out) {
         for (int u = 0; u < units; ++u) unit_chunk.push_back(c);
     }
     p->n_pool_units = p->pool_unit_off[C];
+    {
+        int longest = 0;
+        for (int c = 0; c < C; ++c) longest = std::max(longest, p->off[c + 1] - p->off[c]);
+        p->pool_direct = (int64_t)p->H * C <= 8LL * p->n_sm && C <= 65535 && longest <= 4096;
+    }
     // Key tiles of the backward's key-stationary pass.  A tile's block streams every query that attends its chunk:
     // the rows of the chunks that have it as an anchor (known here) and the routed list.  Tiles of chunks whose
     // anchor rows are far above the average (a caption, which every query attends) go first, for all heads, so

@@ -93,12 +93,71 @@ __global__ void __launch_bounds__(256) chunk_pool_kernel(const __nv_bfloat16 *__
     }
 }
 
+// The same stream with one block per (head, chunk): no partial sums, no arrival counters, so nothing has to be
+// cleared first.  Used when every block is resident at once (few enough chunks) and no chunk is long.
+template <int D>
+__global__ void __launch_bounds__(256) chunk_pool_direct_kernel(const __nv_bfloat16 *__restrict__ K, float *__restrict__ desc,
+                                                                 const int32_t *__restrict__ off, int L, int C) {
+    constexpr int LANES = D / 8;          // 16-byte lanes per token row
+    constexpr int ROWS = 256 / LANES;     // rows per pass
+    __shared__ float red[ROWS][D + 4];
+    const int c = blockIdx.x, h = blockIdx.y;
+    const int lane = threadIdx.x % LANES, rg = threadIdx.x / LANES;
+    const int t0 = off[c], t1 = off[c + 1];
+    float acc[8];
+#pragma unroll
+    for (int x = 0; x < 8; ++x) acc[x] = 0.f;
+    const uint4 *base = reinterpret_cast<const uint4 *>(K + ((size_t)h * L) * D) + lane;
+    int t = t0 + rg;
+    for (; t + 3 * ROWS < t1; t += 4 * ROWS) {          // 4 independent 16-byte loads in flight per thread
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = __ldg(base + (size_t)(t + u * ROWS) * LANES);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&v[u]);
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                float2 f = __bfloat1622float2(b[x]);
+                acc[2 * x] += f.x;
+                acc[2 * x + 1] += f.y;
+            }
+        }
+    }
+    for (; t < t1; t += ROWS) {
+        uint4 v = __ldg(base + (size_t)t * LANES);
+        const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&v);
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            float2 f = __bfloat1622float2(b[x]);
+            acc[2 * x] += f.x;
+            acc[2 * x + 1] += f.y;
+        }
+    }
+#pragma unroll
+    for (int x = 0; x < 8; ++x) red[rg][lane * 8 + x] = acc[x];
+    __syncthreads();
+    if (threadIdx.x < D) {
+        float s = 0.f;
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) s += red[r][threadIdx.x];       // fixed order: the result does not depend on scheduling
+        desc[((size_t)h * C + c) * D + threadIdx.x] = s / (float)(t1 - t0);
+    }
+}
+
 __global__ void zero_i32_kernel(int *p, size_t n) {
     size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
     if (i < n) p[i] = 0;
 }
 
 int launch_chunk_pool(const moc_plan *p, const __nv_bfloat16 *K, float *desc, void *ws, cudaStream_t s) {
+    if (p->pool_direct) {
+        dim3 grid((unsigned)p->C, (unsigned)p->H);
+        if (p->d == 128) chunk_pool_direct_kernel<128><<<grid, 256, 0, s>>>(K, desc, p->d_off, p->L, p->C);
+        else chunk_pool_direct_kernel<64><<<grid, 256, 0, s>>>(K, desc, p->d_off, p->L, p->C);
+        MOC_LAUNCH_CHECK();
+        return MOC_OK;
+    }
     float *part = ws_ptr<float>(ws, p->ws.pool_part);
     int *done = ws_ptr<int>(ws, p->ws.pool_done);
     // the arrival counters live in caller-owned scratch whose contents are unknown

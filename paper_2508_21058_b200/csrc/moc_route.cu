@@ -84,6 +84,8 @@ __global__ void route_prep_kernel(const float *__restrict__ desc, __nv_bfloat16 
 }
 
 struct RouteParams {
+    const float *desc;      // few-chunk case: the fp32 descriptors, split into their three terms by the kernel itself (else nullptr)
+    unsigned wait_us;       // limit of the bounded waits, stated in the status words by the kernel in that case
     int32_t *sel;
     float *part_lse;
     int *cnt;
@@ -153,6 +155,7 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
 
     if (threadIdx.x == 0) {
         s_abort = 0;
+        if (FEW && p.desc) p.status[ST_WAIT_US] = (int)p.wait_us;       // every block writes the same value, before any of its waits
         for (int t = 0; t < kMaxStages; ++t) { mbar_init(bar(Q_FULL + t), 1); mbar_init(bar(Q_EMPTY + t), 1); }
         mbar_init(bar(D_FULL), 1);
         mbar_init(bar(D_EMPTY), 1);
@@ -187,6 +190,41 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
         const int reach = chunks_in_reach(p, unit_of(x));
         s_unit[x] = (uint32_t)reach | (uint32_t)max(1, (reach + p.sb_rows - 1) / p.sb_rows) << 16 | (uint32_t)(x % p.q_stages) << 24 |
                     (uint32_t)((x / p.q_stages) & 1) << 28;
+    }
+    if (FEW && p.desc) {
+        // Few chunks: the head's descriptor block is small enough for the block to split it into its three bf16 terms
+        // itself, straight into the swizzled operand layout (what the copy of the pre-split block would have
+        // written), which saves the launch that prepares the split block.  One 16-byte piece (8 columns) per thread.
+        constexpr int PIECES = D / 8;
+        for (int x = threadIdx.x; x < p.c_pad * PIECES; x += kRtThreads) {
+            const int col = x / PIECES, pc = x % PIECES;
+            float v[8];
+#pragma unroll
+            for (int y = 0; y < 8; ++y) v[y] = 0.f;
+            if (col < p.ncol) {
+                const float4 *src = reinterpret_cast<const float4 *>(p.desc + ((size_t)h * p.C + p.col_chunk[col]) * D + pc * 8);
+                const float4 a = __ldg(src), b = __ldg(src + 1);
+                v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+            }
+            uint32_t t3[3][4];
+#pragma unroll
+            for (int y = 0; y < 4; ++y) {
+                float r0 = v[2 * y], r1 = v[2 * y + 1];
+#pragma unroll
+                for (int term = 0; term < 3; ++term) {
+                    const __nv_bfloat16 b0 = __float2bfloat16_rn(r0), b1 = __float2bfloat16_rn(r1);
+                    r0 -= __bfloat162float(b0);
+                    r1 -= __bfloat162float(b1);
+                    t3[term][y] = (uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16);
+                }
+            }
+            const int sub = pc >> 3, c16 = pc & 7;
+#pragma unroll
+            for (int term = 0; term < 3; ++term)
+                *reinterpret_cast<uint4 *>(gbase + (sub * 3 + term) * d_sub_bytes + sw128_offset(col, c16)) =
+                    make_uint4(t3[term][0], t3[term][1], t3[term][2], t3[term][3]);
+        }
+        fence_proxy_async_smem();       // the tensor core reads these through the async proxy
     }
     auto reach_of = [&](int n) { return (int)(s_unit[n] & 0xffffu); };
     auto steps_of = [&](int n) { return (int)((s_unit[n] >> 16) & 0xffu); };
@@ -227,12 +265,16 @@ __global__ void __launch_bounds__(rt_threads(NG), 1) route_tc_kernel(const __gri
                     if (resident ? dn == 0 : sb != res_sb) {
                         ok = mbar_wait(bar(D_EMPTY), (dn & 1) ^ 1, abort_flag, p.status, RW_DEMPTY);
                         if (!ok) break;
-                        mbar_expect_tx(bar(D_FULL), 3 * SUB * d_sub_bytes);
-                        for (int term = 0; term < 3; ++term)
+                        if (FEW && p.desc) {
+                            mbar_arrive(bar(D_FULL));       // the block wrote the terms itself, before the roles parted
+                        } else {
+                            mbar_expect_tx(bar(D_FULL), 3 * SUB * d_sub_bytes);
+                            for (int term = 0; term < 3; ++term)
 #pragma unroll
-                            for (int sub = 0; sub < SUB; ++sub)
-                                tma_load_2d(sD + (sub * 3 + term) * d_sub_bytes, &tmD, sub * 64,
-                                            (h * 3 + term) * p.c_pad + (resident ? 0 : sb * p.sb_rows), bar(D_FULL));
+                                for (int sub = 0; sub < SUB; ++sub)
+                                    tma_load_2d(sD + (sub * 3 + term) * d_sub_bytes, &tmD, sub * 64,
+                                                (h * 3 + term) * p.c_pad + (resident ? 0 : sb * p.sb_rows), bar(D_FULL));
+                        }
                         ++dn;
                         res_sb = sb;
                     }
@@ -994,13 +1036,20 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
     int *cnt = ws_ptr<int>(ws, p->ws.cnt);
     int *status = ws_ptr<int>(ws, p->ws.status);
     __nv_bfloat16 *desc3 = ws_ptr<__nv_bfloat16>(ws, p->ws.desc3);
-    {
+    // Few chunks: the routing kernel splits the descriptors itself, and the status words and pick counters (next to
+    // each other in the workspace) are cleared by one memset instead of a kernel.
+    const bool few = p->k > 0 && p->c_pad <= 32 && p->k <= 8;
+    const bool fused_prep = few && (reinterpret_cast<uintptr_t>(desc) & 15) == 0 && p->ws.cnt > p->ws.status;
+    if (fused_prep) {
+        MOC_CUDA_TRY(cudaMemsetAsync(status, 0, (p->ws.cnt - p->ws.status) + sizeof(int) * (size_t)p->H * p->C, s));
+    } else {
         const size_t n = std::max((size_t)p->H * p->c_pad * D, (size_t)kStatusWords);   // covers H * C too
         route_prep_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(desc, desc3, cnt, status, p->d_col_chunk, p->H, p->C, p->ncol, p->c_pad, D, p->wait_us);
         MOC_LAUNCH_CHECK();
     }
     if (p->k > 0) {
         RouteParams a;
+        a.desc = fused_prep ? desc : nullptr; a.wait_us = p->wait_us;
         a.sel = sel; a.part_lse = ws_ptr<float>(ws, p->ws.part_lse); a.cnt = cnt;
         a.qlist = ws_ptr<int32_t>(ws, p->ws.qlist);
         a.tok_chunk = p->d_tok_chunk; a.cand_c = p->d_cand_c; a.lim = p->d_lim; a.reach = p->d_reach;
@@ -1020,7 +1069,6 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
         const unsigned grid = (unsigned)(p->H * a.ctas_per_head);
         // Four selection groups with few chunks (more warps to hide the selection's latencies); one when the
         // 64-entry list takes nearly all of a thread's registers; two otherwise.
-        const bool few = p->c_pad <= 32 && p->k <= 8;
         const int ng = few ? 4 : p->k > 32 ? 1 : 2;
         a.n_pass = p->k > 64 ? (p->k + 63) / 64 : 1;
         // one histogram per group, the list offsets, and one byte per unit of a CTA
