@@ -7,6 +7,8 @@
 // and writes one partial sum.  The last block to finish a chunk (arrival counter)
 // adds the partials in slice order and scales by 1/n, so the result does not depend
 // on block scheduling.
+// With few (head, chunk) pairs and no long chunk one block takes a whole chunk
+// (chunk_pool_direct_kernel): no partial sums and no counters.
 #include <mutex>
 
 #include "moc_common.cuh"

@@ -8,7 +8,8 @@
 // (hi + mid + lo carries its 24-bit mantissa), and S = Q hi^T + Q mid^T + Q lo^T is
 // accumulated in fp32 in TMEM: every product is exact, only the fp32 accumulation rounds.
 //
-// route_prep_kernel   splits the descriptors, clears the pick counters and the status words.
+// route_prep_kernel   splits the descriptors, clears the pick counters and the status words (few chunks: the
+//                     routing kernel splits them itself and a memset does the clearing).
 // route_tc_kernel     H x (SMs / H) CTAs; the 128-query tiles ("units") of a head are dealt round-robin
 //                     to the head's CTAs:
 //     warp 0      TMA producer: Q tiles (ring of stages) and the head's descriptor block;
