@@ -1085,7 +1085,7 @@ static int launch_route_d(const moc_plan *p, const __nv_bfloat16 *Q, const float
             const size_t room = budget - d_block - hist - 2 * q_tile - 16, per_slot = (size_t)ng * 160 * sizeof(float);
             // short lists: one scan per scoring step, a few more than k survive; long lists: 64 columns at a time,
             // all of which survive at first
-            const int want = p->k <= 16 ? std::max(12, 2 * p->k + 4) : 64, need = p->k <= 16 ? p->k + 4 : 32;
+            const int want = p->k <= 16 ? std::max(12, 2 * p->k + 12) : 64, need = p->k <= 16 ? p->k + 4 : 32;
             const int have = (int)std::min<size_t>(room / per_slot, 255);
             if (have >= need) a.surv_cap = std::min(want, have);
             surv = 16 + a.surv_cap * per_slot;
