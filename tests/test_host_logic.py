@@ -87,3 +87,50 @@ def test_plan_rejects_bad_arguments_without_a_device():
     with pytest.raises(MocError) as e:
         MocPlan(2, lay.n_tokens, 64, lay.chunk_off, lay.chunk_shot, lay.chunk_mod, 600)
     assert e.value.code == -2
+
+
+def test_roofline_objects_follow_from_the_segment_times():
+    """The fractions the benchmark prints are plain arithmetic on the segment times, the pair count and the
+    peaks: recomputed here by hand; the attention peak is the sustained one only for a long timed region."""
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2508_21058_b200 import workloads as W
+    wl = W.workload("cfg1")
+    peaks = {"hbm_gbs": 6000.0, "bf16_tflops": 1600.0, "bf16_tflops_sustained": 1400.0}
+    pairs = 5_000_000_000
+    r = {"seg": [0.05, 0.06, 3.5], "pairs": pairs, "timed_ms": 80.0}
+    roof, routing = bench.rooflines(wl, r, peaks, "measured")
+    att = 4.0 * wl.head_dim * pairs / 3.5e-3 / 1e12
+    assert roof["achieved"] == pytest.approx(att) and roof["peak"] == 1600.0
+    assert roof["frac"] == pytest.approx(att / 1600.0) == pytest.approx(roof["frac_of_burst"])
+    assert roof["frac_of_sustained"] == pytest.approx(att / 1400.0)
+    H, L, d, C, k = wl.n_heads, wl.n_tokens, wl.head_dim, wl.n_chunks, wl.top_k
+    bytes_ = 2.0 * 2 * L * d * H + 4.0 * k * L * H + 2 * 4.0 * C * d * H
+    assert routing["achieved"] == pytest.approx(bytes_ / 0.11e-3 / 1e9)
+    assert routing["frac"] == pytest.approx(routing["achieved"] / 6000.0)
+    roof_long, _ = bench.rooflines(wl, dict(r, timed_ms=1300.0), peaks, "measured")
+    assert roof_long["peak"] == 1400.0 and roof_long["frac"] == pytest.approx(att / 1400.0)
+
+
+def test_traffic_figure_is_dropped_when_the_kernel_source_has_changed(tmp_path, monkeypatch):
+    sys.path.insert(0, ROOT)
+    import hashlib
+    import bench
+    (tmp_path / "profiles").mkdir()
+    (tmp_path / "k.cu").write_text("kernel v1")
+    sha = hashlib.sha1(b"kernel v1").hexdigest()
+    (tmp_path / "profiles" / "traffic.txt").write_text(f"# comment\nmoc_attend cfgX 1.5e+09 {sha} k.cu\n")
+    monkeypatch.setattr(bench, "ROOT", str(tmp_path))
+    assert bench.measured_traffic("moc_attend", "cfgX") == 1.5e9
+    assert bench.measured_traffic("moc_attend", "other") is None
+    (tmp_path / "k.cu").write_text("kernel v2")
+    assert bench.measured_traffic("moc_attend", "cfgX") is None
+
+
+def test_both_arms_describe_the_workload_with_the_same_config():
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2508_21058_b200 import workloads as W
+    wl = W.workload("cfg2")
+    a, b = bench.config_of(wl, False, 1), bench.config_of(W.workload("cfg2"), False, 1)
+    assert a == b and a["workload"] == "cfg2" and a["tokens"] == 264128 and a["top_k"] == 6 and a["backward"] is False
