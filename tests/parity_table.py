@@ -1,5 +1,5 @@
-"""Turns the per-workload parity records that the GPU tests leave (``gpurun_out/parity/*.json`` or
-``$MOC_PARITY_DIR``) into one markdown table:  python tests/parity_table.py > profiles/parity_full_size.md"""
+"""Turns the per-workload parity records that the GPU tests leave (one JSON per workload in the parity records
+folder, ``$MOC_PARITY_DIR`` if set) into one markdown table:  python tests/parity_table.py > profiles/parity_full_size.md"""
 import glob
 import json
 import os
@@ -9,14 +9,14 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def main():
-    src = os.environ.get("MOC_PARITY_DIR", os.path.join(ROOT, "gpurun_out", "parity"))
+    src = os.environ.get("MOC_PARITY_DIR", os.path.join(ROOT, "gpurun_out", "parity"))      # the default of tests/parity_utils.py
     recs = {os.path.basename(f)[:-5]: json.load(open(f)) for f in sorted(glob.glob(os.path.join(src, "*.json")))}
     order = [n for n in ("cfg0", "cfg1", "cfg2", "cfg4") if n in recs] + sorted(n for n in recs if n.startswith("cfg3")) + \
         sorted(n for n in recs if not n.startswith("cfg"))
     out = ["# Parity of the CUDA path against the fp64 oracle, per workload",
            "",
            "Written by `python tests/parity_table.py` from the records that `python -m pytest tests -m gpu` leaves under",
-           "`gpurun_out/parity/` (one B200).  Routing is compared on EVERY row of the heads listed; a near-tie row is one whose",
+           "the parity records folder (one B200).  Routing is compared on EVERY row of the heads listed; a near-tie row is one whose",
            "GPU and oracle pick sets differ only in chunks whose oracle score lies within 1e-4 of the oracle's k-th score;",
            "`order` counts rows with equal sets whose order differs (`~` inside the near-tie window, `!` beyond it - must be 0).",
            "Attention is compared on sampled rows (half chunk edges, half uniform) at the full-size workloads and on every row",

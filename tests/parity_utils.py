@@ -6,7 +6,7 @@ poisoned guard bands that are verified after the calls: a kernel that writes out
 buffer fails the test even when the stray write lands in memory nobody reads.
 
 Every comparison can be recorded (``report``): one JSON file per workload under
-``gpurun_out/parity/`` (or ``$MOC_PARITY_DIR``) with the rows compared, the near-tie and
+the parity records folder (``PARITY_DIR``: ``$MOC_PARITY_DIR`` if set) with the rows compared, the near-tie and
 hard-mismatch counts and the error figures, from which the committed parity table is made."""
 from __future__ import annotations
 
@@ -30,6 +30,8 @@ GUARD = 4096
 POISON = 0xA5
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+OUT_ROOT = os.path.join(ROOT, "gpurun_out")          # where a run leaves its outputs
+PARITY_DIR = os.environ.get("MOC_PARITY_DIR", os.path.join(OUT_ROOT, "parity"))
 
 
 def near_tie_budget(n_rows: int) -> int:
@@ -38,7 +40,7 @@ def near_tie_budget(n_rows: int) -> int:
 
 def report(workload: str, section: str, values: dict):
     """Merge `values` under `section` into the workload's parity record."""
-    out_dir = os.environ.get("MOC_PARITY_DIR", os.path.join(ROOT, "gpurun_out", "parity"))
+    out_dir = PARITY_DIR
     try:
         os.makedirs(out_dir, exist_ok=True)
         path = os.path.join(out_dir, f"{workload}.json")

@@ -238,6 +238,6 @@ def test_debug_build_checks_every_workspace_index_and_finds_nothing():
     ) % (ROOT, os.path.join(ROOT, "tests"))
     from paper_2508_21058_b200 import build as libbuild
     libbuild.build(debug=True)                  # a no-op when libmoc_debug.so is up to date with the sources
-    env = dict(os.environ, MOC_LIBRARY="debug", MOC_PARITY_DIR=os.path.join(ROOT, "gpurun_out", "parity_debug"))
+    env = dict(os.environ, MOC_LIBRARY="debug", MOC_PARITY_DIR=os.path.join(PU.OUT_ROOT, "parity_debug"))
     res = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, env=env, timeout=600)
     assert res.returncode == 0 and "DEBUG_BUILD_OK" in res.stdout, res.stdout[-2000:] + res.stderr[-4000:]
